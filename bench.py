@@ -1,0 +1,361 @@
+#!/usr/bin/env python
+"""Benchmark of the AdaCons aggregation hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload bert64] [--impl ours|reference]
+
+One "step" = one adacons_aggregate call (pass 1 + coefficient step + pass 2) on one N x d matrix
+of synthetic worker gradients that is already resident in HBM.  Rank 0 prints ONE JSON line.
+
+--gpus N > 1 (launched by torch.distributed.run): the aggregation of one matrix does not shard
+across GPUs in this library, so every rank runs an independent replica of the same workload
+(different seed); `value` = elements aggregated by all ranks / max-over-ranks time.
+
+--impl reference times the float64 CPU oracle (oracle/), as it stands, on the host cores on a
+bounded column sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "aggregated_grad_elements_per_s"
+UNIT = "elements/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+ORACLE_SAMPLE_COLUMNS = 2_000_000      # --impl reference: columns per step
+CPU_BASELINE_COLUMNS = 4_000_000       # cpu_baseline leg of the CUDA arm: 3 steps of this many columns
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
+# profiles/, as a multiple of the algorithmic bytes of that kernel (None = no capture for the
+# current kernel).
+NCU_TRAFFIC_RATIO = {"pass1": None, "pass2": None}
+
+
+def parse_args(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="bert64")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--d", type=int, default=0, help="override the gradient length (debugging)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args(argv)
+
+
+# ------------------------------------------------------------------------------------------------
+# multi-process plumbing (replicas only)
+# ------------------------------------------------------------------------------------------------
+def dist_setup(n_gpus: int, use_cuda: bool):
+    """Returns (rank, world, local_rank).  Initialises torch.distributed when world > 1."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29511")
+        if not dist.is_initialized():
+            dist.init_process_group(backend="nccl" if use_cuda else "gloo", rank=rank, world_size=world)
+    return rank, world, local
+
+
+def reduce_over_ranks(ms_local: float, units_local: float, device="cpu"):
+    """Whole-job figures for independent replicas: (max over ranks of the time, sum of units)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms_local), float(units_local)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# ------------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def _reasons(self):
+        nv = self.nv
+        try:
+            get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+            mask = get(self.h)
+        except Exception:
+            return
+        names = {
+            "sw_power_cap": 0x4, "hw_slowdown": 0x8, "sync_boost": 0x10, "sw_thermal_slowdown": 0x20,
+            "hw_thermal_slowdown": 0x40, "hw_power_brake_slowdown": 0x80, "applications_clocks_setting": 0x2,
+            "display_clock_setting": 0x100,
+        }
+        for k, bit in names.items():
+            if mask & bit:
+                self.reasons.add(k)
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                self._reasons()
+            except Exception:
+                pass
+            self._stop_evt.wait(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        s = sorted(self.samples)
+        return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def physical_gpu_index(local_index: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_index])
+        except Exception:
+            return local_index
+    return local_index
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy read+write)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_steps(w, steps: int, warmup: int, columns: int):
+    """Time oracle.step on a column sample of workload w; returns (mean seconds/step, elements/step)."""
+    import numpy as np  # noqa: F401
+    from oracle import adacons_oracle as oc
+    from paper_2411_03742_b200 import workloads as wl
+    ws = w.scaled(min(columns, w.d))
+    orc = oc.AdaConsOracle(ws.N, ws.d)
+    times = []
+    for t in range(warmup + steps):
+        G64 = wl.generate(ws, t, "cpu").to(dtype=__import__("torch").float64).numpy()
+        t0 = time.perf_counter()
+        orc.step(G64, storage=ws.dtype)
+        dt = time.perf_counter() - t0
+        if t >= warmup:
+            times.append(dt)
+    return sum(times) / len(times), ws.N * ws.d, ws
+
+
+def run_reference(args):
+    from paper_2411_03742_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = wl.WORKLOADS[args.workload]
+    if args.d:
+        w = w.scaled(args.d)
+    sec, elems, ws = oracle_sample_steps(w, args.steps, min(args.warmup, 1), ORACLE_SAMPLE_COLUMNS)
+    value = elems / sec
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": describe(w), "sample": f"first {ws.d} columns of every row, regenerated per step on the CPU"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"N={ws.N} x {ws.d} columns per step (float64 numpy, one thread; "
+                                   f"host has {os.cpu_count()} cores)"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def describe(w) -> str:
+    return (f"{w.name}: N={w.N} workers, d={w.d}, {w.dtype} storage / fp32 accumulate, {w.steps}-step recipe "
+            f"({w.note})")
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA library
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    from paper_2411_03742_b200 import binding as ac, workloads as wl
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU fallback")
+    rank, world, local = dist_setup(args.gpus, use_cuda=True)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    w = wl.WORKLOADS[args.workload]
+    if args.d:
+        w = w.scaled(args.d)
+    w_rank = __import__("dataclasses").replace(w, seed=w.seed + 100_000 * rank)
+
+    G = wl.generate(w_rank, 0, dev)
+    out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
+    h = ac.AdaCons(w.N, w.d, w.dtype, seg_offsets=wl.segment_offsets(w))
+    stream = torch.cuda.current_stream()
+
+    for _ in range(max(args.warmup, 3)):
+        h.aggregate(G, out)
+    torch.cuda.synchronize()
+    h.set_option(ac.OPT_PROFILE, 1)
+    launches0 = h.info(ac.INFO_TOTAL_LAUNCHES)
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        h.aggregate(G, out)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    barrier()
+    ms_local = ev0.elapsed_time(ev1)
+    launches = h.info(ac.INFO_TOTAL_LAUNCHES) - launches0
+    kernel_ms, kcalls = h.profile()
+    status = h.status()
+    assert status == 0, f"library raised status flags {status:#x}"
+    assert h.info(ac.INFO_LAST_PATH) == 1, "benchmark must run the fast path"
+
+    units_local = float(w.N) * w.d * args.steps
+    ms, units = reduce_over_ranks(ms_local, units_local, device=dev)
+    value = units / (ms * 1e-3)
+    b = w.elem_bytes
+    step_bytes = 2.0 * w.N * w.d * b + w.d * b
+    hbm_gbs = step_bytes * args.steps / (ms_local * 1e-3) / 1e9
+
+    # roofline of the dominant kernel, from CUDA events recorded around it inside the timed region
+    peak, peak_src = measured_peak_gbs()
+    alg = {"pass1": float(w.N) * w.d * b, "pass2": float(w.N) * w.d * b + w.d * b}
+    kms = {"pass1": kernel_ms[0], "coeff": kernel_ms[1], "pass2": kernel_ms[2]}
+    dom = "pass1" if kms["pass1"] >= kms["pass2"] else "pass2"
+    achieved = alg[dom] / (kms[dom] * 1e-3) / 1e9
+    ratio = NCU_TRAFFIC_RATIO.get(dom)
+    roofline = {
+        "bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+        "peak_source": peak_src, "traffic": (ratio * alg[dom] if ratio else None),
+        "algorithmic_bytes_per_launch": alg[dom], "kernel_ms": kms, "timed_calls": kcalls,
+        "other_kernel_gbs": {k: alg[k] / (kms[k] * 1e-3) / 1e9 for k in alg if k != dom},
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": describe(w), "N": w.N, "d": w.d, "storage_dtype": w.dtype,
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": f"inputs ({w.N * w.d * b / 1e9:.2f} GB) larger than the 126 MB L2; no flush between steps"},
+        "hbm_gbs": hbm_gbs, "hbm_frac_of_measured_copy": hbm_gbs / peak, "hbm_frac_of_nominal_8tbs": hbm_gbs / NOMINAL_HBM_GBS,
+        "minimal_bytes_per_step": step_bytes,
+        "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches),
+    }
+
+    # ---- end to end through the host-buffer entry point -----------------------------------------
+    if not args.no_e2e:
+        line["e2e"] = run_e2e(h, w, G, dev, args, world)
+    del G
+    # ---- CPU oracle on a bounded sample (rank 0, single GPU run only) ---------------------------
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sec, elems, ws = oracle_sample_steps(w, 3, 1, CPU_BASELINE_COLUMNS)
+        line["cpu_baseline"] = {"value": elems / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"3 steps of N={ws.N} x {ws.d} columns (float64 numpy, one thread; "
+                                          f"host has {os.cpu_count()} cores); {sec:.2f} s per step"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    h.close()
+    return 0
+
+
+def run_e2e(h, w, G, dev, args, world):
+    """adacons_aggregate_host: host -> device copy of the whole matrix, the three kernels, device ->
+    host copy of the result, every step, timed with the wall clock around the (synchronous) calls."""
+    import torch
+    b = w.elem_bytes
+    need = w.N * w.d * b
+    pinned = True
+    try:
+        with open("/proc/meminfo") as fh:
+            avail = next(int(l.split()[1]) * 1024 for l in fh if l.startswith("MemAvailable"))
+    except Exception:
+        avail = None
+    if avail is not None and avail < 1.5 * need * max(1, world):
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": need, "d2h_bytes_per_step": w.d * b,
+                "note": f"skipped: host has {avail / 1e9:.0f} GB available, needs {1.5 * need * world / 1e9:.0f} GB"}
+    try:
+        Gh = torch.empty((w.N, w.d), dtype=w.torch_dtype, pin_memory=True)
+        oh = torch.empty(w.d, dtype=w.torch_dtype, pin_memory=True)
+    except RuntimeError:
+        pinned = False
+        Gh = torch.empty((w.N, w.d), dtype=w.torch_dtype)
+        oh = torch.empty(w.d, dtype=w.torch_dtype)
+    Gh.copy_(G)
+    torch.cuda.synchronize()
+    steps = max(1, min(args.steps, 3))
+    h.aggregate_host(Gh, oh)          # warm-up: allocates the staging buffer
+    barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        h.aggregate_host(Gh, oh)
+    torch.cuda.synchronize()
+    sec_local = time.perf_counter() - t0
+    barrier()
+    ms, units = reduce_over_ranks(sec_local * 1e3, float(w.N) * w.d * steps, device=dev)
+    return {"value": units / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": need, "d2h_bytes_per_step": w.d * b,
+            "steps": steps, "ms_per_step": ms / steps, "pinned_host_memory": pinned,
+            "call": "adacons_aggregate_host (C ABI, host buffers)"}
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

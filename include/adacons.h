@@ -1,0 +1,194 @@
+/*
+ * adacons.h -- C ABI of the AdaCons gradient-aggregation library for NVIDIA B200 (sm_100a).
+ *
+ * AdaCons (arXiv 2411.03742, Section 3) aggregates the gradients g_1..g_N of N data-parallel
+ * workers into one direction psi_t = sum_i gamma_i g_i (Eq. 4, Eq. 12).  The weights come from
+ * a first-order step on the subspace spanned by the gradients (Eq. 5-7), smoothed over time by
+ * a momentum on the *sorted* coefficients (Eq. 11) and rescaled to sum to one (Eq. 12-13).
+ *
+ * One call of adacons_aggregate runs, entirely on the device and asynchronously on the
+ * caller's stream:
+ *   pass 1   one streaming read of the N x d matrix: column sums, p_i = <g_i, gbar>,
+ *            q_i = ||g_i||^2                                              (Eq. 7)
+ *   finish   fixed-order reduction of the per-block partial sums, a_i = p_i/sqrt(q_i),
+ *            sorted momentum, gamma_i                                     (Eq. 11, Eq. 12-13;
+ *                                                                          Algorithm 1, steps 2-3)
+ *   pass 2   a second streaming read: out_k = cast(sum_i gamma_i g_ik)   (Eq. 12; Algorithm 1, step 4)
+ *
+ * Conventions
+ *   - All functions return an adacons_error code (0 = success); none throws or aborts.
+ *   - "device pointer" = memory of the CUDA device that was current when the context was
+ *     created; "host pointer" = ordinary host memory.  `cuda_stream` is a cudaStream_t passed
+ *     as void* (NULL = the legacy default stream).
+ *   - Results are deterministic: the same inputs, state and options give the same bytes on the
+ *     same GPU model (no floating-point atomics, fixed reduction order).
+ *   - A context is not thread-safe; distinct contexts are independent.
+ *   - Numerical degeneracies (a zero gradient, a vanishing or negative normaliser, Inf/NaN in
+ *     the input) are not errors: the call completes with the documented fallback and raises a
+ *     flag that adacons_get_status returns.
+ */
+#ifndef ADACONS_H_
+#define ADACONS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct adacons_ctx adacons_ctx; /* opaque, owned by the library */
+
+/* Storage type of BOTH the gradient matrix and the result.  Accumulation is always fp32 inside
+ * a thread block and fp64 across blocks and in the coefficient step. */
+enum adacons_dtype { ADACONS_F32 = 0, ADACONS_BF16 = 1 };
+
+enum adacons_error {
+  ADACONS_OK = 0,
+  ADACONS_EINVAL = 1, /* bad argument (NULL, N < 1, d < 1, unknown enum, bad offsets, overlap) */
+  ADACONS_EALIGN = 2, /* reserved: misaligned buffers take a slower path instead of failing     */
+  ADACONS_ENOMEM = 3, /* device or host allocation failed                                       */
+  ADACONS_ECUDA = 4,  /* a CUDA runtime/driver call failed, or no CUDA device                   */
+  ADACONS_EARCH = 5,  /* the current device is not compute capability 10.x                      */
+  ADACONS_ETIMEOUT = 6 /* a bounded on-device wait gave up (reported by adacons_get_status)     */
+};
+
+/* Flags returned by adacons_get_status (OR over all segments since the last reset). */
+enum adacons_flag {
+  ADACONS_FLAG_ZERO_ROW = 1u,     /* some ||g_i|| = 0: that worker got weight 0                  */
+  ADACONS_FLAG_DEGENERATE_Z = 2u, /* sum_i u_i = 0 (|Z| <= 1e-12 sum|u_i|) or not finite:
+                                     gamma_i = 1/N (plain mean) was used                         */
+  ADACONS_FLAG_NONFINITE = 4u,    /* Inf/NaN statistic: gamma_i = 1/N, momentum state unchanged  */
+  ADACONS_FLAG_NEG_Z = 8u,        /* sum_i u_i < 0: computed as defined                          */
+  ADACONS_FLAG_TIMEOUT = 0x100u   /* a bounded wait inside a kernel expired; result is invalid   */
+};
+
+/* Options (adacons_set_option / adacons_get_option).  Variants follow the ablation in Table 2. */
+enum adacons_option {
+  ADACONS_OPT_BETA = 0,        /* momentum factor of Eq. 11, in [0,1); default 0.99 (Table 2)    */
+  ADACONS_OPT_MOMENTUM = 1,    /* 1 (default): apply Eq. 11; 0: a~ = a, state untouched          */
+  ADACONS_OPT_SORTED = 2,      /* 1 (default): sorted momentum, Eq. 11; 0: index EMA, Eq. 10     */
+  ADACONS_OPT_NORMALIZE = 3,   /* 1 (default): weights sum to one, Eq. 12-13;
+                                  0: lambda = 1 and the 1/N of Eq. 8, gamma_i = u_i / N          */
+  ADACONS_OPT_PER_SEGMENT = 4, /* 0 (default): one set of coefficients for the whole vector
+                                  ("model-wise"); 1: an independent set, with its own momentum
+                                  state, for each segment given to adacons_create ("layer-wise",
+                                  Section 4).  Changing it resets the state.                     */
+  ADACONS_OPT_PROFILE = 5      /* 0 (default) / 1: record CUDA events around each of the three
+                                  kernels of every aggregate call (see adacons_get_profile).
+                                  Setting it (to either value) clears the recorded samples.      */
+};
+
+/* Which N-vector adacons_get_coeffs returns (values of the most recent aggregate call). */
+enum adacons_coeff {
+  ADACONS_COEFF_A = 0,       /* a_i  = <g_i,gbar>/||g_i||            (Eq. 7)                      */
+  ADACONS_COEFF_A_TILDE = 1, /* a~_i after the momentum of Eq. 11                                */
+  ADACONS_COEFF_GAMMA = 2,   /* gamma_i, the weights applied in pass 2 (Eq. 12)                  */
+  ADACONS_COEFF_P = 3,       /* p_i  = <g_i,gbar>                                                 */
+  ADACONS_COEFF_Q = 4        /* q_i  = ||g_i||^2                                                  */
+};
+
+/* Read-only facts about a context (adacons_get_info). */
+enum adacons_info {
+  ADACONS_INFO_NUM_SEGMENTS = 0,     /* S given to create (1 if none)                            */
+  ADACONS_INFO_COEFF_SETS = 1,       /* 1 in model-wise mode, S in layer-wise mode               */
+  ADACONS_INFO_PASS1_BLOCKS = 2,     /* thread blocks of the pass-1 kernel (= partial-sum rows)  */
+  ADACONS_INFO_SCRATCH_BYTES = 3,    /* device bytes owned by the context                        */
+  ADACONS_INFO_LAUNCHES_PER_CALL = 4,/* kernels launched by one adacons_aggregate                */
+  ADACONS_INFO_LAST_PATH = 5,        /* 0 = none yet, 1 = TMA-staged fast path, 2 = generic path */
+  ADACONS_INFO_TOTAL_LAUNCHES = 6    /* kernels launched by this context so far                  */
+};
+
+/*
+ * Create a context for N workers and gradients of d elements of type `dtype`
+ * (problem statement: Eq. 4, psi_t : {g_i}_{i=1..N} -> R^d, stateful in t).
+ *   out          receives the context (host pointer, must not be NULL).
+ *   N            1 <= N <= 1024.
+ *   d            1 <= d < 2^31.
+ *   seg_offsets  host pointer to num_segments+1 ascending offsets with seg_offsets[0] = 0 and
+ *                seg_offsets[num_segments] = d (segments may be empty and need no alignment);
+ *                NULL / num_segments = 0 means one segment [0, d).  Copied; the caller keeps
+ *                ownership.  The segments matter only with ADACONS_OPT_PER_SEGMENT = 1.
+ * Allocates all device memory the context will ever need on the current device (state,
+ * coefficients, per-block partial sums) and zeroes the momentum state (alpha^m_0 = 0, t = 0).
+ * Errors: EINVAL, ENOMEM, ECUDA (no device / CUDA failure), EARCH (device is not sm_100).
+ */
+int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
+                   const int64_t *seg_offsets, int num_segments);
+
+/*
+ * Aggregate one set of gradients (Eq. 12; Algorithm 1 on a single device).
+ *   grads  device pointer, read-only: N rows of d elements, row-major and contiguous
+ *          (row i = g_i starts at element i*d).
+ *   out    device pointer, d elements of the same type; must not overlap grads.
+ *   Fast path: grads and out 16-byte aligned and d*sizeof(element) a multiple of 16, N <= 64.
+ *   Anything else is served by a slower generic path with the same results.
+ * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
+ * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.
+ * Errors: EINVAL (NULL pointers, overlap), ECUDA (launch failure).
+ */
+int adacons_aggregate(adacons_ctx *ctx, const void *grads, void *out, void *cuda_stream);
+
+/*
+ * The same aggregation for callers whose gradients live in HOST memory.
+ *   host_grads  host pointer, N x d row-major (pinned memory gives asynchronous copies).
+ *   host_out    host pointer, d elements.
+ * Copies the matrix to a device staging buffer owned by the context (allocated on first use,
+ * N*d elements + d elements), runs adacons_aggregate on it and copies the result back, all on
+ * `cuda_stream`; returns after synchronising that stream.  Errors: EINVAL, ENOMEM, ECUDA.
+ */
+int adacons_aggregate_host(adacons_ctx *ctx, const void *host_grads, void *host_out,
+                           void *cuda_stream);
+
+/* alpha^m := 0, t := 0, status flags cleared (asynchronous on the stream). */
+int adacons_reset(adacons_ctx *ctx, void *cuda_stream);
+
+/* Free the context and everything it owns.  The caller must make sure no work of this context
+ * is still running.  NULL is accepted. */
+int adacons_destroy(adacons_ctx *ctx);
+
+/* Options; see enum adacons_option.  Takes effect from the next aggregate call.
+ * Errors: EINVAL (unknown key, beta outside [0,1), per-segment requested without segments). */
+int adacons_set_option(adacons_ctx *ctx, int key, double value);
+int adacons_get_option(adacons_ctx *ctx, int key, double *value);
+
+/*
+ * Copy one coefficient vector of the most recent aggregate call to the host.
+ *   host   receives sets*N doubles, set-major (sets = ADACONS_INFO_COEFF_SETS).
+ * Synchronises `cuda_stream`.
+ */
+int adacons_get_coeffs(adacons_ctx *ctx, int which, double *host, void *cuda_stream);
+
+/*
+ * Momentum state for checkpoint / resume (Eq. 11): host_m receives / provides sets*N doubles,
+ * slot k of a set = EMA of the k-th smallest coefficient; *step = number of aggregations since
+ * the last reset.  Either pointer of get may be NULL.  Both synchronise `cuda_stream`.
+ */
+int adacons_get_state(adacons_ctx *ctx, double *host_m, int64_t *step, void *cuda_stream);
+int adacons_set_state(adacons_ctx *ctx, const double *host_m, int64_t step, void *cuda_stream);
+
+/* OR of the adacons_flag bits raised since the last reset.  Synchronises `cuda_stream`. */
+int adacons_get_status(adacons_ctx *ctx, uint32_t *flags, void *cuda_stream);
+
+/*
+ * Per-kernel device time, for roofline reporting.  With ADACONS_OPT_PROFILE = 1 every aggregate
+ * call records four CUDA events on its stream (before pass 1, after pass 1, after the
+ * coefficient step, after pass 2) into a ring of 64 slots.  This call synchronises
+ * `cuda_stream` and returns the mean duration in milliseconds of {pass 1, coefficient step,
+ * pass 2} over the recorded calls (at most the last 64) and their number.  No paper counterpart.
+ * Errors: EINVAL (NULL, profiling off or nothing recorded), ECUDA.
+ */
+int adacons_get_profile(adacons_ctx *ctx, double ms[3], int64_t *calls, void *cuda_stream);
+
+/* Facts about the context; see enum adacons_info.  No device work. */
+int adacons_get_info(adacons_ctx *ctx, int key, int64_t *value);
+
+/* Static, human-readable text for an adacons_error code. */
+const char *adacons_strerror(int code);
+
+/* Library version as major*10000 + minor*100 + patch. */
+int adacons_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADACONS_H_ */

@@ -1,0 +1,195 @@
+"""ctypes binding of the C ABI in include/adacons.h.
+
+Argument marshalling only: every step of the aggregation runs in the library's CUDA kernels.
+torch is used for device memory and streams.  If the shared library has not been built the
+import of this module's `load_library()` raises -- there is no fallback implementation.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_LIB = None
+LIB_NAME = "libadacons_b200.so"
+
+# enum adacons_dtype
+F32, BF16 = 0, 1
+# enum adacons_option
+OPT_BETA, OPT_MOMENTUM, OPT_SORTED, OPT_NORMALIZE, OPT_PER_SEGMENT, OPT_PROFILE = range(6)
+# enum adacons_coeff
+COEFF_A, COEFF_A_TILDE, COEFF_GAMMA, COEFF_P, COEFF_Q = range(5)
+# enum adacons_info
+(INFO_NUM_SEGMENTS, INFO_COEFF_SETS, INFO_PASS1_BLOCKS, INFO_SCRATCH_BYTES, INFO_LAUNCHES_PER_CALL,
+ INFO_LAST_PATH, INFO_TOTAL_LAUNCHES) = range(7)
+# enum adacons_flag
+FLAG_ZERO_ROW, FLAG_DEGENERATE_Z, FLAG_NONFINITE, FLAG_NEG_Z, FLAG_TIMEOUT = 1, 2, 4, 8, 0x100
+# enum adacons_error
+OK, EINVAL, EALIGN, ENOMEM, ECUDA, EARCH, ETIMEOUT = range(7)
+
+
+class AdaConsError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {strerror(code)} (code {code})")
+
+
+def library_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), LIB_NAME)
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the in-tree shared library and declare its prototypes."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = library_path()
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2411_03742_b200.build` "
+            "(nvcc, sm_100a).  There is no CPU fallback.")
+    lib = ctypes.CDLL(path)
+    vp, i32, i64, dbl = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_double
+    P = ctypes.POINTER
+    protos = {
+        "adacons_create": [P(vp), i32, i64, i32, P(i64), i32],
+        "adacons_aggregate": [vp, vp, vp, vp],
+        "adacons_aggregate_host": [vp, vp, vp, vp],
+        "adacons_reset": [vp, vp],
+        "adacons_destroy": [vp],
+        "adacons_set_option": [vp, i32, dbl],
+        "adacons_get_option": [vp, i32, P(dbl)],
+        "adacons_get_coeffs": [vp, i32, P(dbl), vp],
+        "adacons_get_state": [vp, P(dbl), P(i64), vp],
+        "adacons_set_state": [vp, P(dbl), i64, vp],
+        "adacons_get_status": [vp, P(ctypes.c_uint32), vp],
+        "adacons_get_info": [vp, i32, P(i64)],
+        "adacons_get_profile": [vp, P(dbl), P(i64), vp],
+        "adacons_version": [],
+    }
+    for name, args in protos.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = i32
+    lib.adacons_strerror.argtypes = [i32]
+    lib.adacons_strerror.restype = ctypes.c_char_p
+    _LIB = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().adacons_strerror(int(code)).decode()
+
+
+def _check(code: int, what: str) -> None:
+    if code != OK:
+        raise AdaConsError(code, what)
+
+
+def _stream_handle(stream) -> int:
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+class AdaCons:
+    """One aggregation context: N workers, gradients of d elements of `dtype` ("f32"/"bf16").
+
+    aggregate(grads, out) takes torch CUDA tensors (grads: N x d contiguous, out: d) and
+    enqueues the three kernels on the current (or given) torch stream.
+    """
+
+    def __init__(self, N: int, d: int, dtype: str = "f32", seg_offsets=None):
+        self._lib = load_library()
+        self._ctx = ctypes.c_void_p()
+        self.N, self.d, self.dtype = int(N), int(d), dtype
+        dt = {"f32": F32, "bf16": BF16}[dtype]
+        if seg_offsets is not None:
+            off = (ctypes.c_int64 * len(seg_offsets))(*[int(o) for o in seg_offsets])
+            rc = self._lib.adacons_create(ctypes.byref(self._ctx), N, d, dt, off, len(seg_offsets) - 1)
+        else:
+            rc = self._lib.adacons_create(ctypes.byref(self._ctx), N, d, dt, None, 0)
+        _check(rc, "adacons_create")
+
+    # -- lifetime ---------------------------------------------------------------------------
+    def close(self) -> None:
+        if getattr(self, "_ctx", None) is not None and self._ctx.value:
+            self._lib.adacons_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    # -- hot path ---------------------------------------------------------------------------
+    def aggregate(self, grads, out, stream=None) -> None:
+        self.aggregate_ptr(grads.data_ptr(), out.data_ptr(), _stream_handle(stream))
+
+    def aggregate_ptr(self, grads_ptr: int, out_ptr: int, stream_handle: int) -> None:
+        _check(self._lib.adacons_aggregate(self._ctx, grads_ptr, out_ptr, stream_handle), "adacons_aggregate")
+
+    def aggregate_host(self, host_grads, host_out, stream=None) -> None:
+        """host_grads / host_out: CPU tensors or numpy arrays (contiguous)."""
+        gp = host_grads.data_ptr() if hasattr(host_grads, "data_ptr") else host_grads.ctypes.data
+        op = host_out.data_ptr() if hasattr(host_out, "data_ptr") else host_out.ctypes.data
+        _check(self._lib.adacons_aggregate_host(self._ctx, gp, op, _stream_handle(stream)), "adacons_aggregate_host")
+
+    def reset(self, stream=None) -> None:
+        _check(self._lib.adacons_reset(self._ctx, _stream_handle(stream)), "adacons_reset")
+
+    # -- options, state, diagnostics -----------------------------------------------------------
+    def set_option(self, key: int, value: float) -> None:
+        _check(self._lib.adacons_set_option(self._ctx, key, float(value)), "adacons_set_option")
+
+    def get_option(self, key: int) -> float:
+        v = ctypes.c_double()
+        _check(self._lib.adacons_get_option(self._ctx, key, ctypes.byref(v)), "adacons_get_option")
+        return v.value
+
+    def info(self, key: int) -> int:
+        v = ctypes.c_int64()
+        _check(self._lib.adacons_get_info(self._ctx, key, ctypes.byref(v)), "adacons_get_info")
+        return v.value
+
+    def coeffs(self, which: int = COEFF_GAMMA, stream=None) -> np.ndarray:
+        sets = self.info(INFO_COEFF_SETS)
+        buf = np.empty((sets, self.N), dtype=np.float64)
+        _check(self._lib.adacons_get_coeffs(self._ctx, which, buf.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+                                            _stream_handle(stream)), "adacons_get_coeffs")
+        return buf
+
+    def state(self, stream=None):
+        sets = self.info(INFO_COEFF_SETS)
+        buf = np.empty((sets, self.N), dtype=np.float64)
+        step = ctypes.c_int64()
+        _check(self._lib.adacons_get_state(self._ctx, buf.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+                                           ctypes.byref(step), _stream_handle(stream)), "adacons_get_state")
+        return buf, step.value
+
+    def set_state(self, m: np.ndarray, step: int, stream=None) -> None:
+        m = np.ascontiguousarray(m, dtype=np.float64)
+        assert m.size == self.info(INFO_COEFF_SETS) * self.N
+        _check(self._lib.adacons_set_state(self._ctx, m.ctypes.data_as(ctypes.POINTER(ctypes.c_double)), int(step),
+                                           _stream_handle(stream)), "adacons_set_state")
+
+    def profile(self, stream=None):
+        """Mean device time in ms of (pass 1, coefficient step, pass 2) and the number of calls."""
+        ms = (ctypes.c_double * 3)()
+        n = ctypes.c_int64()
+        _check(self._lib.adacons_get_profile(self._ctx, ms, ctypes.byref(n), _stream_handle(stream)), "adacons_get_profile")
+        return [ms[0], ms[1], ms[2]], n.value
+
+    def status(self, stream=None) -> int:
+        v = ctypes.c_uint32()
+        _check(self._lib.adacons_get_status(self._ctx, ctypes.byref(v), _stream_handle(stream)), "adacons_get_status")
+        return v.value

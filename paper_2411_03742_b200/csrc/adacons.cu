@@ -1,0 +1,539 @@
+// Host side of the AdaCons aggregation library: context, launch plan and the C ABI declared in
+// include/adacons.h.  All arithmetic of the method runs in the kernels of adacons_kernels.cuh;
+// this file validates arguments, owns device memory and launches.
+#include "adacons.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "adacons_kernels.cuh"
+
+using namespace adacons;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct Pass1Plan {            // TMA-staged pass 1 for this (N, dtype)
+  bool available = false;
+  int NR = 0, WR = 0;
+  int tile_cols = 0;
+  int num_tiles = 0;
+  int stages = 0;
+  uint32_t stage_bytes = 0;
+  size_t smem_bytes = 0;
+  int grid = 0;
+  const void* kernel = nullptr;
+};
+
+}  // namespace
+
+struct adacons_ctx {
+  int N = 0;
+  long long d = 0;
+  int dtype = 0;
+  int elem_bytes = 4;
+  int device = 0;
+  int num_sms = 0;
+  std::vector<long long> seg_offsets;   // S + 1 entries
+  int num_segments = 1;
+
+  // options
+  double beta = 0.99;
+  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0;
+
+  // plans
+  Pass1Plan fast;
+  int generic_grid = 0;
+  int generic_tiles = 0;
+  size_t generic_smem = 0;
+  int max_partials = 0;
+
+  // device memory
+  float* partials = nullptr;      // [max_partials][sets][2N]
+  double* coef = nullptr;         // [5][sets][N]
+  float* gamma_f32 = nullptr;     // [sets][N]
+  double* m = nullptr;            // [sets][N]
+  uint32_t* flags = nullptr;
+  long long* step = nullptr;
+  void* staging = nullptr;        // adacons_aggregate_host: N*d + d elements
+  size_t scratch_bytes = 0;
+
+  EncodeTiledFn encode = nullptr;
+  CUtensorMap tmap;
+  const void* tmap_for = nullptr;
+
+  int last_path = 0;
+  long long total_launches = 0;
+
+  // optional per-kernel timing (ADACONS_OPT_PROFILE)
+  static constexpr int kProfSlots = 64;
+  int profile = 0;
+  long long prof_calls = 0;
+  cudaEvent_t prof_ev[kProfSlots][4] = {};
+  bool prof_ready = false;
+
+  int sets() const { return per_segment ? num_segments : 1; }
+};
+
+namespace {
+
+template <int DT, int NR, int WR>
+const void* pass1_fn() { return reinterpret_cast<const void*>(&pass1_tma_kernel<DT, NR, WR>); }
+
+const void* select_pass1(int dtype, int NR, int WR) {
+#define ADACONS_PICK(DT)                                     \
+  if (WR == 1) {                                             \
+    if (NR == 1) return pass1_fn<DT, 1, 1>();                \
+    if (NR == 2) return pass1_fn<DT, 2, 1>();                \
+    if (NR == 4) return pass1_fn<DT, 4, 1>();                \
+    return pass1_fn<DT, 8, 1>();                             \
+  }                                                          \
+  if (WR == 2) return pass1_fn<DT, 8, 2>();                  \
+  if (WR == 4) return pass1_fn<DT, 8, 4>();                  \
+  return pass1_fn<DT, 8, 8>();
+  if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
+  ADACONS_PICK(1)
+#undef ADACONS_PICK
+}
+
+int plan_fast(adacons_ctx* c) {
+  Pass1Plan& f = c->fast;
+  f.available = false;
+  const int N = c->N;
+  if (N > kMaxFastN) return ADACONS_OK;
+  if ((c->d * c->elem_bytes) % 16 != 0) return ADACONS_OK;
+  if (c->d > 2147483647ll - 8192) return ADACONS_OK;
+  if (c->encode == nullptr) return ADACONS_OK;
+  int WR, NR;
+  if (N <= 8) { WR = 1; NR = N <= 1 ? 1 : N <= 2 ? 2 : N <= 4 ? 4 : 8; }
+  else if (N <= 16) { WR = 2; NR = 8; }
+  else if (N <= 32) { WR = 4; NR = 8; }
+  else { WR = 8; NR = 8; }
+  const int WC = kWarps / WR;
+  const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
+  f.NR = NR; f.WR = WR;
+  f.tile_cols = WC * (kBoxRowBytes / c->elem_bytes);
+  f.num_tiles = static_cast<int>((c->d + f.tile_cols - 1) / f.tile_cols);
+  f.stage_bytes = static_cast<uint32_t>(WC) * N * kBoxRowBytes;
+  const size_t xch = WR > 1 ? static_cast<size_t>(2) * WR * WC * 32 * vec * sizeof(float) : 0;
+  const size_t fixed = xch + static_cast<size_t>(kWarps) * NR * 2 * sizeof(float);
+  const size_t budget = 110 * 1024;   // two blocks per SM
+  int stages = static_cast<int>((budget - fixed - 64) / f.stage_bytes);
+  if (stages > 8) stages = 8;
+  if (stages < 2) stages = 2;
+  f.stages = stages;
+  f.smem_bytes = static_cast<size_t>(stages) * f.stage_bytes + fixed + static_cast<size_t>(stages) * 8;
+  f.kernel = select_pass1(c->dtype, NR, WR);
+  if (cudaFuncSetAttribute(f.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(f.smem_bytes)) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    return ADACONS_ECUDA;
+  }
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, f.kernel, kThreads, f.smem_bytes) != cudaSuccess ||
+      per_sm < 1) {
+    cudaGetLastError();
+    return ADACONS_ECUDA;
+  }
+  f.grid = per_sm * c->num_sms;
+  if (f.grid > f.num_tiles) f.grid = f.num_tiles;
+  f.available = true;
+  return ADACONS_OK;
+}
+
+int encode_map(adacons_ctx* c, const void* grads) {
+  if (c->tmap_for == grads) return ADACONS_OK;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->d) * c->elem_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(c->N)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = c->encode(&c->tmap,
+                               c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                               2, const_cast<void*>(grads), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  c->tmap_for = grads;
+  return ADACONS_OK;
+}
+
+bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
+
+struct DeviceGuard {   // make the context's device current for the duration of a call
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+int alloc_sets(adacons_ctx* c) {   // (re)allocate everything whose size depends on sets()
+  cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
+  c->partials = nullptr; c->coef = nullptr; c->gamma_f32 = nullptr; c->m = nullptr;
+  const size_t sets = static_cast<size_t>(c->sets());
+  const size_t N = static_cast<size_t>(c->N);
+  const size_t b_part = static_cast<size_t>(c->max_partials) * sets * 2 * N * sizeof(float);
+  const size_t b_coef = 5 * sets * N * sizeof(double);
+  const size_t b_gam = sets * N * sizeof(float);
+  const size_t b_m = sets * N * sizeof(double);
+  if (cudaMalloc(&c->partials, b_part) != cudaSuccess || cudaMalloc(&c->coef, b_coef) != cudaSuccess ||
+      cudaMalloc(&c->gamma_f32, b_gam) != cudaSuccess || cudaMalloc(&c->m, b_m) != cudaSuccess) {
+    cudaGetLastError();
+    return ADACONS_ENOMEM;
+  }
+  if (cudaMemset(c->partials, 0, b_part) != cudaSuccess || cudaMemset(c->coef, 0, b_coef) != cudaSuccess ||
+      cudaMemset(c->gamma_f32, 0, b_gam) != cudaSuccess || cudaMemset(c->m, 0, b_m) != cudaSuccess)
+    return ADACONS_ECUDA;
+  c->scratch_bytes = b_part + b_coef + b_gam + b_m + sizeof(uint32_t) + sizeof(long long);
+  return ADACONS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int adacons_version(void) { return 100; }
+
+const char* adacons_strerror(int code) {
+  switch (code) {
+    case ADACONS_OK: return "success";
+    case ADACONS_EINVAL: return "invalid argument";
+    case ADACONS_EALIGN: return "misaligned buffer";
+    case ADACONS_ENOMEM: return "out of memory";
+    case ADACONS_ECUDA: return "CUDA call failed or no CUDA device";
+    case ADACONS_EARCH: return "device is not compute capability 10.x (sm_100)";
+    case ADACONS_ETIMEOUT: return "a bounded on-device wait expired";
+    default: return "unknown error code";
+  }
+}
+
+int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t* seg_offsets, int num_segments) {
+  if (out == nullptr) return ADACONS_EINVAL;
+  *out = nullptr;
+  if (N < 1 || N > kMaxN || d < 1 || d >= (1ll << 31)) return ADACONS_EINVAL;
+  if (dtype != ADACONS_F32 && dtype != ADACONS_BF16) return ADACONS_EINVAL;
+  if (num_segments < 0 || (num_segments > 0 && seg_offsets == nullptr)) return ADACONS_EINVAL;
+  if (num_segments > 0) {
+    if (seg_offsets[0] != 0 || seg_offsets[num_segments] != d) return ADACONS_EINVAL;
+    for (int s = 0; s < num_segments; ++s)
+      if (seg_offsets[s + 1] < seg_offsets[s]) return ADACONS_EINVAL;
+  }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  int major = 0, sms = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return ADACONS_ECUDA;
+  }
+  if (major != 10) return ADACONS_EARCH;
+
+  adacons_ctx* c = new (std::nothrow) adacons_ctx();
+  if (c == nullptr) return ADACONS_ENOMEM;
+  c->N = N; c->d = d; c->dtype = dtype; c->elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
+  c->device = dev; c->num_sms = sms;
+  if (num_segments > 0) {
+    c->num_segments = num_segments;
+    c->seg_offsets.assign(seg_offsets, seg_offsets + num_segments + 1);
+  } else {
+    c->num_segments = 1;
+    c->seg_offsets = {0, static_cast<long long>(d)};
+  }
+
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess)
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  else
+    cudaGetLastError();
+
+  int rc = plan_fast(c);
+  if (rc != ADACONS_OK) { delete c; return rc; }
+
+  // generic path: always available
+  c->generic_tiles = static_cast<int>((d + kThreads * 4 - 1) / (kThreads * 4));
+  c->generic_smem = static_cast<size_t>(kWarps) * N * 2 * sizeof(float);
+  cudaFuncSetAttribute(reinterpret_cast<const void*>(&pass1_generic_kernel<0>),
+                       cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->generic_smem));
+  cudaFuncSetAttribute(reinterpret_cast<const void*>(&pass1_generic_kernel<1>),
+                       cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->generic_smem));
+  if (!launch_ok()) { delete c; return ADACONS_ECUDA; }
+  c->generic_grid = sms * 4;
+  if (c->generic_grid > c->generic_tiles) c->generic_grid = c->generic_tiles;
+  c->max_partials = c->generic_grid;
+  if (c->fast.available && c->fast.grid > c->max_partials) c->max_partials = c->fast.grid;
+
+  if (cudaMalloc(&c->flags, sizeof(uint32_t)) != cudaSuccess || cudaMalloc(&c->step, sizeof(long long)) != cudaSuccess) {
+    cudaGetLastError(); adacons_destroy(c); return ADACONS_ENOMEM;
+  }
+  if (cudaMemset(c->flags, 0, sizeof(uint32_t)) != cudaSuccess || cudaMemset(c->step, 0, sizeof(long long)) != cudaSuccess) {
+    adacons_destroy(c); return ADACONS_ECUDA;
+  }
+  rc = alloc_sets(c);
+  if (rc != ADACONS_OK) { adacons_destroy(c); return rc; }
+  if (cudaDeviceSynchronize() != cudaSuccess) { adacons_destroy(c); return ADACONS_ECUDA; }
+  *out = c;
+  return ADACONS_OK;
+}
+
+int adacons_destroy(adacons_ctx* c) {
+  if (c == nullptr) return ADACONS_OK;
+  DeviceGuard g(c->device);
+  cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
+  cudaFree(c->flags); cudaFree(c->step); cudaFree(c->staging);
+  if (c->prof_ready)
+    for (int s = 0; s < adacons_ctx::kProfSlots; ++s)
+      for (int e = 0; e < 4; ++e) cudaEventDestroy(c->prof_ev[s][e]);
+  cudaGetLastError();
+  delete c;
+  return ADACONS_OK;
+}
+
+int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_stream) {
+  if (c == nullptr || grads == nullptr || out == nullptr) return ADACONS_EINVAL;
+  const size_t gbytes = static_cast<size_t>(c->N) * c->d * c->elem_bytes;
+  const size_t obytes = static_cast<size_t>(c->d) * c->elem_bytes;
+  const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads), o0 = reinterpret_cast<uintptr_t>(out);
+  if (o0 < g0 + gbytes && g0 < o0 + obytes) return ADACONS_EINVAL;   // out overlaps grads
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool aligned = (g0 % 16 == 0) && (o0 % 16 == 0) && ((c->d * c->elem_bytes) % 16 == 0);
+  const int N = c->N;
+  int num_partials;
+  cudaEvent_t* ev = (c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
+  if (ev) cudaEventRecord(ev[0], st);
+
+  // ---- pass 1 (Eq. 7) ----
+  if (aligned && c->fast.available) {
+    int rc = encode_map(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    Pass1Params p;
+    p.N = N; p.num_tiles = c->fast.num_tiles; p.stages = c->fast.stages; p.stage_bytes = c->fast.stage_bytes;
+    p.partials = c->partials; p.flags = c->flags;
+    void* args[2] = {&c->tmap, &p};
+    if (cudaLaunchKernel(c->fast.kernel, dim3(c->fast.grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    num_partials = c->fast.grid;
+    c->last_path = 1;
+  } else {
+    if (c->dtype == ADACONS_F32)
+      pass1_generic_kernel<0><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->generic_tiles, c->partials);
+    else
+      pass1_generic_kernel<1><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->generic_tiles, c->partials);
+    if (!launch_ok()) return ADACONS_ECUDA;
+    num_partials = c->generic_grid;
+    c->last_path = 2;
+  }
+  if (ev) cudaEventRecord(ev[1], st);
+
+  // ---- coefficients (Eq. 11, Eq. 12-13) ----
+  CoeffParams q;
+  q.N = N; q.num_partials = num_partials; q.sets = 1; q.beta = c->beta;
+  q.momentum = c->momentum; q.sorted = c->sorted; q.normalize = c->normalize;
+  q.partials = c->partials; q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m;
+  q.flags = c->flags; q.step = c->step;
+  const int cthreads = ((N + 31) / 32) * 32;
+  coeff_kernel<<<1, cthreads, 0, st>>>(q);
+  if (!launch_ok()) return ADACONS_ECUDA;
+  if (ev) cudaEventRecord(ev[2], st);
+
+  // ---- pass 2 (Eq. 12) ----
+  if (aligned) {
+    const long long num_vec = c->d * c->elem_bytes / 16;
+    const unsigned blocks = static_cast<unsigned>((num_vec + kThreads - 1) / kThreads);
+    const long long row_bytes = c->d * c->elem_bytes;
+    if (c->dtype == ADACONS_F32)
+      pass2_vec_kernel<0><<<blocks, kThreads, 0, st>>>(static_cast<const unsigned char*>(grads),
+                                                         static_cast<unsigned char*>(out), c->gamma_f32, N, row_bytes, num_vec);
+    else
+      pass2_vec_kernel<1><<<blocks, kThreads, 0, st>>>(static_cast<const unsigned char*>(grads),
+                                                         static_cast<unsigned char*>(out), c->gamma_f32, N, row_bytes, num_vec);
+  } else {
+    const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);
+    if (c->dtype == ADACONS_F32)
+      pass2_generic_kernel<0><<<blocks, kThreads, 0, st>>>(grads, out, c->gamma_f32, N, c->d);
+    else
+      pass2_generic_kernel<1><<<blocks, kThreads, 0, st>>>(grads, out, c->gamma_f32, N, c->d);
+  }
+  if (!launch_ok()) return ADACONS_ECUDA;
+  if (ev) { cudaEventRecord(ev[3], st); c->prof_calls += 1; }
+  c->total_launches += 3;
+  return ADACONS_OK;
+}
+
+int adacons_aggregate_host(adacons_ctx* c, const void* host_grads, void* host_out, void* cuda_stream) {
+  if (c == nullptr || host_grads == nullptr || host_out == nullptr) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t gbytes = static_cast<size_t>(c->N) * c->d * c->elem_bytes;
+  const size_t obytes = static_cast<size_t>(c->d) * c->elem_bytes;
+  const size_t gpad = (gbytes + 255) / 256 * 256;
+  if (c->staging == nullptr) {
+    if (cudaMalloc(&c->staging, gpad + obytes) != cudaSuccess) { cudaGetLastError(); return ADACONS_ENOMEM; }
+    c->scratch_bytes += gpad + obytes;
+  }
+  unsigned char* dg = static_cast<unsigned char*>(c->staging);
+  unsigned char* dout = dg + gpad;
+  if (cudaMemcpyAsync(dg, host_grads, gbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  const int rc = adacons_aggregate(c, dg, dout, cuda_stream);
+  if (rc != ADACONS_OK) return rc;
+  if (cudaMemcpyAsync(host_out, dout, obytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  return ADACONS_OK;
+}
+
+int adacons_reset(adacons_ctx* c, void* cuda_stream) {
+  if (c == nullptr) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  const long long n = static_cast<long long>(c->sets()) * c->N;
+  reset_kernel<<<static_cast<unsigned>((n + 255) / 256 < 1024 ? (n + 255) / 256 : 1024), 256, 0,
+                 static_cast<cudaStream_t>(cuda_stream)>>>(c->m, n, c->flags, c->step);
+  if (!launch_ok()) return ADACONS_ECUDA;
+  c->total_launches += 1;
+  return ADACONS_OK;
+}
+
+int adacons_set_option(adacons_ctx* c, int key, double value) {
+  if (c == nullptr) return ADACONS_EINVAL;
+  switch (key) {
+    case ADACONS_OPT_BETA:
+      if (!(value >= 0.0 && value < 1.0)) return ADACONS_EINVAL;
+      c->beta = value; return ADACONS_OK;
+    case ADACONS_OPT_MOMENTUM: c->momentum = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_SORTED: c->sorted = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_NORMALIZE: c->normalize = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_PER_SEGMENT:
+      if (value != 0.0) return ADACONS_EINVAL;   // layer-wise mode: not available in this build
+      return ADACONS_OK;
+    case ADACONS_OPT_PROFILE: {
+      DeviceGuard guard(c->device);
+      if (!guard.ok) return ADACONS_ECUDA;
+      if (value != 0.0 && !c->prof_ready) {
+        for (int s = 0; s < adacons_ctx::kProfSlots; ++s)
+          for (int e = 0; e < 4; ++e)
+            if (cudaEventCreate(&c->prof_ev[s][e]) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+        c->prof_ready = true;
+      }
+      c->profile = value != 0.0;
+      c->prof_calls = 0;
+      return ADACONS_OK;
+    }
+    default: return ADACONS_EINVAL;
+  }
+}
+
+int adacons_get_option(adacons_ctx* c, int key, double* value) {
+  if (c == nullptr || value == nullptr) return ADACONS_EINVAL;
+  switch (key) {
+    case ADACONS_OPT_BETA: *value = c->beta; return ADACONS_OK;
+    case ADACONS_OPT_MOMENTUM: *value = c->momentum; return ADACONS_OK;
+    case ADACONS_OPT_SORTED: *value = c->sorted; return ADACONS_OK;
+    case ADACONS_OPT_NORMALIZE: *value = c->normalize; return ADACONS_OK;
+    case ADACONS_OPT_PER_SEGMENT: *value = c->per_segment; return ADACONS_OK;
+    case ADACONS_OPT_PROFILE: *value = c->profile; return ADACONS_OK;
+    default: return ADACONS_EINVAL;
+  }
+}
+
+int adacons_get_coeffs(adacons_ctx* c, int which, double* host, void* cuda_stream) {
+  if (c == nullptr || host == nullptr || which < 0 || which > ADACONS_COEFF_Q) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t n = static_cast<size_t>(c->sets()) * c->N;
+  if (cudaMemcpyAsync(host, c->coef + static_cast<size_t>(which) * n, n * sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  return ADACONS_OK;
+}
+
+int adacons_get_state(adacons_ctx* c, double* host_m, int64_t* step, void* cuda_stream) {
+  if (c == nullptr) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t n = static_cast<size_t>(c->sets()) * c->N;
+  long long s = 0;
+  if (host_m && cudaMemcpyAsync(host_m, c->m, n * sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  if (step && cudaMemcpyAsync(&s, c->step, sizeof(long long), cudaMemcpyDeviceToHost, st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  if (step) *step = s;
+  return ADACONS_OK;
+}
+
+int adacons_set_state(adacons_ctx* c, const double* host_m, int64_t step, void* cuda_stream) {
+  if (c == nullptr || host_m == nullptr || step < 0) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t n = static_cast<size_t>(c->sets()) * c->N;
+  const long long s = step;
+  if (cudaMemcpyAsync(c->m, host_m, n * sizeof(double), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(c->step, &s, sizeof(long long), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  return ADACONS_OK;
+}
+
+int adacons_get_status(adacons_ctx* c, uint32_t* flags, void* cuda_stream) {
+  if (c == nullptr || flags == nullptr) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(flags, c->flags, sizeof(uint32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  return ADACONS_OK;
+}
+
+int adacons_get_profile(adacons_ctx* c, double ms[3], int64_t* calls, void* cuda_stream) {
+  if (c == nullptr || ms == nullptr || calls == nullptr) return ADACONS_EINVAL;
+  if (!c->prof_ready || c->prof_calls == 0) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  const long long n = c->prof_calls < adacons_ctx::kProfSlots ? c->prof_calls : adacons_ctx::kProfSlots;
+  double sum[3] = {0.0, 0.0, 0.0};
+  for (long long s = 0; s < n; ++s)
+    for (int k = 0; k < 3; ++k) {
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, c->prof_ev[s][k], c->prof_ev[s][k + 1]) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+      sum[k] += t;
+    }
+  for (int k = 0; k < 3; ++k) ms[k] = sum[k] / static_cast<double>(n);
+  *calls = n;
+  return ADACONS_OK;
+}
+
+int adacons_get_info(adacons_ctx* c, int key, int64_t* value) {
+  if (c == nullptr || value == nullptr) return ADACONS_EINVAL;
+  switch (key) {
+    case ADACONS_INFO_NUM_SEGMENTS: *value = c->num_segments; return ADACONS_OK;
+    case ADACONS_INFO_COEFF_SETS: *value = c->sets(); return ADACONS_OK;
+    case ADACONS_INFO_PASS1_BLOCKS: *value = c->fast.available ? c->fast.grid : c->generic_grid; return ADACONS_OK;
+    case ADACONS_INFO_SCRATCH_BYTES: *value = static_cast<int64_t>(c->scratch_bytes); return ADACONS_OK;
+    case ADACONS_INFO_LAUNCHES_PER_CALL: *value = 3; return ADACONS_OK;
+    case ADACONS_INFO_LAST_PATH: *value = c->last_path; return ADACONS_OK;
+    case ADACONS_INFO_TOTAL_LAUNCHES: *value = c->total_launches; return ADACONS_OK;
+    default: return ADACONS_EINVAL;
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,77 @@
+"""CPU-only checks of the boundary: the shared library builds, loads and exports every symbol
+that include/adacons.h declares; calls that need a device fail with an error code, not a crash."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2411_03742_b200 import build, binding
+    build.build()
+    return binding.load_library()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "adacons.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(adacons_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_four_core_calls():
+    names = declared_symbols()
+    for core in ("adacons_create", "adacons_aggregate", "adacons_reset", "adacons_destroy"):
+        assert core in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in declared_symbols():
+        assert hasattr(lib, name), name
+
+
+def test_binding_prototypes_cover_the_header(lib):
+    for name in declared_symbols():
+        fn = getattr(lib, name)
+        assert fn.argtypes is not None, f"{name} has no prototype in the binding"
+
+
+def test_strerror_and_version(lib):
+    assert lib.adacons_version() >= 100
+    assert lib.adacons_strerror(0) == b"success"
+    assert b"unknown" in lib.adacons_strerror(12345)
+
+
+def test_argument_validation_needs_no_device(lib):
+    ctx = ctypes.c_void_p()
+    assert lib.adacons_create(None, 4, 10, 0, None, 0) == 1
+    assert lib.adacons_create(ctypes.byref(ctx), 0, 10, 0, None, 0) == 1
+    assert lib.adacons_create(ctypes.byref(ctx), 4, 10, 9, None, 0) == 1
+    assert lib.adacons_destroy(None) == 0
+    assert lib.adacons_aggregate(None, None, None, None) == 1
+    assert lib.adacons_reset(None, None) == 1
+
+
+def test_create_without_a_device_returns_an_error_code(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    ctx = ctypes.c_void_p()
+    rc = lib.adacons_create(ctypes.byref(ctx), 4, 1024, 0, None, 0)
+    assert rc in (4, 5) and not ctx.value
+
+
+def test_product_does_not_import_the_oracle():
+    """The oracle is test infrastructure: nothing in the package may reference it."""
+    pkg = os.path.join(ROOT, "paper_2411_03742_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert not re.search(r"^\s*(import|from)\s+oracle|oracle[/.]adacons_oracle|#include.*oracle", text, re.M), f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith(".py"):
+            assert "paper_2411_03742_b200" not in open(os.path.join(ROOT, "oracle", f)).read(), f

@@ -1,0 +1,353 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 CPU oracle, element by
+element on the same seeded inputs.
+
+Tolerances
+  coefficients (a, a~, gamma, state m): 1e-5 relative, with the floor
+      |x_gpu - x_or| <= 1e-5 * max(|x_or_i|, 1e-3 * max_j |x_or_j|)
+  output: |out_gpu - psi_or| <= 1e-5 * max|g|  (fp32 storage)  or  4e-3 * max|g|  (bf16 storage),
+  and additionally the tighter element-wise bound that follows from the coefficient tolerance:
+      |out_gpu - psi_or| <= 1e-5 * sum_i |gamma_i g_ik| + one rounding to the storage format.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import adacons_oracle as oc
+from paper_2411_03742_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+COEFF_RTOL = 1e-5
+OUT_TOL = {"f32": 1e-5, "bf16": 4e-3}
+ULP = {"f32": 2.0 ** -23, "bf16": 2.0 ** -8}
+
+
+@pytest.fixture(scope="module")
+def ac():
+    from paper_2411_03742_b200 import binding
+    binding.load_library()
+    return binding
+
+
+def to_f64(G: torch.Tensor) -> np.ndarray:
+    return G.detach().cpu().to(torch.float64).numpy()
+
+
+def assert_coeffs(got, want, what):
+    got, want = np.asarray(got, dtype=np.float64).ravel(), np.asarray(want, dtype=np.float64).ravel()
+    floor = 1e-3 * np.max(np.abs(want)) if want.size else 0.0
+    tol = COEFF_RTOL * np.maximum(np.abs(want), floor)
+    bad = np.abs(got - want) > tol
+    assert not bad.any(), f"{what}: max rel err {np.max(np.abs(got - want) / np.maximum(np.abs(want), floor)):.3e}"
+
+
+def assert_output(out_t, res, G64, dtype, what):
+    got = to_f64(out_t)
+    psi = res["psi"]
+    gmax = float(np.max(np.abs(G64))) if G64.size else 0.0
+    err = np.abs(got - psi)
+    assert np.all(err <= OUT_TOL[dtype] * gmax + 1e-300), f"{what}: max err {err.max():.3e} vs max|g| {gmax:.3e}"
+    if res["gamma"].shape[0] == 1:
+        mass = np.abs(res["gamma"][0])[:, None] * np.abs(G64)
+        tight = 1e-5 * mass.sum(axis=0) + ULP[dtype] * np.abs(psi) + 1e-45
+        assert np.all(err <= tight), f"{what}: tight bound violated by {np.max(err / tight):.3f}x"
+
+
+def run_case(ac, w, steps, *, beta=0.99, options=None, oracle_kw=None, offsets=None):
+    dev = torch.device("cuda:0")
+    oracle_kw = oracle_kw or {}
+    h = ac.AdaCons(w.N, w.d, w.dtype, seg_offsets=offsets)
+    h.set_option(ac.OPT_BETA, beta)
+    for k, v in (options or {}).items():
+        h.set_option(k, v)
+    orc = oc.AdaConsOracle(w.N, w.d, beta=beta, **oracle_kw)
+    out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
+    expected_flags = 0
+    for t in range(steps):
+        G = wl.generate(w, t, dev)
+        h.aggregate(G, out)
+        torch.cuda.synchronize()
+        G64 = to_f64(G)
+        res = orc.step(G64, storage=w.dtype)
+        assert_coeffs(h.coeffs(ac.COEFF_P), res["p"], f"{w.name} step {t} p")
+        assert_coeffs(h.coeffs(ac.COEFF_Q), res["q"], f"{w.name} step {t} q")
+        assert_coeffs(h.coeffs(ac.COEFF_A), res["a"], f"{w.name} step {t} a")
+        assert_coeffs(h.coeffs(ac.COEFF_A_TILDE), res["a_tilde"], f"{w.name} step {t} a~")
+        assert_coeffs(h.coeffs(ac.COEFF_GAMMA), res["gamma"], f"{w.name} step {t} gamma")
+        m, step = h.state()
+        assert step == t + 1
+        assert_coeffs(m, res["m"], f"{w.name} step {t} m")
+        assert_output(out, res, G64, w.dtype, f"{w.name} step {t}")
+        expected_flags |= int(np.bitwise_or.reduce(res["flags"]))
+        assert h.status() == expected_flags
+    h.close()
+    return h
+
+
+# ---- the five benchmark configurations, scaled so that the oracle finishes in seconds but the
+# ---- kernels still see several tiles per block and a ragged last tile -------------------------
+def test_config1_full_size(ac):
+    run_case(ac, wl.WORKLOADS["small4"], 1)
+
+
+@pytest.mark.parametrize("name,d,steps", [
+    ("resnet8", 1_000_004, 5),
+    ("mixed16", 1_200_008, 4),
+    ("bert64", 400_008, 3),
+    ("ragged32", 1_000_004, 3),
+])
+def test_scaled_configs(ac, name, d, steps):
+    w = wl.WORKLOADS[name].scaled(d)
+    run_case(ac, w, steps, offsets=wl.segment_offsets(w))
+
+
+def test_config2_full_size_three_steps(ac):
+    w = wl.WORKLOADS["resnet8"]
+    run_case(ac, w, 3)
+
+
+# ---- every pass-1 instantiation, masked rows, both types ---------------------------------------
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N", [1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64])
+def test_all_worker_counts_fast_path(ac, N, dtype):
+    w = wl.Workload(f"n{N}", N, 20_008, dtype, 2, "gauss", seed=50 + N)
+    h = run_case(ac, w, 2, beta=0.7)
+    del h
+
+
+def test_fast_path_is_taken_when_aligned(ac):
+    w = wl.Workload("probe", 8, 8192, "f32", 1, "gauss")
+    h = ac.AdaCons(w.N, w.d, w.dtype)
+    G = wl.generate(w, 0, "cuda:0")
+    out = torch.empty(w.d, device="cuda:0")
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 1
+    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 3 and h.info(ac.INFO_TOTAL_LAUNCHES) == 3
+
+
+# ---- generic path: odd lengths, misaligned pointers, many workers ------------------------------
+@pytest.mark.parametrize("N,d,dtype", [(4, 10_001, "f32"), (8, 10_003, "bf16"), (3, 1, "f32"), (5, 7, "bf16"),
+                                       (65, 5_000, "f32"), (100, 4_099, "bf16"), (128, 3_000, "f32")])
+def test_generic_path(ac, N, d, dtype):
+    w = wl.Workload(f"g{N}x{d}", N, d, dtype, 2, "gauss", seed=7)
+    run_case(ac, w, 2, beta=0.5)
+
+
+def test_misaligned_pointers_take_the_generic_path(ac):
+    N, d = 6, 4096
+    w = wl.Workload("mis", N, d, "f32", 1, "gauss", seed=3)
+    G0 = wl.generate(w, 0, "cuda:0")
+    buf = torch.empty(N * d + 1, device="cuda:0")
+    G = buf[1:].view(N, d)
+    G.copy_(G0)
+    assert G.data_ptr() % 16 != 0
+    out = torch.empty(d, device="cuda:0")
+    h = ac.AdaCons(N, d, "f32")
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 2
+    res = oc.AdaConsOracle(N, d).step(to_f64(G0), storage="f32")
+    assert_coeffs(h.coeffs(ac.COEFF_GAMMA), res["gamma"], "gamma")
+    assert_output(out, res, to_f64(G0), "f32", "misaligned")
+
+
+def test_generic_and_fast_paths_agree(ac):
+    N, d = 16, 50_000
+    w = wl.Workload("agree", N, d, "bf16", 1, "gauss", seed=11)
+    G0 = wl.generate(w, 0, "cuda:0")
+    buf = torch.empty(N * d + 1, device="cuda:0", dtype=torch.bfloat16)
+    G1 = buf[1:].view(N, d)
+    G1.copy_(G0)
+    o0, o1 = torch.empty(d, device="cuda:0", dtype=torch.bfloat16), torch.empty(d, device="cuda:0", dtype=torch.bfloat16)
+    h0, h1 = ac.AdaCons(N, d, "bf16"), ac.AdaCons(N, d, "bf16")
+    h0.aggregate(G0, o0); h1.aggregate(G1, o1)
+    torch.cuda.synchronize()
+    assert (h0.info(ac.INFO_LAST_PATH), h1.info(ac.INFO_LAST_PATH)) == (1, 2)
+    np.testing.assert_allclose(h0.coeffs(), h1.coeffs(), rtol=2e-6)
+
+
+# ---- degenerate inputs --------------------------------------------------------------------------
+def _agg(ac, G, dtype="f32", **opt):
+    N, d = G.shape
+    h = ac.AdaCons(N, d, dtype)
+    for k, v in opt.items():
+        h.set_option(k, v)
+    out = torch.empty(d, device=G.device, dtype=G.dtype)
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    return h, out
+
+
+def test_identical_gradients_and_single_worker(ac):
+    g = torch.randn(5000, device="cuda:0")
+    h, out = _agg(ac, g.repeat(7, 1).contiguous())
+    np.testing.assert_allclose(to_f64(out), to_f64(g), rtol=3e-6, atol=1e-7)
+    h, out = _agg(ac, g.view(1, -1).contiguous())
+    assert h.coeffs()[0, 0] == 1.0
+    assert torch.equal(out, g)
+
+
+def test_zero_row_all_zero_nonfinite_and_negative_normaliser(ac):
+    G = torch.randn(4, 4096, device="cuda:0") + torch.randn(4096, device="cuda:0")
+    G[2] = 0
+    h, out = _agg(ac, G)
+    res = oc.AdaConsOracle(4, 4096).step(to_f64(G))
+    assert h.status() == ac.FLAG_ZERO_ROW == int(res["flags"][0])
+    assert h.coeffs()[0, 2] == 0.0
+    assert_coeffs(h.coeffs(), res["gamma"], "gamma zero row")
+
+    h, out = _agg(ac, torch.zeros(3, 1024, device="cuda:0"))
+    assert h.status() & ac.FLAG_DEGENERATE_Z and h.status() & ac.FLAG_ZERO_ROW
+    np.testing.assert_array_equal(h.coeffs()[0], np.full(3, 1 / 3))
+    assert float(out.abs().max()) == 0.0
+
+    G = torch.randn(3, 2048, device="cuda:0") + torch.randn(2048, device="cuda:0")
+    h = ac.AdaCons(3, 2048, "f32")
+    out = torch.empty(2048, device="cuda:0")
+    h.aggregate(G, out)
+    m_before, _ = h.state()
+    G2 = G.clone(); G2[1, 77] = float("inf")
+    h.aggregate(G2, out)
+    torch.cuda.synchronize()
+    assert h.status() & ac.FLAG_NONFINITE
+    np.testing.assert_array_equal(h.coeffs()[0], np.full(3, 1 / 3))
+    m_after, step = h.state()
+    np.testing.assert_array_equal(m_before, m_after)
+    assert step == 2
+
+    x = torch.randn(1024, device="cuda:0")
+    h, out = _agg(ac, torch.stack([10 * x, -x]).contiguous())
+    assert h.status() & ac.FLAG_NEG_Z
+    assert abs(h.coeffs().sum() - 1) < 1e-12
+
+
+# ---- determinism, state, options ----------------------------------------------------------------
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_bit_stability(ac, dtype):
+    w = wl.Workload("bits", 24, 700_008, dtype, 3, "gauss", seed=21)
+    dev = "cuda:0"
+    Gs = [wl.generate(w, t, dev) for t in range(3)]
+    runs = []
+    for _ in range(2):
+        h = ac.AdaCons(w.N, w.d, dtype)
+        out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
+        outs = []
+        for G in Gs:
+            h.aggregate(G, out)
+            outs.append(out.clone())
+        torch.cuda.synchronize()
+        runs.append((outs, h.coeffs().copy(), h.state()[0].copy()))
+    for a, b in zip(runs[0][0], runs[1][0]):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    assert runs[0][1].tobytes() == runs[1][1].tobytes()
+    assert runs[0][2].tobytes() == runs[1][2].tobytes()
+
+
+def test_state_roundtrip_and_reset(ac):
+    w = wl.Workload("state", 12, 30_000, "f32", 4, "gauss", seed=31)
+    dev = "cuda:0"
+    h1, h2 = ac.AdaCons(w.N, w.d, "f32"), ac.AdaCons(w.N, w.d, "f32")
+    out1, out2 = torch.empty(w.d, device=dev), torch.empty(w.d, device=dev)
+    for t in range(2):
+        h1.aggregate(wl.generate(w, t, dev), out1)
+    m, step = h1.state()
+    assert step == 2
+    h2.set_state(m, step)
+    G = wl.generate(w, 2, dev)
+    h1.aggregate(G, out1); h2.aggregate(G, out2)
+    torch.cuda.synchronize()
+    assert torch.equal(out1, out2) and h2.state()[1] == 3
+    h1.reset()
+    m, step = h1.state()
+    assert step == 0 and not m.any() and h1.status() == 0
+    # after a reset the first step is the momentum-free rule
+    h1.aggregate(G, out1)
+    res = oc.AdaConsOracle(w.N, w.d, beta=0.0).step(to_f64(G))
+    assert_coeffs(h1.coeffs(), res["gamma"], "gamma after reset")
+
+
+@pytest.mark.parametrize("momentum,sorted_,normalize", [(0, 1, 1), (1, 0, 1), (1, 1, 0), (0, 1, 0)])
+def test_ablation_variants(ac, momentum, sorted_, normalize):
+    w = wl.Workload("abl", 10, 40_000, "f32", 3, "gauss", seed=41)
+    run_case(ac, w, 3, beta=0.8,
+             options={ac.OPT_MOMENTUM: momentum, ac.OPT_SORTED: sorted_, ac.OPT_NORMALIZE: normalize},
+             oracle_kw=dict(momentum=bool(momentum), sort=bool(sorted_), normalize=bool(normalize)))
+
+
+def test_argument_errors(ac):
+    lib = ac.load_library()
+    ctx = ctypes.c_void_p()
+    assert lib.adacons_create(ctypes.byref(ctx), 0, 10, 0, None, 0) == ac.EINVAL
+    assert lib.adacons_create(ctypes.byref(ctx), 4, 0, 0, None, 0) == ac.EINVAL
+    assert lib.adacons_create(ctypes.byref(ctx), 4, 10, 7, None, 0) == ac.EINVAL
+    assert lib.adacons_create(ctypes.byref(ctx), 2000, 10, 0, None, 0) == ac.EINVAL
+    bad = (ctypes.c_int64 * 3)(0, 7, 9)
+    assert lib.adacons_create(ctypes.byref(ctx), 4, 10, 0, bad, 2) == ac.EINVAL
+    h = ac.AdaCons(4, 1024, "f32")
+    G = torch.zeros(4, 1024, device="cuda:0")
+    with pytest.raises(ac.AdaConsError):
+        h.aggregate_ptr(0, G.data_ptr(), 0)
+    with pytest.raises(ac.AdaConsError):
+        h.aggregate_ptr(G.data_ptr(), G.data_ptr() + 4096, 0)        # out inside grads
+    with pytest.raises(ac.AdaConsError):
+        h.set_option(ac.OPT_BETA, 1.5)
+    with pytest.raises(ac.AdaConsError):
+        h.set_option(99, 1.0)
+    assert "invalid" in ac.strerror(ac.EINVAL)
+
+
+def test_host_entry_point(ac):
+    w = wl.Workload("host", 8, 200_000, "bf16", 1, "gauss", seed=61)
+    G = wl.generate(w, 0, "cpu").pin_memory()
+    out = torch.empty(w.d, dtype=torch.bfloat16).pin_memory()
+    h = ac.AdaCons(w.N, w.d, "bf16")
+    h.aggregate_host(G, out)
+    res = oc.AdaConsOracle(w.N, w.d).step(to_f64(G), storage="bf16")
+    assert_coeffs(h.coeffs(), res["gamma"], "gamma host")
+    assert_output(out, res, to_f64(G), "bf16", "host entry")
+
+
+# ---- full size of the headline configuration, as the benchmark launches it ---------------------
+def test_headline_config_full_size_sampled(ac):
+    """N=64, d=340M, bf16 (43.5 GB).  The oracle cannot stream all of it in test time, so:
+    pass 2 is checked on sampled columns with the oracle's combine(); q_i is checked for sampled
+    workers with the oracle; p is checked through the identity sum_i N p_i = ||sum_j g_j||^2 and
+    per sampled worker against a float64 torch dot product; and sum(gamma) = 1."""
+    w = wl.WORKLOADS["bert64"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60e9:
+        pytest.skip("needs 60 GB of free device memory")
+    dev = torch.device("cuda:0")
+    G = wl.generate(w, 0, dev)
+    out = torch.empty(w.d, dtype=torch.bfloat16, device=dev)
+    h = ac.AdaCons(w.N, w.d, "bf16")
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 1 and h.status() == 0
+    gamma, p, q = h.coeffs(ac.COEFF_GAMMA)[0], h.coeffs(ac.COEFF_P)[0], h.coeffs(ac.COEFF_Q)[0]
+    assert abs(gamma.sum() - 1.0) < 1e-12
+    assert gamma[0] < 0 and gamma[1] < 0 and np.all(gamma[2:] > 0)     # the sign-flipped workers
+
+    # pass 2 on sampled columns (first, last, random)
+    gcpu = torch.Generator().manual_seed(1)
+    cols = torch.cat([torch.arange(0, 64), torch.arange(w.d - 64, w.d),
+                      torch.randint(0, w.d, (4096,), generator=gcpu)]).to(dev)
+    Gs = to_f64(G[:, cols])
+    psi = oc.combine(Gs, gamma)
+    got = to_f64(out[cols])
+    tight = 1e-5 * (np.abs(gamma)[:, None] * np.abs(Gs)).sum(0) + ULP["bf16"] * np.abs(psi) + 1e-45
+    assert np.all(np.abs(got - psi) <= tight)
+
+    # q_i for sampled workers with the oracle, p_i against float64 column sums
+    s = torch.zeros(w.d, dtype=torch.float64, device=dev)
+    for i in range(w.N):
+        s += G[i].double()
+    assert abs(w.N * p.sum() - float((s * s).sum())) <= 1e-5 * float((s * s).sum())
+    for i in (0, 17, 63):
+        _, qi = oc.consensus_statistics(to_f64(G[i:i + 1]))
+        assert abs(q[i] - qi[0]) <= COEFF_RTOL * qi[0]
+        pi = float((G[i].double() * s).sum()) / w.N
+        assert abs(p[i] - pi) <= COEFF_RTOL * abs(pi)
