@@ -129,11 +129,24 @@ def test_fast_path_is_taken_when_aligned(ac):
 
 
 # ---- generic path: odd lengths, misaligned pointers, many workers ------------------------------
-@pytest.mark.parametrize("N,d,dtype", [(4, 10_001, "f32"), (8, 10_003, "bf16"), (3, 1, "f32"), (5, 7, "bf16"),
+@pytest.mark.parametrize("N,d,dtype", [(4, 10_001, "f32"), (8, 10_003, "bf16"), (3, 2, "f32"), (5, 7, "bf16"),
                                        (65, 5_000, "f32"), (100, 4_099, "bf16"), (128, 3_000, "f32")])
 def test_generic_path(ac, N, d, dtype):
     w = wl.Workload(f"g{N}x{d}", N, d, dtype, 2, "gauss", seed=7)
     run_case(ac, w, 2, beta=0.5)
+
+
+def test_single_column_has_tied_coefficients(ac):
+    """d = 1: a_i = sign(g_i) * gbar, so workers of equal sign tie exactly and which of them gets
+    which sorted slot depends on rounding.  What is unique: the sorted state, sum(gamma) = 1 and,
+    on the first step (where tied slots hold equal values), the output."""
+    G = torch.tensor([[0.5], [2.0], [-0.25]], device="cuda:0")
+    h, out = _agg(ac, G)
+    res = oc.AdaConsOracle(3, 1).step(to_f64(G), storage="f32")
+    m, _ = h.state()
+    assert_coeffs(np.sort(m[0]), np.sort(res["m"][0]), "sorted state")
+    assert abs(h.coeffs().sum() - 1.0) < 1e-12
+    assert_output(out, res, to_f64(G), "f32", "d=1")
 
 
 def test_misaligned_pointers_take_the_generic_path(ac):
