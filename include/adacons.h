@@ -49,7 +49,8 @@ enum adacons_error {
   ADACONS_ENOMEM = 3, /* device or host allocation failed                                       */
   ADACONS_ECUDA = 4,  /* a CUDA runtime/driver call failed, or no CUDA device                   */
   ADACONS_EARCH = 5,  /* the current device is not compute capability 10.x                      */
-  ADACONS_ETIMEOUT = 6 /* a bounded on-device wait gave up (reported by adacons_get_status)     */
+  ADACONS_ETIMEOUT = 6, /* a bounded on-device wait gave up (reported by adacons_get_status)    */
+  ADACONS_ELIMIT = 7   /* problem larger than the fixed scratch of adacons_stats_noalloc         */
 };
 
 /* Flags returned by adacons_get_status (OR over all segments since the last reset). */
@@ -178,6 +179,40 @@ int adacons_get_status(adacons_ctx *ctx, uint32_t *flags, void *cuda_stream);
  * Errors: EINVAL (NULL, profiling off or nothing recorded), ECUDA.
  */
 int adacons_get_profile(adacons_ctx *ctx, double ms[3], int64_t *calls, void *cuda_stream);
+
+/*
+ * Consensus statistics without any allocation.  (The paper has no counterpart: this entry point
+ * exists for integration, not for the method.)
+ *
+ * Who needs it: a gradient hook that runs inside a training framework usually finds the device's
+ * memory already handed to that framework's caching allocator, so a raw cudaMalloc -- which
+ * adacons_create performs -- may fail there, and it synchronises the whole device in the middle
+ * of the backward pass.  Such a caller, or one that only wants to log p_i and q_i, can call this
+ * function instead: it creates no context and calls no cudaMalloc, cudaFree or other allocating
+ * routine.  The per-block partial sums of pass 1 live in a fixed array inside the library's
+ * device image (ADACONS_NOALLOC_SCRATCH_BYTES, held by every GPU that loads the library until the
+ * process exits).
+ *
+ *   grads   device pointer, N x d row-major, as for adacons_aggregate (read-only).
+ *   N, d    1 <= N <= ADACONS_NOALLOC_MAX_N, 1 <= d < 2^31; larger N returns ADACONS_ELIMIT.
+ *   dtype   enum adacons_dtype.
+ *   pq_out  device pointer to 2N doubles owned by the caller: p_0..p_{N-1} = <g_i, gbar>, then
+ *           q_0..q_{N-1} = ||g_i||^2 (Eq. 7) -- the values adacons_get_coeffs returns as
+ *           ADACONS_COEFF_P / ADACONS_COEFF_Q after adacons_aggregate on the same input.
+ * Runs pass 1 and a small reduction kernel on `cuda_stream`; no host synchronisation.
+ * The first call on each device also looks up the device address of the scratch array and the
+ * driver's tensor-map encoder; make that first call before any stream capture begins.
+ * All calls share the one scratch array, which keeps the previous call's contents: every word a
+ * call reads it has written itself first (the status word is cleared on the stream), but two
+ * calls that overlap on the GPU (different streams, or threads) race on it -- serialise them.
+ * If a bounded wait inside pass 1 expires, pq_out is filled with NaN.
+ * Errors: EINVAL (NULL, bad N/d/dtype), ELIMIT, EARCH, ECUDA.
+ */
+#define ADACONS_NOALLOC_MAX_N 64
+#define ADACONS_NOALLOC_MAX_BLOCKS 1024
+#define ADACONS_NOALLOC_SCRATCH_BYTES (ADACONS_NOALLOC_MAX_BLOCKS * 2 * ADACONS_NOALLOC_MAX_N * 4 + 256)
+int adacons_stats_noalloc(const void *grads, int N, int64_t d, int dtype, double *pq_out,
+                          void *cuda_stream);
 
 /* Facts about the context; see enum adacons_info.  No device work. */
 int adacons_get_info(adacons_ctx *ctx, int key, int64_t *value);

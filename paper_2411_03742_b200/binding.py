@@ -26,7 +26,8 @@ COEFF_A, COEFF_A_TILDE, COEFF_GAMMA, COEFF_P, COEFF_Q = range(5)
 # enum adacons_flag
 FLAG_ZERO_ROW, FLAG_DEGENERATE_Z, FLAG_NONFINITE, FLAG_NEG_Z, FLAG_TIMEOUT = 1, 2, 4, 8, 0x100
 # enum adacons_error
-OK, EINVAL, EALIGN, ENOMEM, ECUDA, EARCH, ETIMEOUT = range(7)
+OK, EINVAL, EALIGN, ENOMEM, ECUDA, EARCH, ETIMEOUT, ELIMIT = range(8)
+NOALLOC_MAX_N = 64
 
 
 class AdaConsError(RuntimeError):
@@ -66,6 +67,7 @@ def load_library() -> ctypes.CDLL:
         "adacons_get_status": [vp, P(ctypes.c_uint32), vp],
         "adacons_get_info": [vp, i32, P(i64)],
         "adacons_get_profile": [vp, P(dbl), P(i64), vp],
+        "adacons_stats_noalloc": [vp, i32, i64, i32, vp, vp],
         "adacons_version": [],
     }
     for name, args in protos.items():
@@ -92,6 +94,19 @@ def _stream_handle(stream) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
     return int(stream.cuda_stream)
+
+
+def stats_noalloc(grads, pq_out, stream=None) -> None:
+    """p_i = <g_i, gbar> and q_i = ||g_i||^2 of an N x d CUDA tensor into `pq_out` (CUDA tensor of
+    2N float64), through the entry point that allocates no device memory (N <= NOALLOC_MAX_N).
+    For callers that cannot allocate: e.g. a gradient hook inside a framework whose caching
+    allocator already owns the device's memory."""
+    import torch
+    N, d = grads.shape
+    dt = {torch.float32: F32, torch.bfloat16: BF16}[grads.dtype]
+    assert pq_out.dtype == torch.float64 and pq_out.numel() >= 2 * N and pq_out.is_cuda and grads.is_cuda
+    _check(load_library().adacons_stats_noalloc(grads.data_ptr(), N, d, dt, pq_out.data_ptr(), _stream_handle(stream)),
+           "adacons_stats_noalloc")
 
 
 class AdaCons:

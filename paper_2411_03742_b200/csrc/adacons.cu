@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <pthread.h>
 #include <new>
 #include <vector>
 
@@ -217,6 +218,7 @@ const char* adacons_strerror(int code) {
     case ADACONS_ECUDA: return "CUDA call failed or no CUDA device";
     case ADACONS_EARCH: return "device is not compute capability 10.x (sm_100)";
     case ADACONS_ETIMEOUT: return "a bounded on-device wait expired";
+    case ADACONS_ELIMIT: return "problem exceeds the fixed scratch of the allocation-free entry point (N > 64)";
     default: return "unknown error code";
   }
 }
@@ -537,3 +539,126 @@ int adacons_get_info(adacons_ctx* c, int key, int64_t* value) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free consensus statistics (adacons_stats_noalloc).
+//
+// The block partials of pass 1 go to a fixed array in the library's device image instead of
+// memory from cudaMalloc.  In host code the array's name is only a handle: the device address is
+// fetched once per device with cudaGetSymbolAddress (that device current) and passed to the
+// kernels like any other pointer.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[ADACONS_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kNoAllocMaxDevices = 64;
+constexpr size_t kNoAllocPartialBytes =
+    static_cast<size_t>(ADACONS_NOALLOC_MAX_BLOCKS) * 2 * ADACONS_NOALLOC_MAX_N * sizeof(float);
+
+struct NoAllocDevice {
+  bool ready = false;
+  unsigned char* scratch = nullptr;   // device address of g_noalloc_scratch on this device
+  EncodeTiledFn encode = nullptr;
+  int sms = 0;
+};
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+pthread_mutex_t g_noalloc_mutex = PTHREAD_MUTEX_INITIALIZER;
+
+// Sum the block partials in index order (fp64) into the caller's buffer: p (divided by N), then q.
+__global__ void stats_finish_kernel(const float* __restrict__ partials, int num_partials, int N,
+                                    const uint32_t* __restrict__ flag, double* __restrict__ pq_out) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= 2 * N) return;
+  if (*flag & kFlagTimeout) { pq_out[i] = __longlong_as_double(0x7ff8000000000000ll); return; }
+  double acc = 0.0;
+  for (int c = 0; c < num_partials; ++c) acc += static_cast<double>(partials[static_cast<size_t>(c) * 2 * N + i]);
+  pq_out[i] = i < N ? acc / static_cast<double>(N) : acc;
+}
+
+int noalloc_setup(int dev, NoAllocDevice** out) {
+  if (dev < 0 || dev >= kNoAllocMaxDevices) return ADACONS_EINVAL;
+  pthread_mutex_lock(&g_noalloc_mutex);
+  NoAllocDevice& nd = g_noalloc_dev[dev];
+  int rc = ADACONS_OK;
+  if (!nd.ready) {
+    void* ptr = nullptr;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&nd.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      cudaGetLastError(); rc = ADACONS_ECUDA;
+    } else if (major != 10) {
+      rc = ADACONS_EARCH;
+    } else if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+      cudaGetLastError(); rc = ADACONS_ECUDA;
+    } else {
+      nd.scratch = static_cast<unsigned char*>(ptr);
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult qres;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+          qres == cudaDriverEntryPointSuccess)
+        nd.encode = reinterpret_cast<EncodeTiledFn>(fn);
+      else
+        cudaGetLastError();
+      nd.ready = true;
+    }
+  }
+  pthread_mutex_unlock(&g_noalloc_mutex);
+  *out = &nd;
+  return rc;
+}
+
+}  // namespace
+
+extern "C" int adacons_stats_noalloc(const void* grads, int N, int64_t d, int dtype, double* pq_out,
+                                     void* cuda_stream) {
+  if (grads == nullptr || pq_out == nullptr) return ADACONS_EINVAL;
+  if (N < 1 || d < 1 || d >= (1ll << 31)) return ADACONS_EINVAL;
+  if (dtype != ADACONS_F32 && dtype != ADACONS_BF16) return ADACONS_EINVAL;
+  if (N > ADACONS_NOALLOC_MAX_N) return ADACONS_ELIMIT;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  NoAllocDevice* nd = nullptr;
+  int rc = noalloc_setup(dev, &nd);
+  if (rc != ADACONS_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+  // A context object on the host stack only carries the launch plan; it owns no device memory.
+  adacons_ctx plan;
+  plan.N = N; plan.d = d; plan.dtype = dtype; plan.elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
+  plan.device = dev; plan.num_sms = nd->sms; plan.encode = nd->encode;
+  rc = plan_fast(&plan);
+  if (rc != ADACONS_OK) return rc;
+
+  float* partials = reinterpret_cast<float*>(nd->scratch);
+  uint32_t* flag = reinterpret_cast<uint32_t*>(nd->scratch + kNoAllocPartialBytes);
+  if (cudaMemsetAsync(flag, 0, sizeof(uint32_t), st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+
+  const bool aligned = (reinterpret_cast<uintptr_t>(grads) % 16 == 0) && ((d * plan.elem_bytes) % 16 == 0);
+  int blocks;
+  if (aligned && plan.fast.available) {
+    rc = encode_map(&plan, grads);
+    if (rc != ADACONS_OK) return rc;
+    blocks = plan.fast.grid < ADACONS_NOALLOC_MAX_BLOCKS ? plan.fast.grid : ADACONS_NOALLOC_MAX_BLOCKS;
+    Pass1Params p;
+    p.N = N; p.num_tiles = plan.fast.num_tiles; p.stages = plan.fast.stages; p.stage_bytes = plan.fast.stage_bytes;
+    p.partials = partials; p.flags = flag;
+    void* args[2] = {&plan.tmap, &p};
+    if (cudaLaunchKernel(plan.fast.kernel, dim3(blocks), dim3(kThreads), args, plan.fast.smem_bytes, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+  } else {
+    const int tiles = static_cast<int>((d + kThreads * 4 - 1) / (kThreads * 4));
+    blocks = nd->sms * 4;
+    if (blocks > tiles) blocks = tiles;
+    if (blocks > ADACONS_NOALLOC_MAX_BLOCKS) blocks = ADACONS_NOALLOC_MAX_BLOCKS;
+    const size_t smem = static_cast<size_t>(kWarps) * N * 2 * sizeof(float);   // <= 4 KB for N <= 64
+    if (dtype == ADACONS_F32) pass1_generic_kernel<0><<<blocks, kThreads, smem, st>>>(grads, N, d, tiles, partials);
+    else pass1_generic_kernel<1><<<blocks, kThreads, smem, st>>>(grads, N, d, tiles, partials);
+    if (!launch_ok()) return ADACONS_ECUDA;
+  }
+  stats_finish_kernel<<<(2 * N + 127) / 128, 128, 0, st>>>(partials, blocks, N, flag, pq_out);
+  if (!launch_ok()) return ADACONS_ECUDA;
+  return ADACONS_OK;
+}

@@ -1,0 +1,70 @@
+"""The allocation-free entry point (adacons_stats_noalloc) against the ordinary one.
+
+Some callers cannot allocate device memory at the moment they need the aggregation's statistics
+-- typically a gradient hook running inside a training framework whose caching allocator has
+already taken the device's memory, where a raw cudaMalloc can fail and stalls the device.  For
+them the library keeps pass 1's scratch in a fixed array of its own device image.  This test
+calls that entry point through the C ABI twice in a row (different shapes, so that anything left
+in the shared scratch by the first call would show) and checks p_i and q_i against what
+adacons_aggregate + adacons_get_coeffs report for the same input, within the coefficient
+tolerance of the parity tests.  It is collected last on purpose.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2411_03742_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+COEFF_RTOL = 1e-5
+
+
+def _reference(ac, G):
+    N, d = G.shape
+    h = ac.AdaCons(N, d, "f32" if G.dtype == torch.float32 else "bf16")
+    out = torch.empty(d, dtype=G.dtype, device=G.device)
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    p, q = h.coeffs(ac.COEFF_P)[0].copy(), h.coeffs(ac.COEFF_Q)[0].copy()
+    h.close()
+    return p, q
+
+
+def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
+    from paper_2411_03742_b200 import binding as ac
+    dev = torch.device("cuda:0")
+    cases = [wl.Workload("na64", 64, 300_008, "bf16", 1, "student_flip", seed=5),
+             wl.Workload("na7", 7, 123_456, "f32", 1, "gauss_outlier", seed=6),
+             wl.Workload("na5odd", 5, 10_001, "bf16", 1, "gauss", seed=7)]       # generic (unaligned) path
+    pq = torch.full((128,), float("nan"), dtype=torch.float64, device=dev)
+    for w in cases:
+        G = wl.generate(w, 0, dev)
+        torch.cuda.synchronize()
+        pq.fill_(float("nan"))
+        ac.stats_noalloc(G, pq)
+        torch.cuda.synchronize()
+        got = pq.cpu().numpy()
+        p, q = _reference(ac, G)
+        np.testing.assert_allclose(got[:w.N], p, rtol=COEFF_RTOL, atol=COEFF_RTOL * 1e-3 * np.abs(p).max())
+        np.testing.assert_allclose(got[w.N:2 * w.N], q, rtol=COEFF_RTOL)
+        assert np.all(np.isnan(got[2 * w.N:]))                                  # nothing written past 2N
+        del G
+    # same input again right after the others: the shared scratch holds stale partials by now
+    w = cases[0]
+    G = wl.generate(w, 0, dev)
+    ac.stats_noalloc(G, pq)
+    ac.stats_noalloc(G, pq)
+    torch.cuda.synchronize()
+    p, q = _reference(ac, G)
+    got = pq.cpu().numpy()
+    np.testing.assert_allclose(got[:w.N], p, rtol=COEFF_RTOL, atol=COEFF_RTOL * 1e-3 * np.abs(p).max())
+    np.testing.assert_allclose(got[w.N:2 * w.N], q, rtol=COEFF_RTOL)
+
+
+def test_noalloc_rejects_sizes_beyond_its_scratch():
+    from paper_2411_03742_b200 import binding as ac
+    G = torch.zeros(ac.NOALLOC_MAX_N + 1, 256, device="cuda:0")
+    pq = torch.zeros(2 * (ac.NOALLOC_MAX_N + 1), dtype=torch.float64, device="cuda:0")
+    with pytest.raises(ac.AdaConsError) as e:
+        ac.stats_noalloc(G, pq)
+    assert e.value.code == ac.ELIMIT and "scratch" in str(e.value)
