@@ -45,7 +45,8 @@ enum adacons_dtype { ADACONS_F32 = 0, ADACONS_BF16 = 1 };
 enum adacons_error {
   ADACONS_OK = 0,
   ADACONS_EINVAL = 1, /* bad argument (NULL, N < 1, d < 1, unknown enum, bad offsets, overlap) */
-  ADACONS_EALIGN = 2, /* reserved: misaligned buffers take a slower path instead of failing     */
+  ADACONS_EALIGN = 2, /* per-segment mode only: it needs 16-byte aligned buffers and row pitch
+                         and N <= 64 (model-wise mode serves anything through a slower path)   */
   ADACONS_ENOMEM = 3, /* device or host allocation failed                                       */
   ADACONS_ECUDA = 4,  /* a CUDA runtime/driver call failed, or no CUDA device                   */
   ADACONS_EARCH = 5,  /* the current device is not compute capability 10.x                      */
@@ -73,7 +74,9 @@ enum adacons_option {
   ADACONS_OPT_PER_SEGMENT = 4, /* 0 (default): one set of coefficients for the whole vector
                                   ("model-wise"); 1: an independent set, with its own momentum
                                   state, for each segment given to adacons_create ("layer-wise",
-                                  Section 4).  Changing it resets the state.                     */
+                                  Section 4).  Changing it synchronises the device, allocates
+                                  the per-segment plan and state, and resets the state.
+                                  Errors: EALIGN (see above), ENOMEM.                            */
   ADACONS_OPT_PROFILE = 5      /* 0 (default) / 1: record CUDA events around each of the three
                                   kernels of every aggregate call (see adacons_get_profile).
                                   Setting it (to either value) clears the recorded samples.      */

@@ -88,24 +88,34 @@ def first_order_coefficients(p: np.ndarray, q: np.ndarray) -> np.ndarray:
 
 
 def subspace_momentum(a: np.ndarray, m_prev: np.ndarray, beta: float,
-                      sort: bool = True) -> tuple[np.ndarray, np.ndarray, np.ndarray]:
+                      sort: bool = True, assign=None) -> tuple[np.ndarray, np.ndarray, np.ndarray]:
     """Sorted subspace momentum (Eq. 11):
         m_t      = beta m_{t-1} + (1-beta) S(a)
         a_tilde  = S^{-1}(m_t)
     S sorts ascending and is stable (ties keep worker order).  With sort=False this is
     the index-coupled EMA of Eq. 10.  Returns (m_t, a_tilde, pi) where pi[k] is the
-    worker whose coefficient occupies sorted slot k."""
+    worker whose coefficient occupies sorted slot k.
+
+    The sorted values S(a), hence m_t, depend continuously on a, but which worker gets which
+    slot does not: two workers whose coefficients agree to within rounding may swap slots.
+    `assign` (optional, assign[i] = slot handed back to worker i) lets a caller that compares
+    against an implementation working in lower precision prescribe that implementation's
+    S^{-1}; the caller is responsible for checking that it sorts `a` to within its tolerance.
+    m_t is always computed from this function's own sort."""
     a = np.asarray(a, dtype=np.float64)
     n = a.shape[0]
     pi = np.argsort(a, kind="stable") if sort else np.arange(n)
     m = beta * np.asarray(m_prev, dtype=np.float64) + (1.0 - beta) * a[pi]
     a_tilde = np.empty(n, dtype=np.float64)
-    a_tilde[pi] = m
+    if assign is None:
+        a_tilde[pi] = m
+    else:
+        a_tilde[:] = m[np.asarray(assign, dtype=np.int64)]
     return m, a_tilde, pi
 
 
 def coefficients(p, q, m_prev, beta: float = DEFAULT_BETA, *, momentum: bool = True,
-                 sort: bool = True, normalize: bool = True) -> dict:
+                 sort: bool = True, normalize: bool = True, assign=None) -> dict:
     """Algorithm 1 steps 2-3: from the 2N statistics to the N weights gamma.
 
     momentum=False skips Eq. 11 (a_tilde = a, state untouched); sort=False uses Eq. 10;
@@ -128,7 +138,7 @@ def coefficients(p, q, m_prev, beta: float = DEFAULT_BETA, *, momentum: bool = T
                     flags=flags | FLAG_NONFINITE)
     a = first_order_coefficients(p, q)
     if momentum:
-        m, a_tilde, pi = subspace_momentum(a, m_prev, beta, sort=sort)
+        m, a_tilde, pi = subspace_momentum(a, m_prev, beta, sort=sort, assign=assign)
     else:
         m, a_tilde, pi = m_prev.copy(), a.copy(), np.arange(n)
     # P has unit columns, psi = P alpha  =>  weight on g_i is alpha_i / ||g_i||  (Eq. 8)
@@ -209,10 +219,10 @@ class AdaConsOracle:
         self.m = np.zeros((self.S, self.N), dtype=np.float64)
         self.t = 0
 
-    def step(self, G: np.ndarray, storage: str | None = None) -> dict:
+    def step(self, G: np.ndarray, storage: str | None = None, assign=None) -> dict:
         """One aggregation.  Returns per-segment arrays (S x N) of p, q, a, a_tilde,
         gamma, the new state m, flags (S,), psi (d,) and, if `storage` is given, `out`
-        = psi rounded to that format."""
+        = psi rounded to that format.  `assign` (S x N, optional): see subspace_momentum."""
         G = np.asarray(G, dtype=np.float64)
         assert G.shape == (self.N, self.d)
         keys = ("p", "q", "a", "a_tilde", "u", "gamma")
@@ -225,7 +235,8 @@ class AdaConsOracle:
             Gs = G[:, lo:hi]
             p, q = consensus_statistics(Gs)
             c = coefficients(p, q, self.m[s], self.beta, momentum=self.momentum,
-                             sort=self.sort, normalize=self.normalize)
+                             sort=self.sort, normalize=self.normalize,
+                             assign=None if assign is None else assign[s])
             self.m[s] = c["m"]
             for k in keys:
                 res[k][s] = c[k]

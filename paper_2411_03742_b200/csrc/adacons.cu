@@ -68,6 +68,20 @@ struct adacons_ctx {
   void* staging = nullptr;        // adacons_aggregate_host: N*d + d elements
   size_t scratch_bytes = 0;
 
+  // per-segment ("layer-wise") plan, built when ADACONS_OPT_PER_SEGMENT is switched on
+  int seg_grid = 0;               // blocks of pass1_seg_kernel
+  int seg_records = 0;
+  const void* seg_kernel = nullptr;
+  long long* d_seg_off = nullptr;       // [S+1]
+  int* d_blk_first_seg = nullptr;       // [seg_grid]
+  int* d_blk_last_seg = nullptr;        // [seg_grid]
+  int* d_rec_begin = nullptr;           // [S]
+  int* d_rec_count = nullptr;           // [S]
+  int* d_set_first_block = nullptr;     // [S]
+  float* d_records = nullptr;           // [seg_records][2N]
+  int* d_pass2_blk_seg = nullptr;       // [pass-2 blocks]
+  size_t seg_bytes = 0;
+
   EncodeTiledFn encode = nullptr;
   CUtensorMap tmap;
   const void* tmap_for = nullptr;
@@ -104,6 +118,39 @@ const void* select_pass1(int dtype, int NR, int WR) {
   if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
   ADACONS_PICK(1)
 #undef ADACONS_PICK
+}
+
+template <int DT, int NR, int WR>
+const void* pass1_seg_fn() { return reinterpret_cast<const void*>(&pass1_seg_kernel<DT, NR, WR>); }
+
+const void* select_pass1_seg(int dtype, int NR, int WR) {
+#define ADACONS_PICK(DT)                                     \
+  if (WR == 1) {                                             \
+    if (NR == 1) return pass1_seg_fn<DT, 1, 1>();            \
+    if (NR == 2) return pass1_seg_fn<DT, 2, 1>();            \
+    if (NR == 4) return pass1_seg_fn<DT, 4, 1>();            \
+    return pass1_seg_fn<DT, 8, 1>();                         \
+  }                                                          \
+  if (WR == 2) return pass1_seg_fn<DT, 8, 2>();              \
+  if (WR == 4) return pass1_seg_fn<DT, 8, 4>();              \
+  return pass1_seg_fn<DT, 8, 8>();
+  if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
+  ADACONS_PICK(1)
+#undef ADACONS_PICK
+}
+
+// Launch with (or without) the programmatic-stream-serialisation attribute.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                          Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 int plan_fast(adacons_ctx* c) {
@@ -183,23 +230,109 @@ struct DeviceGuard {   // make the context's device current for the duration of 
 };
 
 int alloc_sets(adacons_ctx* c) {   // (re)allocate everything whose size depends on sets()
-  cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
-  c->partials = nullptr; c->coef = nullptr; c->gamma_f32 = nullptr; c->m = nullptr;
+  cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
+  c->coef = nullptr; c->gamma_f32 = nullptr; c->m = nullptr;
   const size_t sets = static_cast<size_t>(c->sets());
   const size_t N = static_cast<size_t>(c->N);
-  const size_t b_part = static_cast<size_t>(c->max_partials) * sets * 2 * N * sizeof(float);
   const size_t b_coef = 5 * sets * N * sizeof(double);
   const size_t b_gam = sets * N * sizeof(float);
   const size_t b_m = sets * N * sizeof(double);
-  if (cudaMalloc(&c->partials, b_part) != cudaSuccess || cudaMalloc(&c->coef, b_coef) != cudaSuccess ||
-      cudaMalloc(&c->gamma_f32, b_gam) != cudaSuccess || cudaMalloc(&c->m, b_m) != cudaSuccess) {
+  if (cudaMalloc(&c->coef, b_coef) != cudaSuccess || cudaMalloc(&c->gamma_f32, b_gam) != cudaSuccess ||
+      cudaMalloc(&c->m, b_m) != cudaSuccess) {
     cudaGetLastError();
     return ADACONS_ENOMEM;
   }
-  if (cudaMemset(c->partials, 0, b_part) != cudaSuccess || cudaMemset(c->coef, 0, b_coef) != cudaSuccess ||
-      cudaMemset(c->gamma_f32, 0, b_gam) != cudaSuccess || cudaMemset(c->m, 0, b_m) != cudaSuccess)
+  if (cudaMemset(c->coef, 0, b_coef) != cudaSuccess || cudaMemset(c->gamma_f32, 0, b_gam) != cudaSuccess ||
+      cudaMemset(c->m, 0, b_m) != cudaSuccess)
     return ADACONS_ECUDA;
-  c->scratch_bytes = b_part + b_coef + b_gam + b_m + sizeof(uint32_t) + sizeof(long long);
+  const size_t b_part = static_cast<size_t>(c->max_partials) * 2 * N * sizeof(float);
+  c->scratch_bytes = b_part + b_coef + b_gam + b_m + sizeof(uint32_t) + sizeof(long long) + c->seg_bytes;
+  return ADACONS_OK;
+}
+
+void free_seg_plan(adacons_ctx* c) {
+  cudaFree(c->d_seg_off); cudaFree(c->d_blk_first_seg); cudaFree(c->d_blk_last_seg); cudaFree(c->d_rec_begin);
+  cudaFree(c->d_rec_count); cudaFree(c->d_set_first_block); cudaFree(c->d_records); cudaFree(c->d_pass2_blk_seg);
+  c->d_seg_off = nullptr; c->d_blk_first_seg = c->d_blk_last_seg = c->d_rec_begin = c->d_rec_count = nullptr;
+  c->d_set_first_block = c->d_pass2_blk_seg = nullptr; c->d_records = nullptr;
+  c->seg_bytes = 0;
+  cudaGetLastError();
+}
+
+template <typename T>
+int upload(T** dst, const std::vector<T>& src, size_t* bytes) {
+  const size_t b = (src.empty() ? 1 : src.size()) * sizeof(T);
+  if (cudaMalloc(dst, b) != cudaSuccess) { cudaGetLastError(); return ADACONS_ENOMEM; }
+  if (!src.empty() && cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return ADACONS_ECUDA;
+  }
+  *bytes += b;
+  return ADACONS_OK;
+}
+
+// Host plan of the per-segment mode: which block meets which segments, where each (set, block)
+// partial record lives, and which segment each pass-2 block works in.
+int build_seg_plan(adacons_ctx* c) {
+  if (!c->fast.available) return ADACONS_EALIGN;   // needs the TMA path: N <= 64, 16-byte row pitch
+  free_seg_plan(c);
+  const int S = c->num_segments;
+  const std::vector<long long>& off = c->seg_offsets;
+  auto seg_of = [&](long long col) {   // the (non-empty) segment that contains column `col`
+    int lo = 0, hi = S;                // first index with off[idx] > col, minus one
+    while (lo < hi) { const int mid = (lo + hi) / 2; if (off[mid + 1] > col) hi = mid; else lo = mid + 1; }
+    return lo;
+  };
+  const int T = c->fast.num_tiles;
+  int G = c->fast.grid < T ? c->fast.grid : T;
+  const long long tilec = c->fast.tile_cols;
+  std::vector<int> first(G), last(G), rec_begin(S, 0), rec_count(S, 0), set_first(S, 0);
+  for (int b = 0; b < G; ++b) {
+    const long long t0 = static_cast<long long>(b) * T / G, t1 = static_cast<long long>(b + 1) * T / G;
+    const long long c0 = t0 * tilec, c1 = t1 * tilec < c->d ? t1 * tilec : c->d;
+    first[b] = seg_of(c0);
+    last[b] = seg_of(c1 - 1);
+    for (int sgm = first[b]; sgm <= last[b]; ++sgm) {
+      if (rec_count[sgm] == 0) set_first[sgm] = b;
+      rec_count[sgm] += 1;
+    }
+  }
+  int R = 0;
+  for (int sgm = 0; sgm < S; ++sgm) { rec_begin[sgm] = R; R += rec_count[sgm]; }
+  // pass 2: block bid covers vectors num_vec-1-(bid*256+255) .. num_vec-1-bid*256 (clipped at 0)
+  const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
+  const long long num_vec = c->d / vec;
+  const long long blocks2 = (num_vec + kThreads - 1) / kThreads;
+  std::vector<int> blk(static_cast<size_t>(blocks2));
+  for (long long bid = 0; bid < blocks2; ++bid) {
+    long long vlo = num_vec - 1 - (bid * kThreads + kThreads - 1);
+    if (vlo < 0) vlo = 0;
+    const long long vhi = num_vec - 1 - bid * kThreads;
+    const int slo = seg_of(vlo * vec), shi = seg_of(vhi * vec + vec - 1);
+    blk[static_cast<size_t>(bid)] = slo == shi ? slo : -(slo + 1);
+  }
+  size_t bytes = 0;
+  int rc;
+  if ((rc = upload(&c->d_seg_off, off, &bytes)) != ADACONS_OK) return rc;
+  if ((rc = upload(&c->d_blk_first_seg, first, &bytes)) != ADACONS_OK) return rc;
+  if ((rc = upload(&c->d_blk_last_seg, last, &bytes)) != ADACONS_OK) return rc;
+  if ((rc = upload(&c->d_rec_begin, rec_begin, &bytes)) != ADACONS_OK) return rc;
+  if ((rc = upload(&c->d_rec_count, rec_count, &bytes)) != ADACONS_OK) return rc;
+  if ((rc = upload(&c->d_set_first_block, set_first, &bytes)) != ADACONS_OK) return rc;
+  if ((rc = upload(&c->d_pass2_blk_seg, blk, &bytes)) != ADACONS_OK) return rc;
+  const size_t rb = static_cast<size_t>(R > 0 ? R : 1) * 2 * c->N * sizeof(float);
+  if (cudaMalloc(&c->d_records, rb) != cudaSuccess) { cudaGetLastError(); return ADACONS_ENOMEM; }
+  if (cudaMemset(c->d_records, 0, rb) != cudaSuccess) return ADACONS_ECUDA;
+  bytes += rb;
+  c->seg_grid = G;
+  c->seg_records = R;
+  c->seg_bytes = bytes;
+  c->seg_kernel = select_pass1_seg(c->dtype, c->fast.NR, c->fast.WR);
+  if (cudaFuncSetAttribute(c->seg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           static_cast<int>(c->fast.smem_bytes)) != cudaSuccess) {
+    cudaGetLastError();
+    return ADACONS_ECUDA;
+  }
   return ADACONS_OK;
 }
 
@@ -286,6 +419,9 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   if (cudaMemset(c->flags, 0, sizeof(uint32_t)) != cudaSuccess || cudaMemset(c->step, 0, sizeof(long long)) != cudaSuccess) {
     adacons_destroy(c); return ADACONS_ECUDA;
   }
+  const size_t b_part = static_cast<size_t>(c->max_partials) * 2 * N * sizeof(float);
+  if (cudaMalloc(&c->partials, b_part) != cudaSuccess) { cudaGetLastError(); adacons_destroy(c); return ADACONS_ENOMEM; }
+  if (cudaMemset(c->partials, 0, b_part) != cudaSuccess) { adacons_destroy(c); return ADACONS_ECUDA; }
   rc = alloc_sets(c);
   if (rc != ADACONS_OK) { adacons_destroy(c); return rc; }
   if (cudaDeviceSynchronize() != cudaSuccess) { adacons_destroy(c); return ADACONS_ECUDA; }
@@ -298,6 +434,7 @@ int adacons_destroy(adacons_ctx* c) {
   DeviceGuard g(c->device);
   cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
   cudaFree(c->flags); cudaFree(c->step); cudaFree(c->staging);
+  free_seg_plan(c);
   if (c->prof_ready)
     for (int s = 0; s < adacons_ctx::kProfSlots; ++s)
       for (int e = 0; e < 4; ++e) cudaEventDestroy(c->prof_ev[s][e]);
@@ -321,8 +458,27 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   cudaEvent_t* ev = (c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
   if (ev) cudaEventRecord(ev[0], st);
 
+  const bool pdl = (ev == nullptr);   // event records between the kernels would defeat the overlap anyway
+  const bool seg = c->per_segment != 0;
+  if (seg && !(aligned && c->fast.available && c->seg_kernel != nullptr)) return ADACONS_EALIGN;
+
   // ---- pass 1 (Eq. 7) ----
-  if (aligned && c->fast.available) {
+  if (seg) {
+    int rc = encode_map(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    Pass1SegParams p;
+    p.N = N; p.num_tiles = c->fast.num_tiles; p.stages = c->fast.stages; p.stage_bytes = c->fast.stage_bytes;
+    p.d = c->d; p.seg_off = c->d_seg_off; p.blk_first_seg = c->d_blk_first_seg; p.blk_last_seg = c->d_blk_last_seg;
+    p.rec_begin = c->d_rec_begin; p.set_first_block = c->d_set_first_block; p.records = c->d_records;
+    p.flags = c->flags;
+    void* args[2] = {&c->tmap, &p};
+    if (cudaLaunchKernel(c->seg_kernel, dim3(c->seg_grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    num_partials = 0;
+    c->last_path = 1;
+  } else if (aligned && c->fast.available) {
     int rc = encode_map(c, grads);
     if (rc != ADACONS_OK) return rc;
     Pass1Params p;
@@ -348,34 +504,45 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
 
   // ---- coefficients (Eq. 11, Eq. 12-13) ----
   CoeffParams q;
-  q.N = N; q.num_partials = num_partials; q.sets = 1; q.beta = c->beta;
+  q.N = N; q.num_partials = num_partials; q.sets = c->sets(); q.beta = c->beta;
   q.momentum = c->momentum; q.sorted = c->sorted; q.normalize = c->normalize;
-  q.partials = c->partials; q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m;
+  q.partials = seg ? c->d_records : c->partials;
+  q.rec_begin = seg ? c->d_rec_begin : nullptr;
+  q.rec_count = seg ? c->d_rec_count : nullptr;
+  q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m;
   q.flags = c->flags; q.step = c->step;
-  const int cthreads = ((N + 31) / 32) * 32;
-  coeff_kernel<<<1, cthreads, 0, st>>>(q);
-  if (!launch_ok()) return ADACONS_ECUDA;
+  int cthreads = 1024;
+  if (seg) { cthreads = ((2 * N + 31) / 32) * 32; if (cthreads > 1024) cthreads = 1024; }
+  if (launch_kernel(coeff_kernel, dim3(c->sets()), dim3(cthreads), 0, st, pdl, q) != cudaSuccess) {
+    cudaGetLastError();
+    return ADACONS_ECUDA;
+  }
   if (ev) cudaEventRecord(ev[2], st);
 
   // ---- pass 2 (Eq. 12) ----
+  cudaError_t e2;
   if (aligned) {
     const long long num_vec = c->d * c->elem_bytes / 16;
     const unsigned blocks = static_cast<unsigned>((num_vec + kThreads - 1) / kThreads);
     const long long row_bytes = c->d * c->elem_bytes;
+    const unsigned char* g8 = static_cast<const unsigned char*>(grads);
+    unsigned char* o8 = static_cast<unsigned char*>(out);
+    const int* bs = c->d_pass2_blk_seg;
+    const long long* so = c->d_seg_off;
     if (c->dtype == ADACONS_F32)
-      pass2_vec_kernel<0><<<blocks, kThreads, 0, st>>>(static_cast<const unsigned char*>(grads),
-                                                         static_cast<unsigned char*>(out), c->gamma_f32, N, row_bytes, num_vec);
+      e2 = seg ? launch_kernel(pass2_vec_kernel<0, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so)
+               : launch_kernel(pass2_vec_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so);
     else
-      pass2_vec_kernel<1><<<blocks, kThreads, 0, st>>>(static_cast<const unsigned char*>(grads),
-                                                         static_cast<unsigned char*>(out), c->gamma_f32, N, row_bytes, num_vec);
+      e2 = seg ? launch_kernel(pass2_vec_kernel<1, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so)
+               : launch_kernel(pass2_vec_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so);
   } else {
     const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);
     if (c->dtype == ADACONS_F32)
-      pass2_generic_kernel<0><<<blocks, kThreads, 0, st>>>(grads, out, c->gamma_f32, N, c->d);
+      e2 = launch_kernel(pass2_generic_kernel<0>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d);
     else
-      pass2_generic_kernel<1><<<blocks, kThreads, 0, st>>>(grads, out, c->gamma_f32, N, c->d);
+      e2 = launch_kernel(pass2_generic_kernel<1>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d);
   }
-  if (!launch_ok()) return ADACONS_ECUDA;
+  if (e2 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
   if (ev) { cudaEventRecord(ev[3], st); c->prof_calls += 1; }
   c->total_launches += 3;
   return ADACONS_OK;
@@ -424,9 +591,25 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
     case ADACONS_OPT_MOMENTUM: c->momentum = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_SORTED: c->sorted = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_NORMALIZE: c->normalize = value != 0.0; return ADACONS_OK;
-    case ADACONS_OPT_PER_SEGMENT:
-      if (value != 0.0) return ADACONS_EINVAL;   // layer-wise mode: not available in this build
+    case ADACONS_OPT_PER_SEGMENT: {
+      const int want = value != 0.0;
+      if (want == c->per_segment) return ADACONS_OK;
+      DeviceGuard guard(c->device);
+      if (!guard.ok) return ADACONS_ECUDA;
+      if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+      if (want) {
+        const int rc = build_seg_plan(c);
+        if (rc != ADACONS_OK) { free_seg_plan(c); return rc; }
+      } else {
+        free_seg_plan(c);
+      }
+      c->per_segment = want;
+      int rc = alloc_sets(c);                      // state, coefficients: one set per segment; zeroed
+      if (rc != ADACONS_OK) return rc;
+      if (cudaMemset(c->flags, 0, sizeof(uint32_t)) != cudaSuccess || cudaMemset(c->step, 0, sizeof(long long)) != cudaSuccess)
+        return ADACONS_ECUDA;
       return ADACONS_OK;
+    }
     case ADACONS_OPT_PROFILE: {
       DeviceGuard guard(c->device);
       if (!guard.ok) return ADACONS_ECUDA;

@@ -81,6 +81,11 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, u
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may
+// start before its predecessor in the stream has finished; it must call pdl_wait() before it
+// touches anything the predecessor writes.  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ uint4 ld_shared_v4(const void* p) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_addr(p)));
@@ -112,16 +117,160 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
 // ----------------------------------------------------------------------------------------------
 // Pass 1, TMA-staged (N <= 64, 16-byte aligned rows).
 //
-// A block owns column tiles  t = blockIdx.x, blockIdx.x + gridDim.x, ...  A tile is WC boxes of
-// N rows x 512 bytes, laid side by side; the 8 warps form a WR x WC grid (WR * WC = 8): warp
-// (rw, cw) reads box cw and rows rw, rw+WR, ... (NR of them); lane l owns the 16-byte column
-// group l of the box.  Per tile every thread
+// A tile is WC boxes of N rows x 512 bytes, laid side by side; the 8 warps form a WR x WC grid
+// (WR * WC = 8): warp (rw, cw) reads box cw and rows rw, rw+WR, ... (NR of them); lane l owns the
+// 16-byte column group l of the box.  Per tile every thread
 //   1. copies its NR row vectors from shared memory to registers,
 //   2. adds them up (partial column sums); with WR > 1 the WR partials are exchanged through
 //      shared memory and added in a fixed order, giving the column sums s of the tile,
 //   3. accumulates, per row, sum x*s and sum x*x in fp32 (two lanes of packed fp32 FMA).
 // One elected thread refills a stage by TMA as soon as the block has copied it to registers.
+//
+// Two kernels share these steps: pass1_tma_kernel (one set of coefficients for the whole vector;
+// a block owns tiles b, b+grid, ...) and pass1_seg_kernel (one set per segment; a block owns a
+// contiguous tile range and writes one partial record per segment it meets).
 // ----------------------------------------------------------------------------------------------
+template <int DT, int NR_, int WR_>
+struct P1 {
+  static constexpr int NR = NR_, WR = WR_;
+  static constexpr int WC = kWarps / WR;
+  static constexpr int VEC = Elem<DT>::kVec;
+  static constexpr int NP = VEC / 2;
+  static constexpr int BOXC = kBoxRowBytes / Elem<DT>::kBytes;   // columns per box
+  static constexpr int TILEC = WC * BOXC;                        // columns per tile
+  static constexpr int kXchOne = WR * WC * 32 * VEC;             // floats of one exchange buffer
+  static constexpr int kXchFloats = (WR > 1) ? 2 * kXchOne : 0;
+  static constexpr int kRedFloats = kWarps * NR * 2;
+};
+
+struct P1Smem {            // carve-up of the dynamic shared memory of both pass-1 kernels
+  unsigned char* stage_base;
+  float* xch;
+  float* red;
+  uint64_t* full;
+};
+template <class C>
+__device__ __forceinline__ P1Smem p1_carve(unsigned char* raw, int stages, uint32_t stage_bytes) {
+  P1Smem s;
+  s.stage_base = raw;
+  s.xch = reinterpret_cast<float*>(raw + static_cast<size_t>(stages) * stage_bytes);
+  s.red = s.xch + C::kXchFloats;
+  s.full = reinterpret_cast<uint64_t*>(s.red + C::kRedFloats);
+  return s;
+}
+
+// rows of this thread from a landed stage (zeros for rows >= N)
+template <class C>
+__device__ __forceinline__ void p1_load_rows(uint4 (&v)[C::NR], const unsigned char* box_lane, int rw, int N) {
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j) {
+    const int row = rw + C::WR * j;
+    v[j] = (row < N) ? ld_shared_v4(box_lane + row * kBoxRowBytes) : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+template <int DT, class C>
+__device__ __forceinline__ void p1_colsum(const uint4 (&v)[C::NR], float2 (&sp)[C::NP]) {
+#pragma unroll
+  for (int h = 0; h < C::NP; ++h) sp[h] = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j)
+#pragma unroll
+    for (int h = 0; h < C::NP; ++h) sp[h] = __fadd2_rn(sp[h], unpack_pair<DT>(v[j], h));
+}
+// exchange layout [rw][cw][16-byte half h2][lane][4 floats]: conflict-free 16-byte accesses
+template <class C>
+__device__ __forceinline__ void p1_xch_write(float* xbuf, const float2 (&sp)[C::NP], int rw, int cw, int lane) {
+#pragma unroll
+  for (int h2 = 0; h2 < C::VEC / 4; ++h2) {
+    const float4 w4 = make_float4(sp[2 * h2].x, sp[2 * h2].y, sp[2 * h2 + 1].x, sp[2 * h2 + 1].y);
+    *reinterpret_cast<float4*>(xbuf + ((rw * C::WC + cw) * (C::VEC / 4) + h2) * 128 + lane * 4) = w4;
+  }
+}
+template <class C>
+__device__ __forceinline__ void p1_xch_read(const float* xbuf, float2 (&sp)[C::NP], int cw, int lane) {
+#pragma unroll
+  for (int h = 0; h < C::NP; ++h) sp[h] = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int r = 0; r < C::WR; ++r)
+#pragma unroll
+    for (int h2 = 0; h2 < C::VEC / 4; ++h2) {
+      const float4 w4 = *reinterpret_cast<const float4*>(xbuf + ((r * C::WC + cw) * (C::VEC / 4) + h2) * 128 + lane * 4);
+      sp[2 * h2] = __fadd2_rn(sp[2 * h2], make_float2(w4.x, w4.y));
+      sp[2 * h2 + 1] = __fadd2_rn(sp[2 * h2 + 1], make_float2(w4.z, w4.w));
+    }
+}
+template <int DT, class C>
+__device__ __forceinline__ void p1_accumulate(const uint4 (&v)[C::NR], const float2 (&sp)[C::NP],
+                                              float2 (&pacc)[C::NR], float2 (&qacc)[C::NR]) {
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j)
+#pragma unroll
+    for (int h = 0; h < C::NP; ++h) {
+      const float2 x = unpack_pair<DT>(v[j], h);
+      pacc[j] = __ffma2_rn(x, sp[h], pacc[j]);
+      qacc[j] = __ffma2_rn(x, x, qacc[j]);
+    }
+}
+// same, counting only the columns lo <= col < hi; col0 = column of this lane's first element
+template <int DT, class C>
+__device__ __forceinline__ void p1_accumulate_masked(const uint4 (&v)[C::NR], const float2 (&sp)[C::NP],
+                                                     float2 (&pacc)[C::NR], float2 (&qacc)[C::NR],
+                                                     long long col0, long long lo, long long hi) {
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j)
+#pragma unroll
+    for (int h = 0; h < C::NP; ++h) {
+      float2 x = unpack_pair<DT>(v[j], h);
+      const long long c = col0 + 2 * h;
+      if (c < lo || c >= hi) x.x = 0.f;
+      if (c + 1 < lo || c + 1 >= hi) x.y = 0.f;
+      pacc[j] = __ffma2_rn(x, sp[h], pacc[j]);
+      qacc[j] = __ffma2_rn(x, x, qacc[j]);
+    }
+}
+// Block partial of the accumulators: lanes (fixed xor tree), then the WC warps that share a row
+// (fixed order).  dst[0..N) = N p_i (un-divided), dst[N..2N) = q_i.  Contains two barriers; the
+// accumulators are reset.
+template <class C>
+__device__ __forceinline__ void p1_block_store(float2 (&pacc)[C::NR], float2 (&qacc)[C::NR], float* red,
+                                               float* dst, int N) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j) {
+    float p = pacc[j].x + pacc[j].y, q = qacc[j].x + qacc[j].y;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      p += __shfl_xor_sync(0xffffffffu, p, o);
+      q += __shfl_xor_sync(0xffffffffu, q, o);
+    }
+    if (lane == 0) {
+      red[(warp * C::NR + j) * 2 + 0] = p;
+      red[(warp * C::NR + j) * 2 + 1] = q;
+    }
+    pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  }
+  __syncthreads();
+  if (tid < N) {
+    const int r_w = tid % C::WR, j = tid / C::WR;
+    float p = 0.f, q = 0.f;
+#pragma unroll
+    for (int c = 0; c < C::WC; ++c) {
+      p += red[((c * C::WR + r_w) * C::NR + j) * 2 + 0];
+      q += red[((c * C::WR + r_w) * C::NR + j) * 2 + 1];
+    }
+    dst[tid] = p;
+    dst[N + tid] = q;
+  }
+  __syncthreads();
+}
+// After a bounded wait expired: wait (bounded) for the copies still in flight into this block's
+// shared memory so that the block may exit, and report.
+__device__ __forceinline__ void p1_drain_after_timeout(uint64_t* full, int stages, int issued, uint32_t* flags) {
+  for (int k = (issued > stages ? issued - stages : 0); k < issued; ++k)
+    (void)mbar_wait_bounded(&full[k % stages], static_cast<uint32_t>(k / stages) & 1u);
+  atomicOr(flags, kFlagTimeout);
+}
+
 struct Pass1Params {
   int N;
   int num_tiles;        // ceil(d / tile columns)
@@ -134,166 +283,209 @@ struct Pass1Params {
 template <int DT, int NR, int WR>
 __global__ void __launch_bounds__(kThreads, 2)
 pass1_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm) {
-  constexpr int WC = kWarps / WR;
-  constexpr int VEC = Elem<DT>::kVec;
-  constexpr int NP = VEC / 2;
-  constexpr int BOXC = kBoxRowBytes / Elem<DT>::kBytes;   // columns per box
-  constexpr int TILEC = WC * BOXC;                        // columns per tile
-
+  using C = P1<DT, NR, WR>;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int s_abort;
   const int N = prm.N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int cw = warp / WR, rw = warp % WR;
-
-  unsigned char* stage_base = smem_raw;
-  unsigned char* after = smem_raw + static_cast<size_t>(prm.stages) * prm.stage_bytes;
-  float* xch = reinterpret_cast<float*>(after);                           // [2][WR][WC*32*VEC]
-  constexpr int kXchFloats = (WR > 1) ? 2 * WR * WC * 32 * VEC : 0;
-  float* red = xch + kXchFloats;                                          // [kWarps][NR][2]
-  uint64_t* full = reinterpret_cast<uint64_t*>(red + kWarps * NR * 2);    // [stages]
-  __shared__ int s_abort;
+  const P1Smem sm = p1_carve<C>(smem_raw, prm.stages, prm.stage_bytes);
 
   if (tid == 0) {
     s_abort = 0;
-    for (int s = 0; s < prm.stages; ++s) mbar_init(&full[s], 1);
+    for (int s = 0; s < prm.stages; ++s) mbar_init(&sm.full[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async_smem();
   }
   __syncthreads();
+  pdl_launch_dependents();
 
   const int first = blockIdx.x;
   const int stride = gridDim.x;
   const int my_tiles = first < prm.num_tiles ? (prm.num_tiles - first + stride - 1) / stride : 0;
 
-  auto issue = [&](int k) {   // elected thread: fill stage k % stages with tile k of this block
-    const int s = k % prm.stages;
-    const int col0 = (first + k * stride) * TILEC;
-    mbar_expect_tx(&full[s], prm.stage_bytes);
+  auto issue = [&](int k, int s) {   // elected thread: fill stage s with tile k of this block
+    const int col0 = (first + k * stride) * C::TILEC;
+    mbar_expect_tx(&sm.full[s], prm.stage_bytes);
 #pragma unroll
-    for (int c = 0; c < WC; ++c)
-      tma_load_2d(stage_base + static_cast<size_t>(s) * prm.stage_bytes + static_cast<size_t>(c) * N * kBoxRowBytes,
-                  &tmap, &full[s], col0 + c * BOXC, 0);
+    for (int c = 0; c < C::WC; ++c)
+      tma_load_2d(sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes + static_cast<size_t>(c) * N * kBoxRowBytes,
+                  &tmap, &sm.full[s], col0 + c * C::BOXC, 0);
   };
+  int issued = 0;                    // meaningful in thread 0 only
   if (tid == 0) {
     const int pre = my_tiles < prm.stages ? my_tiles : prm.stages;
-    for (int k = 0; k < pre; ++k) issue(k);
+    for (int k = 0; k < pre; ++k) issue(k, k);
+    issued = pre;
   }
 
   float2 pacc[NR], qacc[NR];
 #pragma unroll
   for (int j = 0; j < NR; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
 
-  bool timed_out = false;
-  int issued_upto = my_tiles < prm.stages ? my_tiles : prm.stages;   // meaningful in thread 0 only
-
+  int s = 0;
+  uint32_t parity = 0;
   for (int k = 0; k < my_tiles; ++k) {
-    const int s = k % prm.stages;
-    const uint32_t parity = static_cast<uint32_t>(k / prm.stages) & 1u;
     uint4 v[NR];
-#pragma unroll
-    for (int j = 0; j < NR; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
-    if (mbar_wait_bounded(&full[s], parity)) {
-      const unsigned char* box = stage_base + static_cast<size_t>(s) * prm.stage_bytes +
-                                 static_cast<size_t>(cw) * N * kBoxRowBytes + lane * 16;
-#pragma unroll
-      for (int j = 0; j < NR; ++j) {
-        const int row = rw + WR * j;
-        if (row < N) v[j] = ld_shared_v4(box + row * kBoxRowBytes);
-      }
+    if (mbar_wait_bounded(&sm.full[s], parity)) {
+      p1_load_rows<C>(v, sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes +
+                             static_cast<size_t>(cw) * N * kBoxRowBytes + lane * 16, rw, N);
     } else {
-      timed_out = true;
+#pragma unroll
+      for (int j = 0; j < NR; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
       atomicOr(&s_abort, 1);
     }
-
-    // partial column sums over this warp's rows (rows in index order)
-    float2 sp[NP];
-#pragma unroll
-    for (int h = 0; h < NP; ++h) sp[h] = make_float2(0.f, 0.f);
-#pragma unroll
-    for (int j = 0; j < NR; ++j)
-#pragma unroll
-      for (int h = 0; h < NP; ++h) sp[h] = __fadd2_rn(sp[h], unpack_pair<DT>(v[j], h));
-
-    float* xbuf = xch + (k & 1) * (WR * WC * 32 * VEC);
-    if (WR > 1) {
-      // layout [rw][cw][half h2][lane][4 floats]: conflict-free 16-byte accesses
-#pragma unroll
-      for (int h2 = 0; h2 < VEC / 4; ++h2) {
-        float4 w4 = make_float4(sp[2 * h2].x, sp[2 * h2].y, sp[2 * h2 + 1].x, sp[2 * h2 + 1].y);
-        *reinterpret_cast<float4*>(xbuf + ((rw * WC + cw) * (VEC / 4) + h2) * 128 + lane * 4) = w4;
-      }
-    }
+    float2 sp[C::NP];
+    p1_colsum<DT, C>(v, sp);
+    float* xbuf = sm.xch + (k & 1) * C::kXchOne;
+    if (WR > 1) p1_xch_write<C>(xbuf, sp, rw, cw, lane);
     __syncthreads();   // every thread holds its rows in registers; exchange buffer is written
     if (s_abort) break;
     if (tid == 0 && k + prm.stages < my_tiles) {
       fence_proxy_async_smem();
-      issue(k + prm.stages);
-      issued_upto = k + prm.stages + 1;
+      issue(k + prm.stages, s);
+      issued = k + prm.stages + 1;
     }
-    if (WR > 1) {
+    if (WR > 1) p1_xch_read<C>(xbuf, sp, cw, lane);
+    p1_accumulate<DT, C>(v, sp, pacc, qacc);
+    if (++s == prm.stages) { s = 0; parity ^= 1u; }
+  }
+
+  float* dst = prm.partials + static_cast<size_t>(blockIdx.x) * 2 * N;
+  if (s_abort) {
+    if (tid == 0) p1_drain_after_timeout(sm.full, prm.stages, issued, prm.flags);
+    if (tid < 2 * N) dst[tid] = 0.f;
+    return;
+  }
+  p1_block_store<C>(pacc, qacc, sm.red, dst, N);
+}
+
+// ---- per-segment ("layer-wise") pass 1 ----------------------------------------------------------
+// Block b owns the contiguous tile range [b*T/G, (b+1)*T/G).  The column sums of a tile do not
+// depend on the segments; only the destination of x*s and x*x does.  The block keeps accumulators
+// for its current segment and, whenever that segment ends inside (or at the end of) a tile,
+// reduces them to one record and moves on; a tile that contains a boundary is accumulated once per
+// segment it meets, with the columns outside the segment masked to zero.  Records of set s are
+// contiguous: record (rec_begin[s] + b - set_first_block[s]) belongs to block b.
+struct Pass1SegParams {
+  int N;
+  int num_tiles;
+  int stages;
+  uint32_t stage_bytes;
+  long long d;
+  const long long* seg_off;       // [S+1]
+  const int* blk_first_seg;       // [grid] segment that contains the block's first column
+  const int* blk_last_seg;        // [grid] segment that contains the block's last column
+  const int* rec_begin;           // [S]
+  const int* set_first_block;     // [S]
+  float* records;                 // [num_records][2N]
+  uint32_t* flags;
+};
+
+template <int DT, int NR, int WR>
+__global__ void __launch_bounds__(kThreads, 2)
+pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams prm) {
+  using C = P1<DT, NR, WR>;
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int s_abort;
+  const int N = prm.N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cw = warp / WR, rw = warp % WR;
+  const P1Smem sm = p1_carve<C>(smem_raw, prm.stages, prm.stage_bytes);
+
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < prm.stages; ++s) mbar_init(&sm.full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+
+  const int b = blockIdx.x, G = gridDim.x;
+  const int t0 = static_cast<int>(static_cast<long long>(b) * prm.num_tiles / G);
+  const int t1 = static_cast<int>(static_cast<long long>(b + 1) * prm.num_tiles / G);
+  const int my_tiles = t1 - t0;
+
+  auto issue = [&](int k, int s) {
+    const int col0 = (t0 + k) * C::TILEC;
+    mbar_expect_tx(&sm.full[s], prm.stage_bytes);
 #pragma unroll
-      for (int h = 0; h < NP; ++h) sp[h] = make_float2(0.f, 0.f);
+    for (int c = 0; c < C::WC; ++c)
+      tma_load_2d(sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes + static_cast<size_t>(c) * N * kBoxRowBytes,
+                  &tmap, &sm.full[s], col0 + c * C::BOXC, 0);
+  };
+  int issued = 0;
+  if (tid == 0) {
+    const int pre = my_tiles < prm.stages ? my_tiles : prm.stages;
+    for (int k = 0; k < pre; ++k) issue(k, k);
+    issued = pre;
+  }
+
+  float2 pacc[NR], qacc[NR];
 #pragma unroll
-      for (int r = 0; r < WR; ++r)
+  for (int j = 0; j < NR; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+
+  int seg = prm.blk_first_seg[b];
+  const int last_seg = prm.blk_last_seg[b];
+  long long seg_end = prm.seg_off[seg + 1];
+  auto record = [&](int sg) -> float* {
+    return prm.records + static_cast<size_t>(prm.rec_begin[sg] + b - prm.set_first_block[sg]) * 2 * N;
+  };
+
+  int s = 0;
+  uint32_t parity = 0;
+  for (int k = 0; k < my_tiles; ++k) {
+    uint4 v[NR];
+    if (mbar_wait_bounded(&sm.full[s], parity)) {
+      p1_load_rows<C>(v, sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes +
+                             static_cast<size_t>(cw) * N * kBoxRowBytes + lane * 16, rw, N);
+    } else {
 #pragma unroll
-        for (int h2 = 0; h2 < VEC / 4; ++h2) {
-          const float4 w4 = *reinterpret_cast<const float4*>(xbuf + ((r * WC + cw) * (VEC / 4) + h2) * 128 + lane * 4);
-          sp[2 * h2] = __fadd2_rn(sp[2 * h2], make_float2(w4.x, w4.y));
-          sp[2 * h2 + 1] = __fadd2_rn(sp[2 * h2 + 1], make_float2(w4.z, w4.w));
+      for (int j = 0; j < NR; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
+      atomicOr(&s_abort, 1);
+    }
+    float2 sp[C::NP];
+    p1_colsum<DT, C>(v, sp);
+    float* xbuf = sm.xch + (k & 1) * C::kXchOne;
+    if (WR > 1) p1_xch_write<C>(xbuf, sp, rw, cw, lane);
+    __syncthreads();
+    if (s_abort) break;
+    if (tid == 0 && k + prm.stages < my_tiles) {
+      fence_proxy_async_smem();
+      issue(k + prm.stages, s);
+      issued = k + prm.stages + 1;
+    }
+    if (WR > 1) p1_xch_read<C>(xbuf, sp, cw, lane);
+
+    const long long tile_lo = static_cast<long long>(t0 + k) * C::TILEC;
+    const long long tile_hi = tile_lo + C::TILEC < prm.d ? tile_lo + C::TILEC : prm.d;
+    if (seg_end > tile_hi || seg >= last_seg) {
+      p1_accumulate<DT, C>(v, sp, pacc, qacc);                  // whole tile inside the current segment
+    } else {
+      const long long col0 = tile_lo + cw * C::BOXC + lane * C::VEC;
+      long long lo = tile_lo;
+      for (;;) {                                                // block-uniform control flow
+        const long long hi = seg_end < tile_hi ? seg_end : tile_hi;
+        if (hi > lo) p1_accumulate_masked<DT, C>(v, sp, pacc, qacc, col0, lo, hi);
+        if (seg_end <= tile_hi && seg < last_seg) {
+          p1_block_store<C>(pacc, qacc, sm.red, record(seg), N);
+          ++seg;
+          seg_end = prm.seg_off[seg + 1];
+          lo = hi;                                              // empty segments fall through here
+        } else {
+          break;
         }
-    }
-#pragma unroll
-    for (int j = 0; j < NR; ++j)
-#pragma unroll
-      for (int h = 0; h < NP; ++h) {
-        const float2 x = unpack_pair<DT>(v[j], h);
-        pacc[j] = __ffma2_rn(x, sp[h], pacc[j]);
-        qacc[j] = __ffma2_rn(x, x, qacc[j]);
       }
+    }
+    if (++s == prm.stages) { s = 0; parity ^= 1u; }
   }
 
   if (s_abort) {
-    // Leave cleanly: wait (bounded) for the copies still in flight into this block's shared
-    // memory, report, and write zero partials so that the finish kernel reads defined data.
-    if (tid == 0) {
-      for (int k = 0; k < issued_upto; ++k) {
-        // stages whose latest fill has not been consumed: the last `stages` issued tiles
-        if (k + prm.stages >= issued_upto)
-          (void)mbar_wait_bounded(&full[k % prm.stages], static_cast<uint32_t>(k / prm.stages) & 1u);
-      }
-      atomicOr(prm.flags, kFlagTimeout);
-    }
-    (void)timed_out;
-    if (tid < 2 * N) prm.partials[static_cast<size_t>(blockIdx.x) * 2 * N + tid] = 0.f;
-    return;
+    if (tid == 0) p1_drain_after_timeout(sm.full, prm.stages, issued, prm.flags);
+    return;   // the records keep whatever they held; the status word says the result is invalid
   }
-
-  // block partial: lanes (fixed xor tree), then the WC warps that share a row (fixed order)
-#pragma unroll
-  for (int j = 0; j < NR; ++j) {
-    float p = pacc[j].x + pacc[j].y, q = qacc[j].x + qacc[j].y;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      p += __shfl_xor_sync(0xffffffffu, p, o);
-      q += __shfl_xor_sync(0xffffffffu, q, o);
-    }
-    if (lane == 0) {
-      red[(warp * NR + j) * 2 + 0] = p;
-      red[(warp * NR + j) * 2 + 1] = q;
-    }
-  }
-  __syncthreads();
-  if (tid < N) {
-    const int r_w = tid % WR, j = tid / WR;
-    float p = 0.f, q = 0.f;
-#pragma unroll
-    for (int c = 0; c < WC; ++c) {
-      p += red[((c * WR + r_w) * NR + j) * 2 + 0];
-      q += red[((c * WR + r_w) * NR + j) * 2 + 1];
-    }
-    prm.partials[static_cast<size_t>(blockIdx.x) * 2 * N + tid] = p;
-    prm.partials[static_cast<size_t>(blockIdx.x) * 2 * N + N + tid] = q;
-  }
+  p1_block_store<C>(pacc, qacc, sm.red, record(seg), N);
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -366,15 +558,19 @@ pass1_generic_kernel(const void* __restrict__ grads, int N, long long d, int num
 }
 
 // ----------------------------------------------------------------------------------------------
-// Coefficient step: one block per coefficient set, thread i = worker i.
+// Coefficient step: one block per coefficient set.  The partial records of the set are added in
+// fp64 in a fixed order (threads split them into `groups` interleaved subsequences, which are
+// then added in group order); afterwards thread i = worker i.
 // ----------------------------------------------------------------------------------------------
 struct CoeffParams {
   int N;
-  int num_partials;      // rows of `partials` to add up (fixed order 0..num_partials-1)
-  int sets;              // coefficient sets (1 = whole vector); partials are [num_partials][sets][2N]
+  int num_partials;      // global mode: records 0..num_partials-1 belong to the one set
+  int sets;
   double beta;
   int momentum, sorted, normalize;
-  const float* partials;
+  const float* partials; // [records][2N]
+  const int* rec_begin;  // per set (nullptr in global mode)
+  const int* rec_count;
   double* coef;          // [5][sets][N]: a, a~, gamma, p, q   (enum adacons_coeff order)
   float* gamma_f32;      // [sets][N]   weights as pass 2 reads them
   double* m;             // [sets][N]   momentum state, in place
@@ -384,24 +580,43 @@ struct CoeffParams {
 
 __global__ void __launch_bounds__(kMaxN)
 coeff_kernel(const CoeffParams prm) {
+  __shared__ double sh_part[2 * kMaxN];
   __shared__ double sh_a[kMaxN];
   __shared__ double sh_u[kMaxN];
   __shared__ int sh_bad, sh_zero;
   __shared__ double sh_Z;
   __shared__ int sh_uniform;
-  const int N = prm.N, i = threadIdx.x, set = blockIdx.x;
+  const int N = prm.N, i = threadIdx.x, set = blockIdx.x, T = blockDim.x;
+  const int V = 2 * N;
   const size_t per = static_cast<size_t>(prm.sets) * N;   // stride between coefficient kinds
   if (i == 0) { sh_bad = 0; sh_zero = 0; }
+  pdl_launch_dependents();
+  pdl_wait();                                              // pass 1 has finished and is visible
+  const int begin = prm.rec_begin ? prm.rec_begin[set] : 0;
+  const int count = prm.rec_count ? prm.rec_count[set] : prm.num_partials;
+  const float* base = prm.partials + static_cast<size_t>(begin) * V;
+  const int groups = T >= V ? T / V : 1;
+  if (T >= V) {
+    const int g = i / V, v = i % V;
+    if (g < groups) {
+      double acc = 0.0;
+#pragma unroll 4
+      for (int c = g; c < count; c += groups) acc += static_cast<double>(base[static_cast<size_t>(c) * V + v]);
+      sh_part[g * V + v] = acc;
+    }
+  } else {
+    for (int v = i; v < V; v += T) {
+      double acc = 0.0;
+#pragma unroll 4
+      for (int c = 0; c < count; ++c) acc += static_cast<double>(base[static_cast<size_t>(c) * V + v]);
+      sh_part[v] = acc;
+    }
+  }
   __syncthreads();
   double p = 0.0, q = 0.0;
   if (i < N) {
     double P = 0.0, Q = 0.0;
-    const float* base = prm.partials + static_cast<size_t>(set) * 2 * N;
-    const size_t row = static_cast<size_t>(prm.sets) * 2 * N;
-    for (int c = 0; c < prm.num_partials; ++c) {
-      P += static_cast<double>(base[c * row + i]);
-      Q += static_cast<double>(base[c * row + N + i]);
-    }
+    for (int g = 0; g < groups; ++g) { P += sh_part[g * V + i]; Q += sh_part[g * V + N + i]; }
     p = P / static_cast<double>(N);   // gbar is the mean of the workers (text before Eq. 7)
     q = Q;
     if (!(isfinite(p) && isfinite(q))) atomicOr(&sh_bad, 1);
@@ -475,43 +690,12 @@ coeff_kernel(const CoeffParams prm) {
 // Pass 2, vectorised (16-byte aligned rows).  One thread per 16-byte column group; the groups
 // are visited from the END of the vector so that the columns pass 1 touched last, which are
 // still in L2, are read first.  Rows are added in index order with fp32 FMA.
+// SEG = true: one weight set per segment.  blk_seg[b] >= 0 names the single segment that holds
+// all columns of block b; otherwise -(s+1), s = segment of the block's lowest column, and every
+// thread finds the segment of each of its columns itself.
 // ----------------------------------------------------------------------------------------------
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
-                 const float* __restrict__ gamma, int N, long long row_bytes, long long num_vec) {
-  constexpr int VEC = Elem<DT>::kVec;
-  constexpr int NP = VEC / 2;
-  constexpr int U = 8;                               // row loads in flight per thread
-  __shared__ float g_s[kMaxN];
-  for (int i = threadIdx.x; i < N; i += kThreads) g_s[i] = gamma[i];
-  __syncthreads();
-  const long long v = num_vec - 1 - (static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x);
-  if (v < 0) return;
-  const unsigned char* col = grads + v * 16;
-  float2 acc[NP];
-#pragma unroll
-  for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
-  int i0 = 0;
-  for (; i0 + U <= N; i0 += U) {
-    uint4 x[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) x[u] = ld_stream_v4(col + static_cast<long long>(i0 + u) * row_bytes);
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const float g = g_s[i0 + u];
-      const float2 g2 = make_float2(g, g);
-#pragma unroll
-      for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(x[u], h), g2, acc[h]);
-    }
-  }
-  for (; i0 < N; ++i0) {
-    const uint4 x = ld_stream_v4(col + static_cast<long long>(i0) * row_bytes);
-    const float g = g_s[i0];
-    const float2 g2 = make_float2(g, g);
-#pragma unroll
-    for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, acc[h]);
-  }
+template <int DT, int NP>
+__device__ __forceinline__ void pass2_store(unsigned char* out, long long v, const float2 (&acc)[NP]) {
   uint4 o;
   if constexpr (DT == 0) {
     o = make_uint4(__float_as_uint(acc[0].x), __float_as_uint(acc[0].y), __float_as_uint(acc[1].x),
@@ -523,12 +707,84 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
   *reinterpret_cast<uint4*>(out + v * 16) = o;
 }
 
+template <int DT, bool SEG>
+__global__ void __launch_bounds__(kThreads)
+pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
+                 const float* __restrict__ gamma, int N, long long row_bytes, long long num_vec,
+                 const int* __restrict__ blk_seg, const long long* __restrict__ seg_off) {
+  constexpr int VEC = Elem<DT>::kVec;
+  constexpr int NP = VEC / 2;
+  constexpr int U = 8;                               // row loads in flight per thread
+  __shared__ float g_s[kMaxN];
+  pdl_wait();                                        // the coefficient step has finished
+  int code = 0;
+  if (SEG) code = blk_seg[blockIdx.x];
+  const long long v = num_vec - 1 - (static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x);
+  if (!SEG || code >= 0) {
+    const float* gsrc = gamma + static_cast<size_t>(SEG ? code : 0) * N;
+    for (int i = threadIdx.x; i < N; i += kThreads) g_s[i] = gsrc[i];
+    __syncthreads();
+    if (v < 0) return;
+    const unsigned char* col = grads + v * 16;
+    float2 acc[NP];
+#pragma unroll
+    for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+    int i0 = 0;
+    for (; i0 + U <= N; i0 += U) {
+      uint4 x[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) x[u] = ld_stream_v4(col + static_cast<long long>(i0 + u) * row_bytes);
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const float g = g_s[i0 + u];
+        const float2 g2 = make_float2(g, g);
+#pragma unroll
+        for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(x[u], h), g2, acc[h]);
+      }
+    }
+    for (; i0 < N; ++i0) {
+      const uint4 x = ld_stream_v4(col + static_cast<long long>(i0) * row_bytes);
+      const float g = g_s[i0];
+      const float2 g2 = make_float2(g, g);
+#pragma unroll
+      for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, acc[h]);
+    }
+    pass2_store<DT, NP>(out, v, acc);
+  } else {
+    if (v < 0) return;
+    int sg = -code - 1;
+    int seg_of[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) {
+      const long long c = v * VEC + e;
+      while (c >= seg_off[sg + 1]) ++sg;             // segments are ascending; empty ones are skipped
+      seg_of[e] = sg;
+    }
+    const unsigned char* col = grads + v * 16;
+    float2 acc[NP];
+#pragma unroll
+    for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+    for (int i = 0; i < N; ++i) {
+      const uint4 x = ld_stream_v4(col + static_cast<long long>(i) * row_bytes);
+#pragma unroll
+      for (int h = 0; h < NP; ++h) {
+        const float2 xv = unpack_pair<DT>(x, h);
+        const float2 g2 = make_float2(gamma[static_cast<size_t>(seg_of[2 * h]) * N + i],
+                                      gamma[static_cast<size_t>(seg_of[2 * h + 1]) * N + i]);
+        acc[h] = __ffma2_rn(xv, g2, acc[h]);
+      }
+    }
+    pass2_store<DT, NP>(out, v, acc);
+  }
+}
+
 // Pass 2, generic: one thread per column, scalar loads.
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 pass2_generic_kernel(const void* __restrict__ grads, void* __restrict__ out, const float* __restrict__ gamma,
                      int N, long long d) {
   __shared__ float g_s[kMaxN];
+  pdl_wait();
   for (int i = threadIdx.x; i < N; i += kThreads) g_s[i] = gamma[i];
   __syncthreads();
   const long long k = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;

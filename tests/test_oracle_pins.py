@@ -268,6 +268,22 @@ def test_momentum_state_is_the_ema_of_order_statistics():
         np.testing.assert_allclose(r["a_tilde"][0], np.array(want)[ranks], rtol=1e-12)
 
 
+def test_prescribed_slot_assignment_only_changes_who_gets_which_slot():
+    """`assign` replaces S^{-1} and nothing else: the state is unchanged, the identity assignment
+    of the function's own ranks reproduces the default, and swapping two workers' slots swaps
+    exactly their smoothed coefficients."""
+    a = np.array([0.3, -1.0, 0.7, 0.1])
+    m0 = np.array([0.5, 0.6, 0.7, 0.8])
+    m, at, pi = oc.subspace_momentum(a, m0, 0.9)
+    ranks = np.empty(4, dtype=int); ranks[pi] = np.arange(4)
+    m2, at2, _ = oc.subspace_momentum(a, m0, 0.9, assign=ranks)
+    np.testing.assert_array_equal(m2, m); np.testing.assert_array_equal(at2, at)
+    swapped = ranks.copy(); swapped[[0, 3]] = swapped[[3, 0]]
+    m3, at3, _ = oc.subspace_momentum(a, m0, 0.9, assign=swapped)
+    np.testing.assert_array_equal(m3, m)
+    assert at3[0] == at[3] and at3[3] == at[0] and at3[1] == at[1] and at3[2] == at[2]
+
+
 # ---- variants (Table 2) ------------------------------------------------------------------
 def test_unnormalised_variant_matches_eq8():
     G = rand_G(5, 17, seed=17, noise=1.0)
