@@ -77,9 +77,15 @@ enum adacons_option {
                                   Section 4).  Changing it synchronises the device, allocates
                                   the per-segment plan and state, and resets the state.
                                   Errors: EALIGN (see above), ENOMEM.                            */
-  ADACONS_OPT_PROFILE = 5      /* 0 (default) / 1: record CUDA events around each of the three
+  ADACONS_OPT_PROFILE = 5,     /* 0 (default) / 1: record CUDA events around each of the three
                                   kernels of every aggregate call (see adacons_get_profile).
                                   Setting it (to either value) clears the recorded samples.      */
+  ADACONS_OPT_OVERLAP_LAUNCH = 6 /* 0 (default): plain stream order between the three kernels;
+                                  1: the coefficient step and pass 2 are launched with
+                                  programmatic stream serialisation (their blocks may become
+                                  resident while the kernel before them still runs).  Measured
+                                  slower on B200 for every workload tried, hence off; no effect
+                                  on results.                                                    */
 };
 
 /* Which N-vector adacons_get_coeffs returns (values of the most recent aggregate call). */

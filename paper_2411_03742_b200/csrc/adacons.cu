@@ -49,7 +49,7 @@ struct adacons_ctx {
 
   // options
   double beta = 0.99;
-  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0;
+  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0, overlap_launch = 0;
 
   // plans
   Pass1Plan fast;
@@ -458,7 +458,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   cudaEvent_t* ev = (c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
   if (ev) cudaEventRecord(ev[0], st);
 
-  const bool pdl = (ev == nullptr);   // event records between the kernels would defeat the overlap anyway
+  const bool pdl = (ev == nullptr) && c->overlap_launch;   // event records between the kernels would defeat the overlap
   const bool seg = c->per_segment != 0;
   if (seg && !(aligned && c->fast.available && c->seg_kernel != nullptr)) return ADACONS_EALIGN;
 
@@ -610,6 +610,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
         return ADACONS_ECUDA;
       return ADACONS_OK;
     }
+    case ADACONS_OPT_OVERLAP_LAUNCH: c->overlap_launch = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_PROFILE: {
       DeviceGuard guard(c->device);
       if (!guard.ok) return ADACONS_ECUDA;
@@ -636,6 +637,7 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_NORMALIZE: *value = c->normalize; return ADACONS_OK;
     case ADACONS_OPT_PER_SEGMENT: *value = c->per_segment; return ADACONS_OK;
     case ADACONS_OPT_PROFILE: *value = c->profile; return ADACONS_OK;
+    case ADACONS_OPT_OVERLAP_LAUNCH: *value = c->overlap_launch; return ADACONS_OK;
     default: return ADACONS_EINVAL;
   }
 }
