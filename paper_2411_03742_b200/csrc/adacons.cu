@@ -299,15 +299,16 @@ int build_seg_plan(adacons_ctx* c) {
   }
   int R = 0;
   for (int sgm = 0; sgm < S; ++sgm) { rec_begin[sgm] = R; R += rec_count[sgm]; }
-  // pass 2: block bid covers vectors num_vec-1-(bid*256+255) .. num_vec-1-bid*256 (clipped at 0)
+  // pass 2: block bid covers vectors [num_vec - (bid+1)*span, num_vec - bid*span), clipped at 0
   const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
   const long long num_vec = c->d / vec;
-  const long long blocks2 = (num_vec + kThreads - 1) / kThreads;
+  const long long span = static_cast<long long>(kThreads) * kPass2Groups;
+  const long long blocks2 = (num_vec + span - 1) / span;
   std::vector<int> blk(static_cast<size_t>(blocks2));
   for (long long bid = 0; bid < blocks2; ++bid) {
-    long long vlo = num_vec - 1 - (bid * kThreads + kThreads - 1);
+    long long vlo = num_vec - (bid + 1) * span;
     if (vlo < 0) vlo = 0;
-    const long long vhi = num_vec - 1 - bid * kThreads;
+    const long long vhi = num_vec - 1 - bid * span;
     const int slo = seg_of(vlo * vec), shi = seg_of(vhi * vec + vec - 1);
     blk[static_cast<size_t>(bid)] = slo == shi ? slo : -(slo + 1);
   }
@@ -523,7 +524,8 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   cudaError_t e2;
   if (aligned) {
     const long long num_vec = c->d * c->elem_bytes / 16;
-    const unsigned blocks = static_cast<unsigned>((num_vec + kThreads - 1) / kThreads);
+    const long long span = static_cast<long long>(kThreads) * kPass2Groups;
+    const unsigned blocks = static_cast<unsigned>((num_vec + span - 1) / span);
     const long long row_bytes = c->d * c->elem_bytes;
     const unsigned char* g8 = static_cast<const unsigned char*>(grads);
     unsigned char* o8 = static_cast<unsigned char*>(out);

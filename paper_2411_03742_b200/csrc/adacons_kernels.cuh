@@ -707,74 +707,109 @@ __device__ __forceinline__ void pass2_store(unsigned char* out, long long v, con
   *reinterpret_cast<uint4*>(out + v * 16) = o;
 }
 
-template <int DT, bool SEG>
+constexpr int kPass2Groups = 1;   // 16-byte column groups per thread (a block reads CG * 4 KB per row)
+constexpr int kPass2Rows = 8;     // rows per batch: kPass2Rows * kPass2Groups loads in flight per thread
+
+template <int DT, bool SEG, int CG = kPass2Groups, int U = kPass2Rows>
 __global__ void __launch_bounds__(kThreads)
 pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
                  const float* __restrict__ gamma, int N, long long row_bytes, long long num_vec,
                  const int* __restrict__ blk_seg, const long long* __restrict__ seg_off) {
   constexpr int VEC = Elem<DT>::kVec;
   constexpr int NP = VEC / 2;
-  constexpr int U = 8;                               // row loads in flight per thread
   __shared__ float g_s[kMaxN];
   pdl_wait();                                        // the coefficient step has finished
   int code = 0;
   if (SEG) code = blk_seg[blockIdx.x];
-  const long long v = num_vec - 1 - (static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x);
+  // block b owns vectors [num_vec - (b+1)*256*CG, num_vec - b*256*CG); thread t the CG vectors
+  // base + t + g*256 (those below zero do not exist)
+  const long long base = num_vec - (static_cast<long long>(blockIdx.x) + 1) * (kThreads * CG) + threadIdx.x;
   if (!SEG || code >= 0) {
     const float* gsrc = gamma + static_cast<size_t>(SEG ? code : 0) * N;
     for (int i = threadIdx.x; i < N; i += kThreads) g_s[i] = gsrc[i];
     __syncthreads();
-    if (v < 0) return;
-    const unsigned char* col = grads + v * 16;
-    float2 acc[NP];
+    float2 acc[CG][NP];
 #pragma unroll
-    for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
-    int i0 = 0;
-    for (; i0 + U <= N; i0 += U) {
-      uint4 x[U];
+    for (int g = 0; g < CG; ++g)
 #pragma unroll
-      for (int u = 0; u < U; ++u) x[u] = ld_stream_v4(col + static_cast<long long>(i0 + u) * row_bytes);
+      for (int h = 0; h < NP; ++h) acc[g][h] = make_float2(0.f, 0.f);
+    if (base >= 0) {                                 // all CG vectors exist (every block but the last)
+      const unsigned char* col = grads + base * 16;
+      int i0 = 0;
+      for (; i0 + U <= N; i0 += U) {
+        uint4 x[U][CG];
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const float g = g_s[i0 + u];
-        const float2 g2 = make_float2(g, g);
+        for (int u = 0; u < U; ++u)
 #pragma unroll
-        for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(x[u], h), g2, acc[h]);
+          for (int g = 0; g < CG; ++g)
+            x[u][g] = ld_stream_v4(col + static_cast<long long>(i0 + u) * row_bytes + g * (kThreads * 16));
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const float gm = g_s[i0 + u];
+          const float2 g2 = make_float2(gm, gm);
+#pragma unroll
+          for (int g = 0; g < CG; ++g)
+#pragma unroll
+            for (int h = 0; h < NP; ++h) acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[u][g], h), g2, acc[g][h]);
+        }
+      }
+      for (; i0 < N; ++i0) {
+        const float gm = g_s[i0];
+        const float2 g2 = make_float2(gm, gm);
+#pragma unroll
+        for (int g = 0; g < CG; ++g) {
+          const uint4 x = ld_stream_v4(col + static_cast<long long>(i0) * row_bytes + g * (kThreads * 16));
+#pragma unroll
+          for (int h = 0; h < NP; ++h) acc[g][h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, acc[g][h]);
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < CG; ++g) pass2_store<DT, NP>(out, base + g * kThreads, acc[g]);
+    } else {
+      for (int g = 0; g < CG; ++g) {
+        const long long v = base + g * kThreads;
+        if (v < 0) continue;
+        float2 a1[NP];
+#pragma unroll
+        for (int h = 0; h < NP; ++h) a1[h] = make_float2(0.f, 0.f);
+        for (int i = 0; i < N; ++i) {
+          const uint4 x = ld_stream_v4(grads + v * 16 + static_cast<long long>(i) * row_bytes);
+          const float2 g2 = make_float2(g_s[i], g_s[i]);
+#pragma unroll
+          for (int h = 0; h < NP; ++h) a1[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, a1[h]);
+        }
+        pass2_store<DT, NP>(out, v, a1);
       }
     }
-    for (; i0 < N; ++i0) {
-      const uint4 x = ld_stream_v4(col + static_cast<long long>(i0) * row_bytes);
-      const float g = g_s[i0];
-      const float2 g2 = make_float2(g, g);
-#pragma unroll
-      for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, acc[h]);
-    }
-    pass2_store<DT, NP>(out, v, acc);
   } else {
-    if (v < 0) return;
-    int sg = -code - 1;
-    int seg_of[VEC];
+    int sg0 = -code - 1;
+    for (int g = 0; g < CG; ++g) {
+      const long long v = base + g * kThreads;
+      if (v < 0) continue;
+      int sg = sg0;
+      int seg_of[VEC];
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) {
-      const long long c = v * VEC + e;
-      while (c >= seg_off[sg + 1]) ++sg;             // segments are ascending; empty ones are skipped
-      seg_of[e] = sg;
-    }
-    const unsigned char* col = grads + v * 16;
-    float2 acc[NP];
-#pragma unroll
-    for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
-    for (int i = 0; i < N; ++i) {
-      const uint4 x = ld_stream_v4(col + static_cast<long long>(i) * row_bytes);
-#pragma unroll
-      for (int h = 0; h < NP; ++h) {
-        const float2 xv = unpack_pair<DT>(x, h);
-        const float2 g2 = make_float2(gamma[static_cast<size_t>(seg_of[2 * h]) * N + i],
-                                      gamma[static_cast<size_t>(seg_of[2 * h + 1]) * N + i]);
-        acc[h] = __ffma2_rn(xv, g2, acc[h]);
+      for (int e = 0; e < VEC; ++e) {
+        const long long c = v * VEC + e;
+        while (c >= seg_off[sg + 1]) ++sg;           // segments are ascending; empty ones are skipped
+        seg_of[e] = sg;
       }
+      const unsigned char* col = grads + v * 16;
+      float2 acc[NP];
+#pragma unroll
+      for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+      for (int i = 0; i < N; ++i) {
+        const uint4 x = ld_stream_v4(col + static_cast<long long>(i) * row_bytes);
+#pragma unroll
+        for (int h = 0; h < NP; ++h) {
+          const float2 xv = unpack_pair<DT>(x, h);
+          const float2 g2 = make_float2(gamma[static_cast<size_t>(seg_of[2 * h]) * N + i],
+                                        gamma[static_cast<size_t>(seg_of[2 * h + 1]) * N + i]);
+          acc[h] = __ffma2_rn(xv, g2, acc[h]);
+        }
+      }
+      pass2_store<DT, NP>(out, v, acc);
     }
-    pass2_store<DT, NP>(out, v, acc);
   }
 }
 

@@ -465,3 +465,54 @@ def test_headline_config_full_size_sampled(ac):
         assert abs(q[i] - qi[0]) <= COEFF_RTOL * qi[0]
         pi = float((G[i].double() * s).sum()) / w.N
         assert abs(p[i] - pi) <= COEFF_RTOL * abs(pi)
+
+
+def test_config5_full_size_per_segment_sampled(ac):
+    """N=32, d=340M, fp32, 390 ragged segments (43.5 GB), layer-wise coefficients, as the benchmark
+    launches it.  Checked: sum(gamma_s) = 1 for every segment; the output on sampled columns (first,
+    last, random, and both sides of sampled segment boundaries) against the oracle's combine() with
+    the weights of the column's own segment; for sampled (segment, worker) pairs q with the oracle
+    and p against float64 torch sums; and the per-segment identity sum_i N p_si = ||sum_j g_j||^2."""
+    w = wl.WORKLOADS["ragged32"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60e9:
+        pytest.skip("needs 60 GB of free device memory")
+    dev = torch.device("cuda:0")
+    off = wl.segment_offsets(w)
+    S = len(off) - 1
+    G = wl.generate(w, 0, dev)
+    out = torch.empty(w.d, dtype=torch.float32, device=dev)
+    h = ac.AdaCons(w.N, w.d, "f32", seg_offsets=off)
+    h.set_option(ac.OPT_PER_SEGMENT, 1)
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    assert h.status() == 0
+    gamma, p, q = h.coeffs(ac.COEFF_GAMMA), h.coeffs(ac.COEFF_P), h.coeffs(ac.COEFF_Q)
+    assert gamma.shape == (S, w.N)
+    np.testing.assert_allclose(gamma.sum(axis=1), np.ones(S), atol=1e-12)
+
+    gcpu = torch.Generator().manual_seed(2)
+    bnd = torch.tensor([o for o in off[1:-1:13]])
+    cols = torch.cat([torch.arange(0, 32), torch.arange(w.d - 32, w.d), torch.randint(0, w.d, (4096,), generator=gcpu),
+                      bnd - 1, bnd, bnd + 1]).clamp_(0, w.d - 1)
+    seg = np.searchsorted(np.asarray(off), cols.numpy(), side="right") - 1
+    Gs = to_f64(G[:, cols.to(dev)])
+    got = to_f64(out[cols.to(dev)])
+    for k in range(cols.numel()):
+        g = gamma[seg[k]]
+        psi = float(oc.combine(Gs[:, k:k + 1], g)[0])
+        tight = 1e-5 * float(np.abs(g) @ np.abs(Gs[:, k])) + ULP["f32"] * abs(psi) + 1e-45
+        assert abs(got[k] - psi) <= tight, (k, int(cols[k]), int(seg[k]))
+
+    for s in (0, 57, 200, S - 1):
+        lo, hi = off[s], off[s + 1]
+        ssum = torch.zeros(hi - lo, dtype=torch.float64, device=dev)
+        for i in range(w.N):
+            ssum += G[i, lo:hi].double()
+        ss = float((ssum * ssum).sum())
+        assert abs(w.N * p[s].sum() - ss) <= 1e-5 * ss
+        for i in (0, 31):
+            _, qi = oc.consensus_statistics(to_f64(G[i:i + 1, lo:hi]))
+            assert abs(q[s, i] - qi[0]) <= COEFF_RTOL * qi[0]
+            pi = float((G[i, lo:hi].double() * ssum).sum()) / w.N
+            assert abs(p[s, i] - pi) <= COEFF_RTOL * abs(pi)
