@@ -80,12 +80,17 @@ enum adacons_option {
   ADACONS_OPT_PROFILE = 5,     /* 0 (default) / 1: record CUDA events around each of the three
                                   kernels of every aggregate call (see adacons_get_profile).
                                   Setting it (to either value) clears the recorded samples.      */
-  ADACONS_OPT_OVERLAP_LAUNCH = 6 /* 0 (default): plain stream order between the three kernels;
+  ADACONS_OPT_OVERLAP_LAUNCH = 6, /* 0 (default): plain stream order between the three kernels;
                                   1: the coefficient step and pass 2 are launched with
                                   programmatic stream serialisation (their blocks may become
                                   resident while the kernel before them still runs).  Measured
                                   slower on B200 for every workload tried, hence off; no effect
                                   on results.                                                    */
+  ADACONS_OPT_PASS2_TMA = 7    /* 0 (default): pass 2 reads the matrix with direct 16-byte global
+                                  loads; 1: on the fast path it stages its tiles through shared
+                                  memory by TMA like pass 1 (measured equal for bf16 N=64, slower
+                                  for fp32 N=32).  Results may differ in the last bit (the rows
+                                  are added in a different, equally fixed, order).               */
 };
 
 /* Which N-vector adacons_get_coeffs returns (values of the most recent aggregate call). */

@@ -391,6 +391,12 @@ def test_ablation_variants(ac, momentum, sorted_, normalize):
              oracle_kw=dict(momentum=bool(momentum), sort=bool(sorted_), normalize=bool(normalize)))
 
 
+@pytest.mark.parametrize("N,dtype", [(64, "bf16"), (32, "f32"), (16, "bf16"), (8, "f32"), (3, "bf16"), (1, "f32")])
+def test_pass2_tma_option(ac, N, dtype):
+    w = wl.Workload(f"p2tma{N}", N, 700_008, dtype, 2, "gauss", seed=70 + N)
+    run_case(ac, w, 2, beta=0.5, options={ac.OPT_PASS2_TMA: 1})
+
+
 def test_argument_errors(ac):
     lib = ac.load_library()
     ctx = ctypes.c_void_p()
