@@ -36,7 +36,7 @@ CPU_BASELINE_COLUMNS = 4_000_000       # cpu_baseline leg of the CUDA arm: 3 ste
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/, as a multiple of the algorithmic bytes of that kernel (None = no capture for the
 # current kernel).
-NCU_TRAFFIC_RATIO = {"pass1": None, "pass2": None}
+NCU_TRAFFIC_RATIO = {"pass1": 1.0018, "pass2": 0.9884}
 
 
 def parse_args(argv=None):
@@ -103,12 +103,15 @@ class ClockSampler(threading.Thread):
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop_evt = threading.Event()
         self.ok = False
+        self.uuid = None
         try:
             import pynvml
             pynvml.nvmlInit()
             self.nv = pynvml
             self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            u = pynvml.nvmlDeviceGetUUID(self.h)
+            self.uuid = u.decode() if isinstance(u, bytes) else str(u)
             self.ok = True
         except Exception:
             self.nv = None
@@ -146,7 +149,7 @@ class ClockSampler(threading.Thread):
             self.join(timeout=2)
         s = sorted(self.samples)
         return {"sm_mhz": (s[len(s) // 2] if s else None), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(s)}
+                "reasons": sorted(self.reasons), "samples": len(s), "gpu_uuid": self.uuid}
 
 
 def physical_gpu_index(local_index: int) -> int:
