@@ -86,11 +86,15 @@ enum adacons_option {
                                   resident while the kernel before them still runs).  Measured
                                   slower on B200 for every workload tried, hence off; no effect
                                   on results.                                                    */
-  ADACONS_OPT_PASS2_TMA = 7    /* 0 (default): pass 2 reads the matrix with direct 16-byte global
+  ADACONS_OPT_PASS2_TMA = 7,   /* 0 (default): pass 2 reads the matrix with direct 16-byte global
                                   loads; 1: on the fast path it stages its tiles through shared
                                   memory by TMA like pass 1 (measured equal for bf16 N=64, slower
                                   for fp32 N=32).  Results may differ in the last bit (the rows
                                   are added in a different, equally fixed, order).               */
+  ADACONS_OPT_FUSED_SMALL = 8  /* 1 (default): when the whole matrix fits in the shared memory of
+                                  the grid (about 148 x 160 KB) and the buffers are 16-byte
+                                  aligned, one cooperative kernel reads it from HBM once and does
+                                  all three steps; 0: always the three-kernel path.              */
 };
 
 /* Which N-vector adacons_get_coeffs returns (values of the most recent aggregate call). */
@@ -108,8 +112,9 @@ enum adacons_info {
   ADACONS_INFO_COEFF_SETS = 1,       /* 1 in model-wise mode, S in layer-wise mode               */
   ADACONS_INFO_PASS1_BLOCKS = 2,     /* thread blocks of the pass-1 kernel (= partial-sum rows)  */
   ADACONS_INFO_SCRATCH_BYTES = 3,    /* device bytes owned by the context                        */
-  ADACONS_INFO_LAUNCHES_PER_CALL = 4,/* kernels launched by one adacons_aggregate                */
-  ADACONS_INFO_LAST_PATH = 5,        /* 0 = none yet, 1 = TMA-staged fast path, 2 = generic path */
+  ADACONS_INFO_LAUNCHES_PER_CALL = 4,/* kernels launched by the most recent adacons_aggregate    */
+  ADACONS_INFO_LAST_PATH = 5,        /* 0 = none yet, 1 = TMA-staged fast path, 2 = generic path,
+                                        3 = single-pass kernel (matrix held in shared memory)   */
   ADACONS_INFO_TOTAL_LAUNCHES = 6    /* kernels launched by this context so far                  */
 };
 

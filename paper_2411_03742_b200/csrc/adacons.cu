@@ -51,7 +51,7 @@ struct adacons_ctx {
 
   // options
   double beta = 0.99;
-  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0, overlap_launch = 0, pass2_tma = 0;
+  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0, overlap_launch = 0, pass2_tma = 0, fused_small = 1;
 
   // plans
   Pass1Plan fast;
@@ -69,6 +69,12 @@ struct adacons_ctx {
   long long* step = nullptr;
   void* staging = nullptr;        // adacons_aggregate_host: N*d + d elements
   size_t scratch_bytes = 0;
+
+  // single-pass path for problems that fit in the grid's shared memory
+  bool fused_available = false;
+  int fused_grid = 0, fused_vpb = 0;
+  size_t fused_smem = 0;
+  unsigned long long* d_barrier = nullptr;
 
   // per-segment ("layer-wise") plan, built when ADACONS_OPT_PER_SEGMENT is switched on
   int seg_grid = 0;               // blocks of pass1_seg_kernel
@@ -226,6 +232,37 @@ int plan_fast(adacons_ctx* c) {
   f.grid2 = per_sm * c->num_sms;
   if (f.grid2 > f.num_tiles) f.grid2 = f.num_tiles;
   f.available = true;
+  return ADACONS_OK;
+}
+
+int plan_fused(adacons_ctx* c) {
+  c->fused_available = false;
+  int coop = 0;
+  if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) != cudaSuccess || !coop) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  if ((c->d * c->elem_bytes) % 16 != 0) return ADACONS_OK;
+  const long long num_vec = c->d * c->elem_bytes / 16;
+  long long grid = (num_vec + 63) / 64;
+  if (grid > c->num_sms) grid = c->num_sms;
+  if (grid < 1) grid = 1;
+  const long long vpb = (num_vec + grid - 1) / grid;
+  const size_t smem = static_cast<size_t>(c->N) * vpb * 16 + static_cast<size_t>(kFusedThreads / 32) * c->N * 2 * sizeof(float);
+  if (smem > 160 * 1024) return ADACONS_OK;
+  const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&fused_small_kernel<0>)
+                                          : reinterpret_cast<const void*>(&fused_small_kernel<1>);
+  int per_sm = 0;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kFusedThreads, smem) != cudaSuccess) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  if (per_sm < 1) return ADACONS_OK;
+  c->fused_grid = static_cast<int>(grid);
+  c->fused_vpb = static_cast<int>(vpb);
+  c->fused_smem = smem;
+  c->fused_available = true;
   return ADACONS_OK;
 }
 
@@ -444,11 +481,15 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   if (c->generic_grid > c->generic_tiles) c->generic_grid = c->generic_tiles;
   c->max_partials = c->generic_grid;
   if (c->fast.available && c->fast.grid > c->max_partials) c->max_partials = c->fast.grid;
+  plan_fused(c);
+  if (c->fused_available && c->fused_grid > c->max_partials) c->max_partials = c->fused_grid;
 
-  if (cudaMalloc(&c->flags, sizeof(uint32_t)) != cudaSuccess || cudaMalloc(&c->step, sizeof(long long)) != cudaSuccess) {
+  if (cudaMalloc(&c->flags, sizeof(uint32_t)) != cudaSuccess || cudaMalloc(&c->step, sizeof(long long)) != cudaSuccess ||
+      cudaMalloc(&c->d_barrier, sizeof(unsigned long long)) != cudaSuccess) {
     cudaGetLastError(); adacons_destroy(c); return ADACONS_ENOMEM;
   }
-  if (cudaMemset(c->flags, 0, sizeof(uint32_t)) != cudaSuccess || cudaMemset(c->step, 0, sizeof(long long)) != cudaSuccess) {
+  if (cudaMemset(c->flags, 0, sizeof(uint32_t)) != cudaSuccess || cudaMemset(c->step, 0, sizeof(long long)) != cudaSuccess ||
+      cudaMemset(c->d_barrier, 0, sizeof(unsigned long long)) != cudaSuccess) {
     adacons_destroy(c); return ADACONS_ECUDA;
   }
   const size_t b_part = static_cast<size_t>(c->max_partials) * 2 * N * sizeof(float);
@@ -465,7 +506,7 @@ int adacons_destroy(adacons_ctx* c) {
   if (c == nullptr) return ADACONS_OK;
   DeviceGuard g(c->device);
   cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
-  cudaFree(c->flags); cudaFree(c->step); cudaFree(c->staging);
+  cudaFree(c->flags); cudaFree(c->step); cudaFree(c->staging); cudaFree(c->d_barrier);
   free_seg_plan(c);
   if (c->prof_ready)
     for (int s = 0; s < adacons_ctx::kProfSlots; ++s)
@@ -493,6 +534,30 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   const bool pdl = (ev == nullptr) && c->overlap_launch;   // event records between the kernels would defeat the overlap
   const bool seg = c->per_segment != 0;
   if (seg && !(aligned && c->fast.available && c->seg_kernel != nullptr)) return ADACONS_EALIGN;
+
+  // ---- single-pass path: the whole matrix fits in the grid's shared memory ----
+  if (!seg && aligned && c->fused_available && c->fused_small) {
+    FusedParams f;
+    f.N = N; f.num_vec = c->d * c->elem_bytes / 16; f.row_bytes = c->d * c->elem_bytes; f.vec_per_block = c->fused_vpb;
+    f.grads = static_cast<const unsigned char*>(grads); f.out = static_cast<unsigned char*>(out);
+    f.barrier = c->d_barrier;
+    CoeffParams& q = f.coeff;
+    q.N = N; q.num_partials = c->fused_grid; q.sets = 1; q.beta = c->beta;
+    q.momentum = c->momentum; q.sorted = c->sorted; q.normalize = c->normalize;
+    q.partials = c->partials; q.rec_begin = nullptr; q.rec_count = nullptr;
+    q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.flags = c->flags; q.step = c->step;
+    const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&fused_small_kernel<0>)
+                                            : reinterpret_cast<const void*>(&fused_small_kernel<1>);
+    void* args[1] = {&f};
+    if (cudaLaunchCooperativeKernel(k, dim3(c->fused_grid), dim3(kFusedThreads), args, c->fused_smem, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); cudaEventRecord(ev[3], st); c->prof_calls += 1; }
+    c->last_path = 3;
+    c->total_launches += 1;
+    return ADACONS_OK;
+  }
 
   // ---- pass 1 (Eq. 7) ----
   if (seg) {
@@ -622,7 +687,7 @@ int adacons_reset(adacons_ctx* c, void* cuda_stream) {
   if (!guard.ok) return ADACONS_ECUDA;
   const long long n = static_cast<long long>(c->sets()) * c->N;
   reset_kernel<<<static_cast<unsigned>((n + 255) / 256 < 1024 ? (n + 255) / 256 : 1024), 256, 0,
-                 static_cast<cudaStream_t>(cuda_stream)>>>(c->m, n, c->flags, c->step);
+                 static_cast<cudaStream_t>(cuda_stream)>>>(c->m, n, c->flags, c->step, c->d_barrier);
   if (!launch_ok()) return ADACONS_ECUDA;
   c->total_launches += 1;
   return ADACONS_OK;
@@ -658,6 +723,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
     }
     case ADACONS_OPT_OVERLAP_LAUNCH: c->overlap_launch = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_PASS2_TMA: c->pass2_tma = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_FUSED_SMALL: c->fused_small = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_PROFILE: {
       DeviceGuard guard(c->device);
       if (!guard.ok) return ADACONS_ECUDA;
@@ -686,6 +752,7 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_PROFILE: *value = c->profile; return ADACONS_OK;
     case ADACONS_OPT_OVERLAP_LAUNCH: *value = c->overlap_launch; return ADACONS_OK;
     case ADACONS_OPT_PASS2_TMA: *value = c->pass2_tma; return ADACONS_OK;
+    case ADACONS_OPT_FUSED_SMALL: *value = c->fused_small; return ADACONS_OK;
     default: return ADACONS_EINVAL;
   }
 }
@@ -764,7 +831,7 @@ int adacons_get_info(adacons_ctx* c, int key, int64_t* value) {
     case ADACONS_INFO_COEFF_SETS: *value = c->sets(); return ADACONS_OK;
     case ADACONS_INFO_PASS1_BLOCKS: *value = c->fast.available ? c->fast.grid : c->generic_grid; return ADACONS_OK;
     case ADACONS_INFO_SCRATCH_BYTES: *value = static_cast<int64_t>(c->scratch_bytes); return ADACONS_OK;
-    case ADACONS_INFO_LAUNCHES_PER_CALL: *value = 3; return ADACONS_OK;
+    case ADACONS_INFO_LAUNCHES_PER_CALL: *value = c->last_path == 3 ? 1 : 3; return ADACONS_OK;
     case ADACONS_INFO_LAST_PATH: *value = c->last_path; return ADACONS_OK;
     case ADACONS_INFO_TOTAL_LAUNCHES: *value = c->total_launches; return ADACONS_OK;
     default: return ADACONS_EINVAL;

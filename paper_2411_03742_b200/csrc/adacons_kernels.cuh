@@ -578,20 +578,17 @@ struct CoeffParams {
   long long* step;       // aggregation counter
 };
 
-__global__ void __launch_bounds__(kMaxN)
-coeff_kernel(const CoeffParams prm) {
+__device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set) {
   __shared__ double sh_part[2 * kMaxN];
   __shared__ double sh_a[kMaxN];
   __shared__ double sh_u[kMaxN];
   __shared__ int sh_bad, sh_zero;
   __shared__ double sh_Z;
   __shared__ int sh_uniform;
-  const int N = prm.N, i = threadIdx.x, set = blockIdx.x, T = blockDim.x;
+  const int N = prm.N, i = threadIdx.x, T = blockDim.x;
   const int V = 2 * N;
   const size_t per = static_cast<size_t>(prm.sets) * N;   // stride between coefficient kinds
   if (i == 0) { sh_bad = 0; sh_zero = 0; }
-  pdl_launch_dependents();
-  pdl_wait();                                              // pass 1 has finished and is visible
   const int begin = prm.rec_begin ? prm.rec_begin[set] : 0;
   const int count = prm.rec_count ? prm.rec_count[set] : prm.num_partials;
   const float* base = prm.partials + static_cast<size_t>(begin) * V;
@@ -601,14 +598,14 @@ coeff_kernel(const CoeffParams prm) {
     if (g < groups) {
       double acc = 0.0;
 #pragma unroll 4
-      for (int c = g; c < count; c += groups) acc += static_cast<double>(base[static_cast<size_t>(c) * V + v]);
+      for (int c = g; c < count; c += groups) acc += static_cast<double>(__ldcg(base + static_cast<size_t>(c) * V + v));
       sh_part[g * V + v] = acc;
     }
   } else {
     for (int v = i; v < V; v += T) {
       double acc = 0.0;
 #pragma unroll 4
-      for (int c = 0; c < count; ++c) acc += static_cast<double>(base[static_cast<size_t>(c) * V + v]);
+      for (int c = 0; c < count; ++c) acc += static_cast<double>(__ldcg(base + static_cast<size_t>(c) * V + v));
       sh_part[v] = acc;
     }
   }
@@ -684,6 +681,13 @@ coeff_kernel(const CoeffParams prm) {
     prm.coef[2 * per + set * N + i] = g;
     prm.gamma_f32[set * N + i] = static_cast<float>(g);
   }
+}
+
+__global__ void __launch_bounds__(kMaxN)
+coeff_kernel(const CoeffParams prm) {
+  pdl_launch_dependents();
+  pdl_wait();                                              // pass 1 has finished and is visible
+  coeff_body(prm, blockIdx.x);
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -934,11 +938,144 @@ pass2_generic_kernel(const void* __restrict__ grads, void* __restrict__ out, con
   else reinterpret_cast<unsigned short*>(out)[k] = static_cast<unsigned short>(pack_bf16x2_rn(acc, 0.f) & 0xffffu);
 }
 
-__global__ void reset_kernel(double* m, long long n, uint32_t* flags, long long* step) {
+// ----------------------------------------------------------------------------------------------
+// Single-pass path for problems that fit in the grid's shared memory (N*d*sizeof(element) up to
+// about 148 x 160 KB): ONE cooperative kernel reads the matrix from HBM once.  Block b keeps all N
+// rows of its column slice in shared memory, computes its partial statistics (Eq. 7), meets the
+// other blocks at a grid barrier, block 0 runs the coefficient step (Eq. 11, Eq. 12-13), a second
+// grid barrier, and every block forms its slice of sum_i gamma_i g_i (Eq. 12) from shared memory.
+// The barriers are counters in global memory; the launch is cooperative, so all blocks are
+// resident, and every wait is bounded (2 s), after which the block raises the time-out flag and
+// leaves.
+// ----------------------------------------------------------------------------------------------
+constexpr int kFusedThreads = 1024;
+
+struct FusedParams {
+  int N;
+  long long num_vec;            // 16-byte column groups per row
+  long long row_bytes;
+  int vec_per_block;            // column groups owned by one block (shared-memory row pitch)
+  const unsigned char* grads;
+  unsigned char* out;
+  unsigned long long* barrier;  // monotonically increasing arrival counter
+  CoeffParams coeff;            // partials [gridDim.x][2N], sets = 1
+};
+
+__device__ __forceinline__ bool grid_barrier_bounded(unsigned long long* counter, unsigned int G, uint32_t* flags) {
+  __shared__ int s_ok;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned long long old = atomicAdd(counter, 1ull);
+    const unsigned long long target = (old / G + 1ull) * G;
+    const unsigned long long t0 = global_timer_ns();
+    int ok = 1;
+    for (;;) {
+      unsigned long long cur;
+      asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(cur) : "l"(counter) : "memory");
+      if (cur >= target) break;
+      if (global_timer_ns() - t0 > kWaitLimitNs) { ok = 0; atomicOr(flags, kFlagTimeout); break; }
+    }
+    __threadfence();
+    s_ok = ok;
+  }
+  __syncthreads();
+  return s_ok != 0;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+fused_small_kernel(const FusedParams prm) {
+  constexpr int VEC = Elem<DT>::kVec;
+  constexpr int NP = VEC / 2;
+  constexpr int kW = kFusedThreads / 32;
+  extern __shared__ __align__(16) unsigned char fs_raw[];
+  const int N = prm.N, vpb = prm.vec_per_block;
+  uint4* tile = reinterpret_cast<uint4*>(fs_raw);                                   // [N][vpb]
+  float* acc = reinterpret_cast<float*>(fs_raw + static_cast<size_t>(N) * vpb * 16); // [kW][N][2]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long vb0 = static_cast<long long>(blockIdx.x) * vpb;
+  long long rem = prm.num_vec - vb0;
+  const int nv = rem <= 0 ? 0 : (rem < vpb ? static_cast<int>(rem) : vpb);
+
+  // ---- the only read of the matrix from HBM
+  for (int idx = tid; idx < N * nv; idx += kFusedThreads) {
+    const int row = idx / nv, v = idx - row * nv;
+    tile[row * vpb + v] = ld_stream_v4(prm.grads + static_cast<long long>(row) * prm.row_bytes + (vb0 + v) * 16);
+  }
+  for (int i = tid; i < kW * N * 2; i += kFusedThreads) acc[i] = 0.f;
+  __syncthreads();
+
+  // ---- statistics of the slice: a warp takes 32 column groups at a time
+  float* mine = acc + static_cast<size_t>(warp) * N * 2;
+  for (int v0 = warp * 32; v0 < nv; v0 += kFusedThreads) {
+    const int v = v0 + lane;
+    const bool valid = v < nv;
+    float2 sp[NP];
+#pragma unroll
+    for (int h = 0; h < NP; ++h) sp[h] = make_float2(0.f, 0.f);
+    if (valid)
+      for (int i = 0; i < N; ++i) {
+        const uint4 x = tile[i * vpb + v];
+#pragma unroll
+        for (int h = 0; h < NP; ++h) sp[h] = __fadd2_rn(sp[h], unpack_pair<DT>(x, h));
+      }
+    for (int i = 0; i < N; ++i) {
+      float2 pa = make_float2(0.f, 0.f), qa = make_float2(0.f, 0.f);
+      if (valid) {
+        const uint4 x = tile[i * vpb + v];
+#pragma unroll
+        for (int h = 0; h < NP; ++h) {
+          const float2 xv = unpack_pair<DT>(x, h);
+          pa = __ffma2_rn(xv, sp[h], pa);
+          qa = __ffma2_rn(xv, xv, qa);
+        }
+      }
+      float p = pa.x + pa.y, q = qa.x + qa.y;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        p += __shfl_xor_sync(0xffffffffu, p, o);
+        q += __shfl_xor_sync(0xffffffffu, q, o);
+      }
+      if (lane == 0) { mine[2 * i] += p; mine[2 * i + 1] += q; }
+    }
+  }
+  __syncthreads();
+  float* part = const_cast<float*>(prm.coeff.partials) + static_cast<size_t>(blockIdx.x) * 2 * N;
+  for (int i = tid; i < N; i += kFusedThreads) {
+    float p = 0.f, q = 0.f;
+    for (int w = 0; w < kW; ++w) { p += acc[(static_cast<size_t>(w) * N + i) * 2]; q += acc[(static_cast<size_t>(w) * N + i) * 2 + 1]; }
+    part[i] = p;
+    part[N + i] = q;
+  }
+  if (!grid_barrier_bounded(prm.barrier, gridDim.x, prm.coeff.flags)) return;
+
+  if (blockIdx.x == 0) coeff_body(prm.coeff, 0);
+  if (!grid_barrier_bounded(prm.barrier, gridDim.x, prm.coeff.flags)) return;
+
+  // ---- weighted combination of the slice, from shared memory
+  float* g_s = acc;                                   // reuse: N floats
+  for (int i = tid; i < N; i += kFusedThreads) g_s[i] = __ldcg(prm.coeff.gamma_f32 + i);
+  __syncthreads();
+  for (int v = tid; v < nv; v += kFusedThreads) {
+    float2 o[NP];
+#pragma unroll
+    for (int h = 0; h < NP; ++h) o[h] = make_float2(0.f, 0.f);
+    for (int i = 0; i < N; ++i) {
+      const uint4 x = tile[i * vpb + v];
+      const float2 g2 = make_float2(g_s[i], g_s[i]);
+#pragma unroll
+      for (int h = 0; h < NP; ++h) o[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, o[h]);
+    }
+    pass2_store<DT, NP>(prm.out, vb0 + v, o);
+  }
+}
+
+__global__ void reset_kernel(double* m, long long n, uint32_t* flags, long long* step, unsigned long long* barrier) {
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
        i += static_cast<long long>(gridDim.x) * blockDim.x)
     m[i] = 0.0;
-  if (blockIdx.x == 0 && threadIdx.x == 0) { *flags = 0u; *step = 0; }
+  if (blockIdx.x == 0 && threadIdx.x == 0) { *flags = 0u; *step = 0; *barrier = 0ull; }
 }
 
 }  // namespace adacons

@@ -102,10 +102,14 @@ def oracle_step_with_kernel_ranks(orc, G64, dtype, a_gpu, sort=True, momentum=Tr
     return orc.step(G64, storage=dtype, assign=r_gpu)
 
 
-def run_case(ac, w, steps, *, beta=0.99, options=None, oracle_kw=None, offsets=None, per_segment=False):
+def run_case(ac, w, steps, *, beta=0.99, options=None, oracle_kw=None, offsets=None, per_segment=False,
+             fused=False, expect_path=None):
+    """fused=False keeps small cases on the three-kernel path (the one the large workloads take);
+    fused=True lets the library pick the single-pass kernel when the matrix fits in shared memory."""
     dev = torch.device("cuda:0")
     oracle_kw = dict(oracle_kw or {})
     h = ac.AdaCons(w.N, w.d, w.dtype, seg_offsets=offsets)
+    h.set_option(ac.OPT_FUSED_SMALL, 1 if fused else 0)
     if per_segment:
         h.set_option(ac.OPT_PER_SEGMENT, 1)
         oracle_kw.update(seg_offsets=offsets, per_segment=True)
@@ -134,14 +138,17 @@ def run_case(ac, w, steps, *, beta=0.99, options=None, oracle_kw=None, offsets=N
         assert_output(out, res, G64, w.dtype, f"{w.name} step {t}", offsets)
         expected_flags |= int(np.bitwise_or.reduce(res["flags"]))
         assert h.status() == expected_flags
+        if expect_path is not None:
+            assert h.info(ac.INFO_LAST_PATH) == expect_path
     h.close()
     return h
 
 
 # ---- the five benchmark configurations, scaled so that the oracle finishes in seconds but the
 # ---- kernels still see several tiles per block and a ragged last tile -------------------------
-def test_config1_full_size(ac):
-    run_case(ac, wl.WORKLOADS["small4"], 1)
+@pytest.mark.parametrize("fused", [False, True])
+def test_config1_full_size(ac, fused):
+    run_case(ac, wl.WORKLOADS["small4"], 1, fused=fused, expect_path=3 if fused else 1)
 
 
 @pytest.mark.parametrize("name,d,steps", [
@@ -165,19 +172,62 @@ def test_config2_full_size_three_steps(ac):
 @pytest.mark.parametrize("N", [1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64])
 def test_all_worker_counts_fast_path(ac, N, dtype):
     w = wl.Workload(f"n{N}", N, 20_008, dtype, 2, "gauss", seed=50 + N)
-    h = run_case(ac, w, 2, beta=0.7)
-    del h
+    run_case(ac, w, 2, beta=0.7, expect_path=1)
 
 
-def test_fast_path_is_taken_when_aligned(ac):
+# ---- single-pass kernel (matrix resident in shared memory) --------------------------------------
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N", [1, 2, 3, 5, 8, 16, 33, 64, 100])
+def test_single_pass_kernel_all_worker_counts(ac, N, dtype):
+    w = wl.Workload(f"f{N}", N, 20_008, dtype, 3, "gauss", seed=150 + N)
+    run_case(ac, w, 3, beta=0.7, fused=True, expect_path=3)
+
+
+@pytest.mark.parametrize("N,d,dtype", [(4, 4, "f32"), (3, 8, "bf16"), (2, 64 * 4, "f32"), (16, 700_000, "bf16"),
+                                       (8, 640_000, "f32")])
+def test_single_pass_kernel_sizes(ac, N, d, dtype):
+    """One 16-byte vector, exactly one block's worth, and close to the shared-memory capacity."""
+    w = wl.Workload(f"fs{N}x{d}", N, d, dtype, 2, "gauss", seed=9)
+    run_case(ac, w, 2, beta=0.5, fused=True, expect_path=3)
+
+
+def test_single_pass_kernel_is_not_used_when_the_matrix_does_not_fit(ac):
+    w = wl.Workload("big", 64, 400_008, "bf16", 1, "gauss", seed=1)     # 51 MB > grid shared memory
+    run_case(ac, w, 1, fused=True, expect_path=1)
+
+
+def test_single_pass_and_three_kernel_paths_share_state(ac):
+    """Switching between the two paths mid-run continues the same momentum state."""
+    w = wl.Workload("mix", 12, 50_000, "f32", 4, "gauss", seed=33)
+    dev = "cuda:0"
+    h = ac.AdaCons(w.N, w.d, "f32")
+    orc = oc.AdaConsOracle(w.N, w.d)
+    out = torch.empty(w.d, device=dev)
+    for t in range(4):
+        h.set_option(ac.OPT_FUSED_SMALL, t % 2)
+        G = wl.generate(w, t, dev)
+        h.aggregate(G, out)
+        torch.cuda.synchronize()
+        assert h.info(ac.INFO_LAST_PATH) == (3 if t % 2 else 1)
+        res = oracle_step_with_kernel_ranks(orc, to_f64(G), "f32", h.coeffs(ac.COEFF_A))
+        assert_coeffs(h.coeffs(), res["gamma"], f"gamma step {t}")
+        assert_coeffs(h.state()[0], res["m"], f"m step {t}")
+
+
+def test_path_selection_and_launch_counts(ac):
     w = wl.Workload("probe", 8, 8192, "f32", 1, "gauss")
     h = ac.AdaCons(w.N, w.d, w.dtype)
     G = wl.generate(w, 0, "cuda:0")
     out = torch.empty(w.d, device="cuda:0")
     h.aggregate(G, out)
     torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 3                      # fits in shared memory: one kernel
+    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 1 and h.info(ac.INFO_TOTAL_LAUNCHES) == 1
+    h.set_option(ac.OPT_FUSED_SMALL, 0)
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
     assert h.info(ac.INFO_LAST_PATH) == 1
-    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 3 and h.info(ac.INFO_TOTAL_LAUNCHES) == 3
+    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 3 and h.info(ac.INFO_TOTAL_LAUNCHES) == 4
 
 
 # ---- generic path: odd lengths, misaligned pointers, many workers ------------------------------
@@ -228,6 +278,7 @@ def test_generic_and_fast_paths_agree(ac):
     G1.copy_(G0)
     o0, o1 = torch.empty(d, device="cuda:0", dtype=torch.bfloat16), torch.empty(d, device="cuda:0", dtype=torch.bfloat16)
     h0, h1 = ac.AdaCons(N, d, "bf16"), ac.AdaCons(N, d, "bf16")
+    h0.set_option(ac.OPT_FUSED_SMALL, 0)
     h0.aggregate(G0, o0); h1.aggregate(G1, o1)
     torch.cuda.synchronize()
     assert (h0.info(ac.INFO_LAST_PATH), h1.info(ac.INFO_LAST_PATH)) == (1, 2)
@@ -284,9 +335,20 @@ def test_per_segment_needs_the_aligned_path(ac):
 
 
 # ---- degenerate inputs --------------------------------------------------------------------------
+FUSED_MODE = [0]          # set by the fixture below: the degenerate-input tests run on both paths
+
+
+@pytest.fixture(params=[0, 1], ids=["three-kernel", "single-pass"])
+def both_paths(request):
+    FUSED_MODE[0] = request.param
+    yield request.param
+    FUSED_MODE[0] = 0
+
+
 def _agg(ac, G, dtype="f32", **opt):
     N, d = G.shape
     h = ac.AdaCons(N, d, dtype)
+    h.set_option(ac.OPT_FUSED_SMALL, FUSED_MODE[0])
     for k, v in opt.items():
         h.set_option(k, v)
     out = torch.empty(d, device=G.device, dtype=G.dtype)
@@ -295,7 +357,7 @@ def _agg(ac, G, dtype="f32", **opt):
     return h, out
 
 
-def test_identical_gradients_and_single_worker(ac):
+def test_identical_gradients_and_single_worker(ac, both_paths):
     g = torch.randn(5000, device="cuda:0")
     h, out = _agg(ac, g.repeat(7, 1).contiguous())
     np.testing.assert_allclose(to_f64(out), to_f64(g), rtol=3e-6, atol=1e-7)
@@ -304,7 +366,7 @@ def test_identical_gradients_and_single_worker(ac):
     assert torch.equal(out, g)
 
 
-def test_zero_row_all_zero_nonfinite_and_negative_normaliser(ac):
+def test_zero_row_all_zero_nonfinite_and_negative_normaliser(ac, both_paths):
     G = torch.randn(4, 4096, device="cuda:0") + torch.randn(4096, device="cuda:0")
     G[2] = 0
     h, out = _agg(ac, G)
@@ -320,6 +382,7 @@ def test_zero_row_all_zero_nonfinite_and_negative_normaliser(ac):
 
     G = torch.randn(3, 2048, device="cuda:0") + torch.randn(2048, device="cuda:0")
     h = ac.AdaCons(3, 2048, "f32")
+    h.set_option(ac.OPT_FUSED_SMALL, FUSED_MODE[0])
     out = torch.empty(2048, device="cuda:0")
     h.aggregate(G, out)
     m_before, _ = h.state()
@@ -339,9 +402,9 @@ def test_zero_row_all_zero_nonfinite_and_negative_normaliser(ac):
 
 
 # ---- determinism, state, options ----------------------------------------------------------------
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_bit_stability(ac, dtype):
-    w = wl.Workload("bits", 24, 700_008, dtype, 3, "gauss", seed=21)
+@pytest.mark.parametrize("dtype,d", [("f32", 700_008), ("bf16", 700_008), ("f32", 100_000)])
+def test_bit_stability(ac, dtype, d):
+    w = wl.Workload("bits", 24, d, dtype, 3, "gauss", seed=21)           # d = 100k: single-pass kernel
     dev = "cuda:0"
     Gs = [wl.generate(w, t, dev) for t in range(3)]
     runs = []
