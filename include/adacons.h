@@ -91,10 +91,17 @@ enum adacons_option {
                                   memory by TMA like pass 1 (measured equal for bf16 N=64, slower
                                   for fp32 N=32).  Results may differ in the last bit (the rows
                                   are added in a different, equally fixed, order).               */
-  ADACONS_OPT_FUSED_SMALL = 8  /* 1 (default): when the whole matrix fits in the shared memory of
+  ADACONS_OPT_FUSED_SMALL = 8, /* 1 (default): when the whole matrix fits in the shared memory of
                                   the grid (about 148 x 160 KB) and the buffers are 16-byte
                                   aligned, one cooperative kernel reads it from HBM once and does
                                   all three steps; 0: always the three-kernel path.              */
+  ADACONS_OPT_ROW_PITCH = 9    /* elements between the starts of two consecutive rows of the
+                                  gradient matrix, >= d; default d (contiguous rows).  Applies to
+                                  adacons_aggregate and adacons_aggregate_host.  A gradient length
+                                  that is not a multiple of 16 bytes runs on the fast path when the
+                                  rows are padded to a pitch that is; the padding is never read
+                                  as data and nothing is written past out[d-1].  Setting it
+                                  synchronises the device and may re-allocate scratch.           */
 };
 
 /* Which N-vector adacons_get_coeffs returns (values of the most recent aggregate call). */
@@ -138,9 +145,10 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
 /*
  * Aggregate one set of gradients (Eq. 12; Algorithm 1 on a single device).
  *   grads  device pointer, read-only: N rows of d elements, row-major and contiguous
- *          (row i = g_i starts at element i*d).
+ *          (row i = g_i starts at element i*pitch; pitch = d unless ADACONS_OPT_ROW_PITCH is set).
  *   out    device pointer, d elements of the same type; must not overlap grads.
- *   Fast path: grads and out 16-byte aligned and d*sizeof(element) a multiple of 16, N <= 64.
+ *   Fast path: grads and out 16-byte aligned, the row pitch in bytes (d*sizeof(element) unless
+ *   ADACONS_OPT_ROW_PITCH says otherwise) a multiple of 16, N <= 64.
  *   Anything else is served by a slower generic path with the same results.
  * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
  * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.

@@ -44,6 +44,7 @@ struct adacons_ctx {
   long long d = 0;
   int dtype = 0;
   int elem_bytes = 4;
+  long long pitch = 0;                  // elements between the starts of two rows (>= d)
   int device = 0;
   int num_sms = 0;
   std::vector<long long> seg_offsets;   // S + 1 entries
@@ -67,7 +68,8 @@ struct adacons_ctx {
   double* m = nullptr;            // [sets][N]
   uint32_t* flags = nullptr;
   long long* step = nullptr;
-  void* staging = nullptr;        // adacons_aggregate_host: N*d + d elements
+  void* staging = nullptr;        // adacons_aggregate_host: N*pitch + d elements
+  size_t staging_bytes = 0;
   size_t scratch_bytes = 0;
 
   // single-pass path for problems that fit in the grid's shared memory
@@ -185,7 +187,7 @@ int plan_fast(adacons_ctx* c) {
   f.available = false;
   const int N = c->N;
   if (N > kMaxFastN) return ADACONS_OK;
-  if ((c->d * c->elem_bytes) % 16 != 0) return ADACONS_OK;
+  if ((c->pitch * c->elem_bytes) % 16 != 0) return ADACONS_OK;
   if (c->d > 2147483647ll - 8192) return ADACONS_OK;
   if (c->encode == nullptr) return ADACONS_OK;
   int WR, NR;
@@ -242,8 +244,8 @@ int plan_fused(adacons_ctx* c) {
     cudaGetLastError();
     return ADACONS_OK;
   }
-  if ((c->d * c->elem_bytes) % 16 != 0) return ADACONS_OK;
-  const long long num_vec = c->d * c->elem_bytes / 16;
+  if ((c->pitch * c->elem_bytes) % 16 != 0) return ADACONS_OK;
+  const long long num_vec = (c->d * c->elem_bytes + 15) / 16;
   long long grid = (num_vec + 63) / 64;
   if (grid > c->num_sms) grid = c->num_sms;
   if (grid < 1) grid = 1;
@@ -269,7 +271,7 @@ int plan_fused(adacons_ctx* c) {
 int encode_map(adacons_ctx* c, const void* grads) {
   if (c->tmap_for == grads) return ADACONS_OK;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->d) * c->elem_bytes};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(c->N)};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = c->encode(&c->tmap,
@@ -369,7 +371,7 @@ int build_seg_plan(adacons_ctx* c) {
   for (int sgm = 0; sgm < S; ++sgm) { rec_begin[sgm] = R; R += rec_count[sgm]; }
   // pass 2: block bid covers vectors [num_vec - (bid+1)*span, num_vec - bid*span), clipped at 0
   const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
-  const long long num_vec = c->d / vec;
+  const long long num_vec = (c->d + vec - 1) / vec;
   const long long span = static_cast<long long>(kThreads) * kPass2Groups;
   const long long blocks2 = (num_vec + span - 1) / span;
   std::vector<int> blk(static_cast<size_t>(blocks2));
@@ -377,7 +379,8 @@ int build_seg_plan(adacons_ctx* c) {
     long long vlo = num_vec - (bid + 1) * span;
     if (vlo < 0) vlo = 0;
     const long long vhi = num_vec - 1 - bid * span;
-    const int slo = seg_of(vlo * vec), shi = seg_of(vhi * vec + vec - 1);
+    const long long chi = vhi * vec + vec - 1 < c->d - 1 ? vhi * vec + vec - 1 : c->d - 1;
+    const int slo = seg_of(vlo * vec), shi = seg_of(chi);
     blk[static_cast<size_t>(bid)] = slo == shi ? slo : -(slo + 1);
   }
   size_t bytes = 0;
@@ -448,7 +451,7 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
 
   adacons_ctx* c = new (std::nothrow) adacons_ctx();
   if (c == nullptr) return ADACONS_ENOMEM;
-  c->N = N; c->d = d; c->dtype = dtype; c->elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
+  c->N = N; c->d = d; c->pitch = d; c->dtype = dtype; c->elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
   c->device = dev; c->num_sms = sms;
   if (num_segments > 0) {
     c->num_segments = num_segments;
@@ -518,14 +521,17 @@ int adacons_destroy(adacons_ctx* c) {
 
 int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_stream) {
   if (c == nullptr || grads == nullptr || out == nullptr) return ADACONS_EINVAL;
-  const size_t gbytes = static_cast<size_t>(c->N) * c->d * c->elem_bytes;
+  const size_t gbytes = (static_cast<size_t>(c->N - 1) * c->pitch + c->d) * c->elem_bytes;
   const size_t obytes = static_cast<size_t>(c->d) * c->elem_bytes;
   const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads), o0 = reinterpret_cast<uintptr_t>(out);
   if (o0 < g0 + gbytes && g0 < o0 + obytes) return ADACONS_EINVAL;   // out overlaps grads
   DeviceGuard guard(c->device);
   if (!guard.ok) return ADACONS_ECUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const bool aligned = (g0 % 16 == 0) && (o0 % 16 == 0) && ((c->d * c->elem_bytes) % 16 == 0);
+  const bool aligned = (g0 % 16 == 0) && (o0 % 16 == 0) && ((c->pitch * c->elem_bytes) % 16 == 0);
+  const long long num_vec = (c->d * c->elem_bytes + 15) / 16;              // 16-byte column groups per row
+  const int tail_elems = static_cast<int>((c->d * c->elem_bytes % 16) / c->elem_bytes);   // 0: the last group is full
+  const long long row_bytes = c->pitch * c->elem_bytes;
   const int N = c->N;
   int num_partials;
   cudaEvent_t* ev = (c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
@@ -538,7 +544,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   // ---- single-pass path: the whole matrix fits in the grid's shared memory ----
   if (!seg && aligned && c->fused_available && c->fused_small) {
     FusedParams f;
-    f.N = N; f.num_vec = c->d * c->elem_bytes / 16; f.row_bytes = c->d * c->elem_bytes; f.vec_per_block = c->fused_vpb;
+    f.N = N; f.num_vec = num_vec; f.tail_elems = tail_elems; f.row_bytes = row_bytes; f.vec_per_block = c->fused_vpb;
     f.grads = static_cast<const unsigned char*>(grads); f.out = static_cast<unsigned char*>(out);
     f.barrier = c->d_barrier;
     CoeffParams& q = f.coeff;
@@ -590,9 +596,9 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     c->last_path = 1;
   } else {
     if (c->dtype == ADACONS_F32)
-      pass1_generic_kernel<0><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->generic_tiles, c->partials);
+      pass1_generic_kernel<0><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->pitch, c->generic_tiles, c->partials);
     else
-      pass1_generic_kernel<1><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->generic_tiles, c->partials);
+      pass1_generic_kernel<1><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->pitch, c->generic_tiles, c->partials);
     if (!launch_ok()) return ADACONS_ECUDA;
     num_partials = c->generic_grid;
     c->last_path = 2;
@@ -621,7 +627,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   if (aligned && c->fast.available && !seg && c->pass2_tma) {
     Pass2Params p2;
     p2.N = N; p2.num_tiles = c->fast.num_tiles; p2.stages = c->fast.stages; p2.stage_bytes = c->fast.stage_bytes;
-    p2.num_vec = c->d * c->elem_bytes / 16; p2.gamma = c->gamma_f32; p2.out = static_cast<unsigned char*>(out);
+    p2.num_vec = num_vec; p2.tail_elems = tail_elems; p2.gamma = c->gamma_f32; p2.out = static_cast<unsigned char*>(out);
     p2.flags = c->flags;
     void* args[2] = {&c->tmap, &p2};
     cudaLaunchConfig_t cfg = {};
@@ -632,26 +638,24 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
     e2 = cudaLaunchKernelExC(&cfg, c->fast.kernel2, args);
   } else if (aligned) {
-    const long long num_vec = c->d * c->elem_bytes / 16;
     const long long span = static_cast<long long>(kThreads) * kPass2Groups;
     const unsigned blocks = static_cast<unsigned>((num_vec + span - 1) / span);
-    const long long row_bytes = c->d * c->elem_bytes;
     const unsigned char* g8 = static_cast<const unsigned char*>(grads);
     unsigned char* o8 = static_cast<unsigned char*>(out);
     const int* bs = c->d_pass2_blk_seg;
     const long long* so = c->d_seg_off;
     if (c->dtype == ADACONS_F32)
-      e2 = seg ? launch_kernel(pass2_vec_kernel<0, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so)
-               : launch_kernel(pass2_vec_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so);
+      e2 = seg ? launch_kernel(pass2_vec_kernel<0, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
+               : launch_kernel(pass2_vec_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
     else
-      e2 = seg ? launch_kernel(pass2_vec_kernel<1, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so)
-               : launch_kernel(pass2_vec_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so);
+      e2 = seg ? launch_kernel(pass2_vec_kernel<1, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
+               : launch_kernel(pass2_vec_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
   } else {
     const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);
     if (c->dtype == ADACONS_F32)
-      e2 = launch_kernel(pass2_generic_kernel<0>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d);
+      e2 = launch_kernel(pass2_generic_kernel<0>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d, c->pitch);
     else
-      e2 = launch_kernel(pass2_generic_kernel<1>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d);
+      e2 = launch_kernel(pass2_generic_kernel<1>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d, c->pitch);
   }
   if (e2 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
   if (ev) { cudaEventRecord(ev[3], st); c->prof_calls += 1; }
@@ -664,11 +668,17 @@ int adacons_aggregate_host(adacons_ctx* c, const void* host_grads, void* host_ou
   DeviceGuard guard(c->device);
   if (!guard.ok) return ADACONS_ECUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const size_t gbytes = static_cast<size_t>(c->N) * c->d * c->elem_bytes;
+  const size_t gbytes = (static_cast<size_t>(c->N - 1) * c->pitch + c->d) * c->elem_bytes;
   const size_t obytes = static_cast<size_t>(c->d) * c->elem_bytes;
-  const size_t gpad = (gbytes + 255) / 256 * 256;
+  const size_t gpad = (static_cast<size_t>(c->N) * c->pitch * c->elem_bytes + 255) / 256 * 256;
+  if (c->staging != nullptr && c->staging_bytes < gpad + obytes) {
+    cudaFree(c->staging);
+    c->staging = nullptr;
+    c->scratch_bytes -= c->staging_bytes;
+  }
   if (c->staging == nullptr) {
     if (cudaMalloc(&c->staging, gpad + obytes) != cudaSuccess) { cudaGetLastError(); return ADACONS_ENOMEM; }
+    c->staging_bytes = gpad + obytes;
     c->scratch_bytes += gpad + obytes;
   }
   unsigned char* dg = static_cast<unsigned char*>(c->staging);
@@ -724,6 +734,35 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
     case ADACONS_OPT_OVERLAP_LAUNCH: c->overlap_launch = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_PASS2_TMA: c->pass2_tma = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: c->fused_small = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_ROW_PITCH: {
+      const long long pitch = static_cast<long long>(value);
+      if (static_cast<double>(pitch) != value || pitch < c->d || pitch >= (1ll << 40)) return ADACONS_EINVAL;
+      if (pitch == c->pitch) return ADACONS_OK;
+      DeviceGuard guard(c->device);
+      if (!guard.ok) return ADACONS_ECUDA;
+      if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+      c->pitch = pitch;
+      c->tmap_for = nullptr;
+      int rc = plan_fast(c);
+      if (rc != ADACONS_OK) return rc;
+      plan_fused(c);
+      int need = c->generic_grid;
+      if (c->fast.available && c->fast.grid > need) need = c->fast.grid;
+      if (c->fused_available && c->fused_grid > need) need = c->fused_grid;
+      if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
+        cudaFree(c->partials);
+        c->partials = nullptr;
+        c->max_partials = need;
+        const size_t b_part = static_cast<size_t>(need) * 2 * c->N * sizeof(float);
+        if (cudaMalloc(&c->partials, b_part) != cudaSuccess) { cudaGetLastError(); return ADACONS_ENOMEM; }
+        if (cudaMemset(c->partials, 0, b_part) != cudaSuccess) return ADACONS_ECUDA;
+      }
+      if (c->per_segment) {
+        rc = build_seg_plan(c);
+        if (rc != ADACONS_OK) { free_seg_plan(c); c->per_segment = 0; alloc_sets(c); return rc; }
+      }
+      return ADACONS_OK;
+    }
     case ADACONS_OPT_PROFILE: {
       DeviceGuard guard(c->device);
       if (!guard.ok) return ADACONS_ECUDA;
@@ -753,6 +792,7 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_OVERLAP_LAUNCH: *value = c->overlap_launch; return ADACONS_OK;
     case ADACONS_OPT_PASS2_TMA: *value = c->pass2_tma; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: *value = c->fused_small; return ADACONS_OK;
+    case ADACONS_OPT_ROW_PITCH: *value = static_cast<double>(c->pitch); return ADACONS_OK;
     default: return ADACONS_EINVAL;
   }
 }
@@ -925,7 +965,7 @@ extern "C" int adacons_stats_noalloc(const void* grads, int N, int64_t d, int dt
 
   // A context object on the host stack only carries the launch plan; it owns no device memory.
   adacons_ctx plan;
-  plan.N = N; plan.d = d; plan.dtype = dtype; plan.elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
+  plan.N = N; plan.d = d; plan.pitch = d; plan.dtype = dtype; plan.elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
   plan.device = dev; plan.num_sms = nd->sms; plan.encode = nd->encode;
   rc = plan_fast(&plan);
   if (rc != ADACONS_OK) return rc;
@@ -954,8 +994,8 @@ extern "C" int adacons_stats_noalloc(const void* grads, int N, int64_t d, int dt
     if (blocks > tiles) blocks = tiles;
     if (blocks > ADACONS_NOALLOC_MAX_BLOCKS) blocks = ADACONS_NOALLOC_MAX_BLOCKS;
     const size_t smem = static_cast<size_t>(kWarps) * N * 2 * sizeof(float);   // <= 4 KB for N <= 64
-    if (dtype == ADACONS_F32) pass1_generic_kernel<0><<<blocks, kThreads, smem, st>>>(grads, N, d, tiles, partials);
-    else pass1_generic_kernel<1><<<blocks, kThreads, smem, st>>>(grads, N, d, tiles, partials);
+    if (dtype == ADACONS_F32) pass1_generic_kernel<0><<<blocks, kThreads, smem, st>>>(grads, N, d, d, tiles, partials);
+    else pass1_generic_kernel<1><<<blocks, kThreads, smem, st>>>(grads, N, d, d, tiles, partials);
     if (!launch_ok()) return ADACONS_ECUDA;
   }
   stats_finish_kernel<<<(2 * N + 127) / 128, 128, 0, st>>>(partials, blocks, N, flag, pq_out);

@@ -505,7 +505,8 @@ template <> __device__ __forceinline__ float load_elem<1>(const void* base, long
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
-pass1_generic_kernel(const void* __restrict__ grads, int N, long long d, int num_tiles, float* __restrict__ partials) {
+pass1_generic_kernel(const void* __restrict__ grads, int N, long long d, long long pitch, int num_tiles,
+                     float* __restrict__ partials) {
   constexpr int CPT = 4;
   extern __shared__ float acc[];                   // [kWarps][N][2]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -521,7 +522,7 @@ pass1_generic_kernel(const void* __restrict__ grads, int N, long long d, int num
 #pragma unroll
       for (int c = 0; c < CPT; ++c) {
         const long long col = c0 + c * kThreads;
-        if (col < d) s[c] += load_elem<DT>(grads, static_cast<long long>(i) * d + col);
+        if (col < d) s[c] += load_elem<DT>(grads, static_cast<long long>(i) * pitch + col);
       }
     for (int i = 0; i < N; ++i) {
       float p = 0.f, q = 0.f;
@@ -529,7 +530,7 @@ pass1_generic_kernel(const void* __restrict__ grads, int N, long long d, int num
       for (int c = 0; c < CPT; ++c) {
         const long long col = c0 + c * kThreads;
         if (col < d) {
-          const float x = load_elem<DT>(grads, static_cast<long long>(i) * d + col);
+          const float x = load_elem<DT>(grads, static_cast<long long>(i) * pitch + col);
           p = fmaf(x, s[c], p);
           q = fmaf(x, x, q);
         }
@@ -714,11 +715,31 @@ __device__ __forceinline__ void pass2_store(unsigned char* out, long long v, con
 constexpr int kPass2Groups = 1;   // 16-byte column groups per thread (a block reads CG * 4 KB per row)
 constexpr int kPass2Rows = 8;     // rows per batch: kPass2Rows * kPass2Groups loads in flight per thread
 
+// The last 16-byte group of a row holds only `tail_elems` real columns when d is not a multiple of
+// the vector width (rows padded to a 16-byte pitch): store those element by element.
+template <int DT, int NP>
+__device__ __forceinline__ void pass2_store_tail(unsigned char* out, long long v, const float2 (&acc)[NP], int tail_elems) {
+  constexpr int VEC = Elem<DT>::kVec;
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    if (e >= tail_elems) break;
+    const float x = (e & 1) ? acc[e / 2].y : acc[e / 2].x;
+    if constexpr (DT == 0) reinterpret_cast<float*>(out)[v * VEC + e] = x;
+    else reinterpret_cast<unsigned short*>(out)[v * VEC + e] = static_cast<unsigned short>(pack_bf16x2_rn(x, 0.f) & 0xffffu);
+  }
+}
+template <int DT, int NP>
+__device__ __forceinline__ void pass2_store_any(unsigned char* out, long long v, const float2 (&acc)[NP],
+                                                long long num_vec, int tail_elems) {
+  if (tail_elems != 0 && v == num_vec - 1) pass2_store_tail<DT, NP>(out, v, acc, tail_elems);
+  else pass2_store<DT, NP>(out, v, acc);
+}
+
 template <int DT, bool SEG, int CG = kPass2Groups, int U = kPass2Rows>
 __global__ void __launch_bounds__(kThreads)
 pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
                  const float* __restrict__ gamma, int N, long long row_bytes, long long num_vec,
-                 const int* __restrict__ blk_seg, const long long* __restrict__ seg_off) {
+                 const int* __restrict__ blk_seg, const long long* __restrict__ seg_off, int tail_elems) {
   constexpr int VEC = Elem<DT>::kVec;
   constexpr int NP = VEC / 2;
   __shared__ float g_s[kMaxN];
@@ -768,7 +789,7 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
         }
       }
 #pragma unroll
-      for (int g = 0; g < CG; ++g) pass2_store<DT, NP>(out, base + g * kThreads, acc[g]);
+      for (int g = 0; g < CG; ++g) pass2_store_any<DT, NP>(out, base + g * kThreads, acc[g], num_vec, tail_elems);
     } else {
       for (int g = 0; g < CG; ++g) {
         const long long v = base + g * kThreads;
@@ -782,7 +803,7 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
 #pragma unroll
           for (int h = 0; h < NP; ++h) a1[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, a1[h]);
         }
-        pass2_store<DT, NP>(out, v, a1);
+        pass2_store_any<DT, NP>(out, v, a1, num_vec, tail_elems);
       }
     }
   } else {
@@ -793,10 +814,13 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
       int sg = sg0;
       int seg_of[VEC];
 #pragma unroll
+      const long long d_cols = (num_vec - 1) * VEC + (tail_elems ? tail_elems : VEC);
+#pragma unroll
       for (int e = 0; e < VEC; ++e) {
         const long long c = v * VEC + e;
-        while (c >= seg_off[sg + 1]) ++sg;           // segments are ascending; empty ones are skipped
-        seg_of[e] = sg;
+        if (c < d_cols)
+          while (c >= seg_off[sg + 1]) ++sg;         // segments are ascending; empty ones are skipped
+        seg_of[e] = sg;                              // padding columns: any set, never stored
       }
       const unsigned char* col = grads + v * 16;
       float2 acc[NP];
@@ -812,7 +836,7 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
           acc[h] = __ffma2_rn(xv, g2, acc[h]);
         }
       }
-      pass2_store<DT, NP>(out, v, acc);
+      pass2_store_any<DT, NP>(out, v, acc, num_vec, tail_elems);
     }
   }
 }
@@ -829,7 +853,8 @@ struct Pass2Params {
   int num_tiles;
   int stages;
   uint32_t stage_bytes;
-  long long num_vec;     // d * sizeof(element) / 16
+  long long num_vec;     // ceil(d * sizeof(element) / 16)
+  int tail_elems;        // real columns in the last 16-byte group (0 = all)
   const float* gamma;    // [N]
   unsigned char* out;
   uint32_t* flags;
@@ -914,7 +939,7 @@ pass2_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass2Params prm
     if (rw == 0) {
       if (WR > 1) p1_xch_read<C>(xbuf, acc, cw, lane);
       const long long vec = (static_cast<long long>(tile_of(k)) * C::TILEC + cw * C::BOXC) / C::VEC + lane;
-      if (vec < prm.num_vec) pass2_store<DT, C::NP>(prm.out, vec, acc);
+      if (vec < prm.num_vec) pass2_store_any<DT, C::NP>(prm.out, vec, acc, prm.num_vec, prm.tail_elems);
     }
     if (++s == prm.stages) { s = 0; parity ^= 1u; }
   }
@@ -925,7 +950,7 @@ pass2_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass2Params prm
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 pass2_generic_kernel(const void* __restrict__ grads, void* __restrict__ out, const float* __restrict__ gamma,
-                     int N, long long d) {
+                     int N, long long d, long long pitch) {
   __shared__ float g_s[kMaxN];
   pdl_wait();
   for (int i = threadIdx.x; i < N; i += kThreads) g_s[i] = gamma[i];
@@ -933,7 +958,7 @@ pass2_generic_kernel(const void* __restrict__ grads, void* __restrict__ out, con
   const long long k = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
   if (k >= d) return;
   float acc = 0.f;
-  for (int i = 0; i < N; ++i) acc = fmaf(load_elem<DT>(grads, static_cast<long long>(i) * d + k), g_s[i], acc);
+  for (int i = 0; i < N; ++i) acc = fmaf(load_elem<DT>(grads, static_cast<long long>(i) * pitch + k), g_s[i], acc);
   if constexpr (DT == 0) reinterpret_cast<float*>(out)[k] = acc;
   else reinterpret_cast<unsigned short*>(out)[k] = static_cast<unsigned short>(pack_bf16x2_rn(acc, 0.f) & 0xffffu);
 }
@@ -952,7 +977,8 @@ constexpr int kFusedThreads = 1024;
 
 struct FusedParams {
   int N;
-  long long num_vec;            // 16-byte column groups per row
+  long long num_vec;            // 16-byte column groups per row (the last may be partial)
+  int tail_elems;               // real columns in the last group (0 = all)
   long long row_bytes;
   int vec_per_block;            // column groups owned by one block (shared-memory row pitch)
   const unsigned char* grads;
@@ -1001,7 +1027,19 @@ fused_small_kernel(const FusedParams prm) {
   // ---- the only read of the matrix from HBM
   for (int idx = tid; idx < N * nv; idx += kFusedThreads) {
     const int row = idx / nv, v = idx - row * nv;
-    tile[row * vpb + v] = ld_stream_v4(prm.grads + static_cast<long long>(row) * prm.row_bytes + (vb0 + v) * 16);
+    uint4 x = ld_stream_v4(prm.grads + static_cast<long long>(row) * prm.row_bytes + (vb0 + v) * 16);
+    if (prm.tail_elems != 0 && vb0 + v == prm.num_vec - 1) {     // row padding is not data: zero it
+      uint32_t wds[4] = {x.x, x.y, x.z, x.w};
+      constexpr int kPerWord = 4 / Elem<DT>::kBytes;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int first = k * kPerWord;
+        if (first >= prm.tail_elems) wds[k] = 0u;
+        else if (kPerWord == 2 && first + 1 >= prm.tail_elems) wds[k] &= 0x0000ffffu;
+      }
+      x = make_uint4(wds[0], wds[1], wds[2], wds[3]);
+    }
+    tile[row * vpb + v] = x;
   }
   for (int i = tid; i < kW * N * 2; i += kFusedThreads) acc[i] = 0.f;
   __syncthreads();
@@ -1067,7 +1105,7 @@ fused_small_kernel(const FusedParams prm) {
 #pragma unroll
       for (int h = 0; h < NP; ++h) o[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, o[h]);
     }
-    pass2_store<DT, NP>(prm.out, vb0 + v, o);
+    pass2_store_any<DT, NP>(prm.out, vb0 + v, o, prm.num_vec, prm.tail_elems);
   }
 }
 
