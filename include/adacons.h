@@ -241,6 +241,18 @@ int adacons_get_profile(adacons_ctx *ctx, double ms[3], int64_t *calls, void *cu
 int adacons_stats_noalloc(const void *grads, int N, int64_t d, int dtype, double *pq_out,
                           void *cuda_stream);
 
+/*
+ * Self-test of the hang protection (no paper counterpart).  Every wait inside the library's
+ * kernels -- on a TMA completion barrier, on the grid barrier of the single-pass kernel -- gives
+ * up after 2 s, raises ADACONS_FLAG_TIMEOUT and lets the kernel return.  This call launches a tiny
+ * kernel whose wait can never be satisfied (which = 0: an mbarrier nobody arrives on; which = 1: a
+ * grid barrier that expects one more block than was launched) so that the give-up path can be
+ * exercised without faulting or hanging the device: about 2 s later adacons_get_status reports
+ * ADACONS_FLAG_TIMEOUT.  Call adacons_reset afterwards (it clears the flag and the barrier
+ * counter that which = 1 leaves odd).  Errors: EINVAL, ECUDA.
+ */
+int adacons_selftest_bounded_wait(adacons_ctx *ctx, int which, void *cuda_stream);
+
 /* Facts about the context; see enum adacons_info.  No device work. */
 int adacons_get_info(adacons_ctx *ctx, int key, int64_t *value);
 

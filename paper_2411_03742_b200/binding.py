@@ -67,6 +67,7 @@ def load_library() -> ctypes.CDLL:
         "adacons_set_state": [vp, P(dbl), i64, vp],
         "adacons_get_status": [vp, P(ctypes.c_uint32), vp],
         "adacons_get_info": [vp, i32, P(i64)],
+        "adacons_selftest_bounded_wait": [vp, i32, vp],
         "adacons_get_profile": [vp, P(dbl), P(i64), vp],
         "adacons_stats_noalloc": [vp, i32, i64, i32, vp, vp],
         "adacons_version": [],
@@ -204,6 +205,10 @@ class AdaCons:
         n = ctypes.c_int64()
         _check(self._lib.adacons_get_profile(self._ctx, ms, ctypes.byref(n), _stream_handle(stream)), "adacons_get_profile")
         return [ms[0], ms[1], ms[2]], n.value
+
+    def selftest_bounded_wait(self, which: int, stream=None) -> None:
+        _check(self._lib.adacons_selftest_bounded_wait(self._ctx, int(which), _stream_handle(stream)),
+               "adacons_selftest_bounded_wait")
 
     def status(self, stream=None) -> int:
         v = ctypes.c_uint32()

@@ -864,6 +864,16 @@ int adacons_get_profile(adacons_ctx* c, double ms[3], int64_t* calls, void* cuda
   return ADACONS_OK;
 }
 
+int adacons_selftest_bounded_wait(adacons_ctx* c, int which, void* cuda_stream) {
+  if (c == nullptr || (which != 0 && which != 1)) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(which, c->d_barrier, c->flags);
+  if (!launch_ok()) return ADACONS_ECUDA;
+  c->total_launches += 1;
+  return ADACONS_OK;
+}
+
 int adacons_get_info(adacons_ctx* c, int key, int64_t* value) {
   if (c == nullptr || value == nullptr) return ADACONS_EINVAL;
   switch (key) {

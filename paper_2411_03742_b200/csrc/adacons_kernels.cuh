@@ -1109,6 +1109,23 @@ fused_small_kernel(const FusedParams prm) {
   }
 }
 
+// Self-test of the bounded waits (no data path): which = 0 waits on an mbarrier that nobody arrives
+// on, which = 1 on a grid barrier that expects one more block than exists.  Both give up after
+// kWaitLimitNs, raise the time-out flag and return; the context stays usable.
+__global__ void selftest_wait_kernel(int which, unsigned long long* barrier, uint32_t* flags) {
+  __shared__ __align__(8) uint64_t bar;
+  if (which == 0) {
+    if (threadIdx.x == 0) {
+      mbar_init(&bar, 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait_bounded(&bar, 0u)) atomicOr(flags, kFlagTimeout);
+  } else {
+    (void)grid_barrier_bounded(barrier, gridDim.x + 1u, flags);
+  }
+}
+
 __global__ void reset_kernel(double* m, long long n, uint32_t* flags, long long* step, unsigned long long* barrier) {
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
        i += static_cast<long long>(gridDim.x) * blockDim.x)
