@@ -4,8 +4,8 @@ The objective is the one of the paper's first experiment (Section 4.1, Eq. 14):
     min_w  E_{zeta ~ U[0,1]^d} [ (w^T zeta)^2 / 2 ],   d = 1000,
 each worker drawing its own mini-batch per step; the workers' gradients are stacked as an N x d
 matrix on the GPU and aggregated either by the plain mean or by AdaCons (`adacons_aggregate`).
-Both runs use the same step size and the same random batches.  The paper gives each method "the
-optimal analytical step size" without printing it and its figures are not available, so this
+Both runs use the same step size and the same random batches.  The paper tunes the step size
+analytically per method but prints neither the rule nor numbers (its curves are figures), so this
 driver only supports a qualitative comparison (final loss of the two aggregation rules).
 
     python -m paper_2411_03742_b200.examples.linear_regression --workers 32 --batch 16 --steps 200
