@@ -86,16 +86,11 @@ enum adacons_option {
                                   resident while the kernel before them still runs).  Measured
                                   slower on B200 for every workload tried, hence off; no effect
                                   on results.                                                    */
-  ADACONS_OPT_PASS2_TMA = 7,   /* 0 (default): pass 2 reads the matrix with direct 16-byte global
-                                  loads; 1: on the fast path it stages its tiles through shared
-                                  memory by TMA like pass 1 (measured equal for bf16 N=64, slower
-                                  for fp32 N=32).  Results may differ in the last bit (the rows
-                                  are added in a different, equally fixed, order).               */
-  ADACONS_OPT_FUSED_SMALL = 8, /* 1 (default): when the whole matrix fits in the shared memory of
+  ADACONS_OPT_FUSED_SMALL = 7, /* 1 (default): when the whole matrix fits in the shared memory of
                                   the grid (about 148 x 160 KB) and the buffers are 16-byte
                                   aligned, one cooperative kernel reads it from HBM once and does
                                   all three steps; 0: always the three-kernel path.              */
-  ADACONS_OPT_ROW_PITCH = 9    /* elements between the starts of two consecutive rows of the
+  ADACONS_OPT_ROW_PITCH = 8    /* elements between the starts of two consecutive rows of the
                                   gradient matrix, >= d; default d (contiguous rows).  Applies to
                                   adacons_aggregate and adacons_aggregate_host.  A gradient length
                                   that is not a multiple of 16 bytes runs on the fast path when the

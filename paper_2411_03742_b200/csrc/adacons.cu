@@ -33,8 +33,6 @@ struct Pass1Plan {            // TMA-staged pass 1 for this (N, dtype)
   size_t smem_bytes = 0;
   int grid = 0;
   const void* kernel = nullptr;
-  const void* kernel2 = nullptr;   // TMA-staged pass 2 with the same tiles and ring
-  int grid2 = 0;
 };
 
 }  // namespace
@@ -52,7 +50,7 @@ struct adacons_ctx {
 
   // options
   double beta = 0.99;
-  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0, overlap_launch = 0, pass2_tma = 0, fused_small = 1;
+  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0, overlap_launch = 0, fused_small = 1;
 
   // plans
   Pass1Plan fast;
@@ -149,25 +147,6 @@ const void* select_pass1_seg(int dtype, int NR, int WR) {
 #undef ADACONS_PICK
 }
 
-template <int DT, int NR, int WR>
-const void* pass2_tma_fn() { return reinterpret_cast<const void*>(&pass2_tma_kernel<DT, NR, WR>); }
-
-const void* select_pass2_tma(int dtype, int NR, int WR) {
-#define ADACONS_PICK(DT)                                     \
-  if (WR == 1) {                                             \
-    if (NR == 1) return pass2_tma_fn<DT, 1, 1>();            \
-    if (NR == 2) return pass2_tma_fn<DT, 2, 1>();            \
-    if (NR == 4) return pass2_tma_fn<DT, 4, 1>();            \
-    return pass2_tma_fn<DT, 8, 1>();                         \
-  }                                                          \
-  if (WR == 2) return pass2_tma_fn<DT, 8, 2>();              \
-  if (WR == 4) return pass2_tma_fn<DT, 8, 4>();              \
-  return pass2_tma_fn<DT, 8, 8>();
-  if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
-  ADACONS_PICK(1)
-#undef ADACONS_PICK
-}
-
 // Launch with (or without) the programmatic-stream-serialisation attribute.
 template <typename... KArgs, typename... Args>
 cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
@@ -223,16 +202,6 @@ int plan_fast(adacons_ctx* c) {
   }
   f.grid = per_sm * c->num_sms;
   if (f.grid > f.num_tiles) f.grid = f.num_tiles;
-  f.kernel2 = select_pass2_tma(c->dtype, NR, WR);
-  if (cudaFuncSetAttribute(f.kernel2, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(f.smem_bytes)) !=
-          cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, f.kernel2, kThreads, f.smem_bytes) != cudaSuccess ||
-      per_sm < 1) {
-    cudaGetLastError();
-    return ADACONS_ECUDA;
-  }
-  f.grid2 = per_sm * c->num_sms;
-  if (f.grid2 > f.num_tiles) f.grid2 = f.num_tiles;
   f.available = true;
   return ADACONS_OK;
 }
@@ -624,20 +593,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
 
   // ---- pass 2 (Eq. 12) ----
   cudaError_t e2;
-  if (aligned && c->fast.available && !seg && c->pass2_tma) {
-    Pass2Params p2;
-    p2.N = N; p2.num_tiles = c->fast.num_tiles; p2.stages = c->fast.stages; p2.stage_bytes = c->fast.stage_bytes;
-    p2.num_vec = num_vec; p2.tail_elems = tail_elems; p2.gamma = c->gamma_f32; p2.out = static_cast<unsigned char*>(out);
-    p2.flags = c->flags;
-    void* args[2] = {&c->tmap, &p2};
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(c->fast.grid2); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = c->fast.smem_bytes; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
-    e2 = cudaLaunchKernelExC(&cfg, c->fast.kernel2, args);
-  } else if (aligned) {
+  if (aligned) {
     const long long span = static_cast<long long>(kThreads) * kPass2Groups;
     const unsigned blocks = static_cast<unsigned>((num_vec + span - 1) / span);
     const unsigned char* g8 = static_cast<const unsigned char*>(grads);
@@ -732,7 +688,6 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       return ADACONS_OK;
     }
     case ADACONS_OPT_OVERLAP_LAUNCH: c->overlap_launch = value != 0.0; return ADACONS_OK;
-    case ADACONS_OPT_PASS2_TMA: c->pass2_tma = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: c->fused_small = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: {
       const long long pitch = static_cast<long long>(value);
@@ -790,7 +745,6 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_PER_SEGMENT: *value = c->per_segment; return ADACONS_OK;
     case ADACONS_OPT_PROFILE: *value = c->profile; return ADACONS_OK;
     case ADACONS_OPT_OVERLAP_LAUNCH: *value = c->overlap_launch; return ADACONS_OK;
-    case ADACONS_OPT_PASS2_TMA: *value = c->pass2_tma; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: *value = c->fused_small; return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: *value = static_cast<double>(c->pitch); return ADACONS_OK;
     default: return ADACONS_EINVAL;

@@ -841,111 +841,6 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
   }
 }
 
-// ----------------------------------------------------------------------------------------------
-// Pass 2, TMA-staged (model-wise weights, N <= 64, 16-byte aligned rows): the same tiles, ring and
-// warp grid as pass 1.  Warp (rw, cw) forms sum_j gamma_row(j) * x_row(j) over its NR rows of box
-// cw; with WR > 1 the WR partial sums are exchanged through shared memory and added in rw order by
-// the rw = 0 warp, which rounds and stores 512 contiguous bytes.  Tiles are visited from the END
-// of the vector: the columns pass 1 touched last are still in L2.
-// ----------------------------------------------------------------------------------------------
-struct Pass2Params {
-  int N;
-  int num_tiles;
-  int stages;
-  uint32_t stage_bytes;
-  long long num_vec;     // ceil(d * sizeof(element) / 16)
-  int tail_elems;        // real columns in the last 16-byte group (0 = all)
-  const float* gamma;    // [N]
-  unsigned char* out;
-  uint32_t* flags;
-};
-
-template <int DT, int NR, int WR>
-__global__ void __launch_bounds__(kThreads, 2)
-pass2_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass2Params prm) {
-  using C = P1<DT, NR, WR>;
-  extern __shared__ __align__(1024) unsigned char smem_raw[];
-  __shared__ int s_abort;
-  const int N = prm.N;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int cw = warp / WR, rw = warp % WR;
-  const P1Smem sm = p1_carve<C>(smem_raw, prm.stages, prm.stage_bytes);
-
-  if (tid == 0) {
-    s_abort = 0;
-    for (int s = 0; s < prm.stages; ++s) mbar_init(&sm.full[s], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    fence_proxy_async_smem();
-  }
-  __syncthreads();
-
-  const int first = blockIdx.x;
-  const int stride = gridDim.x;
-  const int my_tiles = first < prm.num_tiles ? (prm.num_tiles - first + stride - 1) / stride : 0;
-  auto tile_of = [&](int k) { return prm.num_tiles - 1 - (first + k * stride); };
-
-  auto issue = [&](int k, int s) {
-    const int col0 = tile_of(k) * C::TILEC;
-    mbar_expect_tx(&sm.full[s], prm.stage_bytes);
-#pragma unroll
-    for (int c = 0; c < C::WC; ++c)
-      tma_load_2d(sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes + static_cast<size_t>(c) * N * kBoxRowBytes,
-                  &tmap, &sm.full[s], col0 + c * C::BOXC, 0);
-  };
-  int issued = 0;
-  if (tid == 0) {                    // the matrix does not depend on the kernels before this one
-    const int pre = my_tiles < prm.stages ? my_tiles : prm.stages;
-    for (int k = 0; k < pre; ++k) issue(k, k);
-    issued = pre;
-  }
-  pdl_wait();                        // the weights do
-  float gw[NR];
-#pragma unroll
-  for (int j = 0; j < NR; ++j) {
-    const int row = rw + WR * j;
-    gw[j] = row < N ? prm.gamma[row] : 0.f;
-  }
-
-  int s = 0;
-  uint32_t parity = 0;
-  for (int k = 0; k < my_tiles; ++k) {
-    uint4 v[NR];
-    if (mbar_wait_bounded(&sm.full[s], parity)) {
-      p1_load_rows<C>(v, sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes +
-                             static_cast<size_t>(cw) * N * kBoxRowBytes + lane * 16, rw, N);
-    } else {
-#pragma unroll
-      for (int j = 0; j < NR; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
-      atomicOr(&s_abort, 1);
-    }
-    float2 acc[C::NP];
-#pragma unroll
-    for (int h = 0; h < C::NP; ++h) acc[h] = make_float2(0.f, 0.f);
-#pragma unroll
-    for (int j = 0; j < NR; ++j) {
-      const float2 g2 = make_float2(gw[j], gw[j]);
-#pragma unroll
-      for (int h = 0; h < C::NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(v[j], h), g2, acc[h]);
-    }
-    float* xbuf = sm.xch + (k & 1) * C::kXchOne;
-    if (WR > 1) p1_xch_write<C>(xbuf, acc, rw, cw, lane);
-    __syncthreads();
-    if (s_abort) break;
-    if (tid == 0 && k + prm.stages < my_tiles) {
-      fence_proxy_async_smem();
-      issue(k + prm.stages, s);
-      issued = k + prm.stages + 1;
-    }
-    if (rw == 0) {
-      if (WR > 1) p1_xch_read<C>(xbuf, acc, cw, lane);
-      const long long vec = (static_cast<long long>(tile_of(k)) * C::TILEC + cw * C::BOXC) / C::VEC + lane;
-      if (vec < prm.num_vec) pass2_store_any<DT, C::NP>(prm.out, vec, acc, prm.num_vec, prm.tail_elems);
-    }
-    if (++s == prm.stages) { s = 0; parity ^= 1u; }
-  }
-  if (s_abort && tid == 0) p1_drain_after_timeout(sm.full, prm.stages, issued, prm.flags);
-}
-
 // Pass 2, generic: one thread per column, scalar loads.
 template <int DT>
 __global__ void __launch_bounds__(kThreads)

@@ -454,12 +454,6 @@ def test_ablation_variants(ac, momentum, sorted_, normalize):
              oracle_kw=dict(momentum=bool(momentum), sort=bool(sorted_), normalize=bool(normalize)))
 
 
-@pytest.mark.parametrize("N,dtype", [(64, "bf16"), (32, "f32"), (16, "bf16"), (8, "f32"), (3, "bf16"), (1, "f32")])
-def test_pass2_tma_option(ac, N, dtype):
-    w = wl.Workload(f"p2tma{N}", N, 700_008, dtype, 2, "gauss", seed=70 + N)
-    run_case(ac, w, 2, beta=0.5, options={ac.OPT_PASS2_TMA: 1})
-
-
 def test_argument_errors(ac):
     lib = ac.load_library()
     ctx = ctypes.c_void_p()
@@ -648,3 +642,117 @@ def test_config3_full_size_streamed_oracle(ac):
     got = to_f64(out[cols])
     tight = 1e-5 * (np.abs(c["gamma"])[:, None] * np.abs(Gs)).sum(0) + ULP["bf16"] * np.abs(psi) + 1e-45
     assert np.all(np.abs(got - psi) <= tight)
+
+
+# ---- largest worker counts: the coefficient step's other reduction branch (2N > block size) -----
+@pytest.mark.parametrize("N", [512, 600, 1024])
+def test_many_workers(ac, N):
+    w = wl.Workload(f"many{N}", N, 3_000, "f32", 2, "gauss", seed=N)
+    run_case(ac, w, 2, beta=0.9, expect_path=2)
+
+
+# ---- the call neither allocates nor synchronises: it can be recorded once and replayed -----------
+def test_replay_from_a_cuda_graph_advances_the_state(ac):
+    w = wl.Workload("graph", 16, 600_000, "bf16", 3, "gauss", seed=123)
+    dev = torch.device("cuda:0")
+    G = wl.generate(w, 0, dev)
+    static_G = torch.empty_like(G)
+    out = torch.empty(w.d, dtype=torch.bfloat16, device=dev)
+    h = ac.AdaCons(w.N, w.d, "bf16")
+    h.set_option(ac.OPT_FUSED_SMALL, 0)
+    static_G.copy_(G)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        h.aggregate(static_G, out)                    # warm-up outside the capture (encodes the tensor map)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    h.reset()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        h.aggregate(static_G, out)
+    orc = oc.AdaConsOracle(w.N, w.d)
+    for t in range(3):
+        static_G.copy_(wl.generate(w, t, dev))
+        graph.replay()
+        torch.cuda.synchronize()
+        res = oracle_step_with_kernel_ranks(orc, to_f64(static_G), "bf16", h.coeffs(ac.COEFF_A))
+        assert_coeffs(h.coeffs(), res["gamma"], f"gamma replay {t}")
+        assert_coeffs(h.state()[0], res["m"], f"m replay {t}")
+        assert_output(out, res, to_f64(static_G), "bf16", f"replay {t}")
+    assert h.state()[1] == 3
+
+
+# ---- padded rows: any gradient length on the fast paths ------------------------------------------
+def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=None, per_segment=False, expect_path=None):
+    """Rows live in an N x pitch buffer whose padding is NaN; the result buffer is followed by a
+    sentinel.  Neither may influence, or be touched by, the aggregation."""
+    dev = torch.device("cuda:0")
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    w = wl.Workload(f"pad{N}x{d}", N, d, dtype, steps, "gauss", seed=d % 1000 + N)
+    buf = torch.full((N, pitch), float("nan"), dtype=tdt, device=dev)
+    obuf = torch.full((d + 32,), 7.0, dtype=tdt, device=dev)
+    out = obuf[:d]
+    h = ac.AdaCons(N, d, dtype, seg_offsets=offsets)
+    h.set_option(ac.OPT_ROW_PITCH, pitch)
+    h.set_option(ac.OPT_FUSED_SMALL, 1 if fused else 0)
+    oracle_kw = {}
+    if per_segment:
+        h.set_option(ac.OPT_PER_SEGMENT, 1)
+        oracle_kw = dict(seg_offsets=offsets, per_segment=True)
+    for k, v in (options or {}).items():
+        h.set_option(k, v)
+    h.set_option(ac.OPT_BETA, 0.8)
+    orc = oc.AdaConsOracle(N, d, beta=0.8, **oracle_kw)
+    for t in range(steps):
+        G = wl.generate(w, t, dev)
+        buf[:, :d] = G
+        h.aggregate(buf, out)
+        torch.cuda.synchronize()
+        if expect_path is not None:
+            assert h.info(ac.INFO_LAST_PATH) == expect_path
+        G64 = to_f64(G)
+        res = oracle_step_with_kernel_ranks(orc, G64, dtype, h.coeffs(ac.COEFF_A))
+        assert h.status() == int(np.bitwise_or.reduce(res["flags"]))      # an empty segment raises flags
+        assert_coeffs_by_set(h.coeffs(ac.COEFF_GAMMA), res["gamma"], f"pad gamma {t}")
+        assert_coeffs_by_set(h.state()[0], res["m"], f"pad m {t}")
+        assert_output(out, res, G64, dtype, f"pad out {t}", offsets)
+        assert bool((obuf[d:] == 7.0).all()), "wrote past the end of out"
+        assert bool(torch.isnan(buf[:, d:]).all())
+
+
+@pytest.mark.parametrize("N,d,dtype,pitch", [(8, 300_001, "f32", 300_004), (64, 200_003, "bf16", 200_008),
+                                             (16, 123_457, "bf16", 123_520), (5, 77_777, "f32", 80_000)])
+@pytest.mark.parametrize("fused", [False, True])
+def test_padded_rows_odd_length(ac, N, d, dtype, pitch, fused):
+    big = N * pitch * (4 if dtype == "f32" else 2) > 20e6
+    _padded_case(ac, N, d, dtype, pitch, 2, fused=fused, expect_path=1 if (not fused or big) else 3)
+
+
+def test_padded_rows_per_segment(ac):
+    d = 400_003
+    off = [0, 3, 100_001, 100_001, 250_000, d - 2, d]
+    _padded_case(ac, 12, d, "bf16", 400_008, 2, fused=False, offsets=off, per_segment=True, expect_path=1)
+
+
+def test_row_pitch_validation_and_unaligned_pitch(ac):
+    h = ac.AdaCons(4, 1001, "f32")
+    with pytest.raises(ac.AdaConsError):
+        h.set_option(ac.OPT_ROW_PITCH, 1000)            # shorter than a row
+    _padded_case(ac, 4, 1001, "f32", 1003, 1, fused=True, expect_path=2)   # pitch not 16-byte: generic path
+
+
+def test_host_entry_point_with_padded_rows(ac):
+    N, d, pitch = 6, 50_001, 50_008
+    w = wl.Workload("hostpad", N, d, "bf16", 1, "gauss", seed=4)
+    G = wl.generate(w, 0, "cpu")
+    buf = torch.full((N, pitch), float("nan"), dtype=torch.bfloat16).pin_memory()
+    buf[:, :d] = G
+    out = torch.empty(d, dtype=torch.bfloat16).pin_memory()
+    h = ac.AdaCons(N, d, "bf16")
+    h.set_option(ac.OPT_ROW_PITCH, pitch)
+    h.aggregate_host(buf, out)
+    res = oc.AdaConsOracle(N, d).step(to_f64(G), storage="bf16")
+    assert_coeffs(h.coeffs(), res["gamma"], "gamma host padded")
+    assert_output(out, res, to_f64(G), "bf16", "host padded")
