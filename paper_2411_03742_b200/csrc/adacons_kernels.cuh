@@ -122,7 +122,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
 // 16-byte column group l of the box.  Per tile every thread
 //   1. copies its NR row vectors from shared memory to registers,
 //   2. adds them up (partial column sums); with WR > 1 the WR partials are exchanged through
-//      shared memory and added in a fixed order, giving the column sums s of the tile,
+//      shared memory and added in a fixed order (p1_xch_finish), giving the column sums s,
 //   3. accumulates, per row, sum x*s and sum x*x in fp32 (two lanes of packed fp32 FMA).
 // One elected thread refills a stage by TMA as soon as the block has copied it to registers.
 //
@@ -198,6 +198,37 @@ __device__ __forceinline__ void p1_xch_read(const float* xbuf, float2 (&sp)[C::N
       sp[2 * h2] = __fadd2_rn(sp[2 * h2], make_float2(w4.x, w4.y));
       sp[2 * h2 + 1] = __fadd2_rn(sp[2 * h2 + 1], make_float2(w4.z, w4.w));
     }
+}
+// Where a tile's partial column sums are written, and how they become the column sums.
+// WR < 8: double-buffered partials, every thread adds the WR partials of its own column group.
+// WR = 8: adding 8 partials per thread costs more than the tile's own arithmetic warrants, so the
+// 256 threads first finish one column each (the 8 partials in rw order) into the second half of
+// the exchange area, meet at a second barrier, and read back the finished sums of their group.
+template <class C>
+__device__ __forceinline__ float* p1_xch_buffer(float* xch, int k) {
+  return (C::WR == 8) ? xch : xch + (k & 1) * C::kXchOne;
+}
+template <class C>
+__device__ __forceinline__ void p1_xch_finish(float* xch, int k, float2 (&sp)[C::NP], int cw, int lane) {
+  if constexpr (C::WR == 8) {
+    constexpr int per = C::kXchOne / C::WR;
+    float* sbuf = xch + C::kXchOne;
+    for (int idx = threadIdx.x; idx < per; idx += kThreads) {
+      float a = 0.f;
+#pragma unroll
+      for (int r = 0; r < C::WR; ++r) a += xch[r * per + idx];
+      sbuf[idx] = a;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int h2 = 0; h2 < C::VEC / 4; ++h2) {
+      const float4 w4 = *reinterpret_cast<const float4*>(sbuf + (cw * (C::VEC / 4) + h2) * 128 + lane * 4);
+      sp[2 * h2] = make_float2(w4.x, w4.y);
+      sp[2 * h2 + 1] = make_float2(w4.z, w4.w);
+    }
+  } else if constexpr (C::WR > 1) {
+    p1_xch_read<C>(xch + (k & 1) * C::kXchOne, sp, cw, lane);
+  }
 }
 template <int DT, class C>
 __device__ __forceinline__ void p1_accumulate(const uint4 (&v)[C::NR], const float2 (&sp)[C::NP],
@@ -337,7 +368,7 @@ pass1_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm
     }
     float2 sp[C::NP];
     p1_colsum<DT, C>(v, sp);
-    float* xbuf = sm.xch + (k & 1) * C::kXchOne;
+    float* xbuf = p1_xch_buffer<C>(sm.xch, k);
     if (WR > 1) p1_xch_write<C>(xbuf, sp, rw, cw, lane);
     __syncthreads();   // every thread holds its rows in registers; exchange buffer is written
     if (s_abort) break;
@@ -346,7 +377,7 @@ pass1_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm
       issue(k + prm.stages, s);
       issued = k + prm.stages + 1;
     }
-    if (WR > 1) p1_xch_read<C>(xbuf, sp, cw, lane);
+    p1_xch_finish<C>(sm.xch, k, sp, cw, lane);
     p1_accumulate<DT, C>(v, sp, pacc, qacc);
     if (++s == prm.stages) { s = 0; parity ^= 1u; }
   }
@@ -447,7 +478,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
     }
     float2 sp[C::NP];
     p1_colsum<DT, C>(v, sp);
-    float* xbuf = sm.xch + (k & 1) * C::kXchOne;
+    float* xbuf = p1_xch_buffer<C>(sm.xch, k);
     if (WR > 1) p1_xch_write<C>(xbuf, sp, rw, cw, lane);
     __syncthreads();
     if (s_abort) break;
@@ -456,7 +487,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
       issue(k + prm.stages, s);
       issued = k + prm.stages + 1;
     }
-    if (WR > 1) p1_xch_read<C>(xbuf, sp, cw, lane);
+    p1_xch_finish<C>(sm.xch, k, sp, cw, lane);
 
     const long long tile_lo = static_cast<long long>(t0 + k) * C::TILEC;
     const long long tile_hi = tile_lo + C::TILEC < prm.d ? tile_lo + C::TILEC : prm.d;
