@@ -756,3 +756,89 @@ def test_host_entry_point_with_padded_rows(ac):
     res = oc.AdaConsOracle(N, d).step(to_f64(G), storage="bf16")
     assert_coeffs(h.coeffs(), res["gamma"], "gamma host padded")
     assert_output(out, res, to_f64(G), "bf16", "host padded")
+
+
+def test_replay_of_the_single_pass_kernel_from_a_cuda_graph(ac):
+    """The cooperative single-pass launch can be recorded and replayed as well."""
+    w = wl.Workload("graphs", 8, 60_000, "f32", 3, "gauss", seed=321)
+    dev = torch.device("cuda:0")
+    static_G = wl.generate(w, 0, dev)
+    out = torch.empty(w.d, device=dev)
+    h = ac.AdaCons(w.N, w.d, "f32")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        h.aggregate(static_G, out)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 3
+    h.reset()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        h.aggregate(static_G, out)
+    orc = oc.AdaConsOracle(w.N, w.d)
+    for t in range(3):
+        static_G.copy_(wl.generate(w, t, dev))
+        graph.replay()
+        torch.cuda.synchronize()
+        res = oracle_step_with_kernel_ranks(orc, to_f64(static_G), "f32", h.coeffs(ac.COEFF_A))
+        assert_coeffs(h.coeffs(), res["gamma"], f"gamma replay {t}")
+        assert_output(out, res, to_f64(static_G), "f32", f"replay {t}")
+    assert h.state()[1] == 3 and h.status() == 0
+
+
+def test_two_contexts_on_two_streams_are_independent(ac):
+    """Distinct contexts share nothing: interleaved on two streams they give what each gives alone."""
+    dev = torch.device("cuda:0")
+    wa = wl.Workload("ctxa", 16, 900_008, "bf16", 3, "gauss", seed=1)
+    wb = wl.Workload("ctxb", 5, 1_300_000, "f32", 3, "gauss_outlier", seed=2)
+    Ga = [wl.generate(wa, t, dev) for t in range(3)]
+    Gb = [wl.generate(wb, t, dev) for t in range(3)]
+
+    def alone(w, Gs, dtype):
+        h = ac.AdaCons(w.N, w.d, dtype)
+        h.set_option(ac.OPT_FUSED_SMALL, 0)
+        out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
+        outs = []
+        for G in Gs:
+            h.aggregate(G, out)
+            outs.append(out.clone())
+        torch.cuda.synchronize()
+        return outs, h.coeffs().copy()
+
+    ref_a, ca = alone(wa, Ga, "bf16")
+    ref_b, cb = alone(wb, Gb, "f32")
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    ha, hb = ac.AdaCons(wa.N, wa.d, "bf16"), ac.AdaCons(wb.N, wb.d, "f32")
+    ha.set_option(ac.OPT_FUSED_SMALL, 0); hb.set_option(ac.OPT_FUSED_SMALL, 0)
+    oa = [torch.empty(wa.d, dtype=torch.bfloat16, device=dev) for _ in range(3)]
+    ob = [torch.empty(wb.d, device=dev) for _ in range(3)]
+    torch.cuda.synchronize()
+    for t in range(3):
+        ha.aggregate(Ga[t], oa[t], stream=sa)
+        hb.aggregate(Gb[t], ob[t], stream=sb)
+    torch.cuda.synchronize()
+    for t in range(3):
+        assert torch.equal(oa[t].view(torch.uint8), ref_a[t].view(torch.uint8))
+        assert torch.equal(ob[t], ref_b[t])
+    assert ha.coeffs(stream=sa).tobytes() == ca.tobytes() and hb.coeffs(stream=sb).tobytes() == cb.tobytes()
+
+
+def test_profile_and_info_getters(ac):
+    w = wl.Workload("prof", 8, 2_000_000, "f32", 1, "gauss", seed=5)
+    G = wl.generate(w, 0, "cuda:0")
+    out = torch.empty(w.d, device="cuda:0")
+    h = ac.AdaCons(w.N, w.d, "f32")
+    with pytest.raises(ac.AdaConsError):
+        h.profile()                                   # profiling is off
+    h.set_option(ac.OPT_PROFILE, 1)
+    for _ in range(5):
+        h.aggregate(G, out)
+    ms, n = h.profile()
+    assert n == 5 and all(m > 0 for m in ms) and sum(ms) < 50
+    assert h.info(ac.INFO_PASS1_BLOCKS) > 0 and h.info(ac.INFO_SCRATCH_BYTES) > 0
+    assert h.info(ac.INFO_NUM_SEGMENTS) == 1 and h.info(ac.INFO_COEFF_SETS) == 1
+    assert h.get_option(ac.OPT_BETA) == 0.99 and h.get_option(ac.OPT_ROW_PITCH) == w.d
+    with pytest.raises(ac.AdaConsError):
+        h.info(99)
