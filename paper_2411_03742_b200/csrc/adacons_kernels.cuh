@@ -624,22 +624,33 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
   const int begin = prm.rec_begin ? prm.rec_begin[set] : 0;
   const int count = prm.rec_count ? prm.rec_count[set] : prm.num_partials;
   const float* base = prm.partials + static_cast<size_t>(begin) * V;
-  const int groups = T >= V ? T / V : 1;
-  if (T >= V) {
-    const int g = i / V, v = i % V;
-    if (g < groups) {
-      double acc = 0.0;
+  // A record is V = 2N floats, read as 16-byte (N even) or 8-byte vectors; `groups` interleaved
+  // subsequences of the records are summed in parallel (at most 32, and groups * V <= 2048).
+  const int w = (V % 4 == 0) ? 4 : 2;
+  const int units = V / w;
+  int groups = T / units;
+  if (groups > 32) groups = 32;
+  if (groups > 2 * kMaxN / V) groups = 2 * kMaxN / V;
+  if (groups < 1) groups = 1;
+  for (int slot = i; slot < units * groups; slot += T) {
+    const int g = slot / units, u = slot - g * units;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    const float* src = base + static_cast<size_t>(u) * w;
+    if (w == 4) {
 #pragma unroll 4
-      for (int c = g; c < count; c += groups) acc += static_cast<double>(__ldcg(base + static_cast<size_t>(c) * V + v));
-      sh_part[g * V + v] = acc;
-    }
-  } else {
-    for (int v = i; v < V; v += T) {
-      double acc = 0.0;
+      for (int c = g; c < count; c += groups) {
+        const float4 x = __ldcg(reinterpret_cast<const float4*>(src + static_cast<size_t>(c) * V));
+        acc[0] += static_cast<double>(x.x); acc[1] += static_cast<double>(x.y);
+        acc[2] += static_cast<double>(x.z); acc[3] += static_cast<double>(x.w);
+      }
+    } else {
 #pragma unroll 4
-      for (int c = 0; c < count; ++c) acc += static_cast<double>(__ldcg(base + static_cast<size_t>(c) * V + v));
-      sh_part[v] = acc;
+      for (int c = g; c < count; c += groups) {
+        const float2 x = __ldcg(reinterpret_cast<const float2*>(src + static_cast<size_t>(c) * V));
+        acc[0] += static_cast<double>(x.x); acc[1] += static_cast<double>(x.y);
+      }
     }
+    for (int e = 0; e < w; ++e) sh_part[g * V + u * w + e] = acc[e];
   }
   __syncthreads();
   double p = 0.0, q = 0.0;
