@@ -116,7 +116,8 @@ enum adacons_info {
   ADACONS_INFO_SCRATCH_BYTES = 3,    /* device bytes owned by the context                        */
   ADACONS_INFO_LAUNCHES_PER_CALL = 4,/* kernels launched by the most recent adacons_aggregate    */
   ADACONS_INFO_LAST_PATH = 5,        /* 0 = none yet, 1 = TMA-staged fast path, 2 = generic path,
-                                        3 = single-pass kernel (matrix held in shared memory)   */
+                                        3 = single-pass kernel (matrix held in shared memory),
+                                        4 = N > 64: column sums, then dot products per 64 rows  */
   ADACONS_INFO_TOTAL_LAUNCHES = 6    /* kernels launched by this context so far                  */
 };
 
@@ -143,8 +144,10 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  *          (row i = g_i starts at element i*pitch; pitch = d unless ADACONS_OPT_ROW_PITCH is set).
  *   out    device pointer, d elements of the same type; must not overlap grads.
  *   Fast path: grads and out 16-byte aligned, the row pitch in bytes (d*sizeof(element) unless
- *   ADACONS_OPT_ROW_PITCH says otherwise) a multiple of 16, N <= 64.
- *   Anything else is served by a slower generic path with the same results.
+ *   ADACONS_OPT_ROW_PITCH says otherwise) a multiple of 16.  With N <= 64 the matrix is read
+ *   twice; with N > 64 three times (column sums first, then dot products per 64 rows; needs d
+ *   floats of scratch, allocated in adacons_create).  Misaligned buffers or pitch are served by a
+ *   slower generic path with the same results.
  * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
  * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.
  * Errors: EINVAL (NULL pointers, overlap), ECUDA (launch failure).

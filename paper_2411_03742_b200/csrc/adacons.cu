@@ -60,7 +60,7 @@ struct adacons_ctx {
   int max_partials = 0;
 
   // device memory
-  float* partials = nullptr;      // [max_partials][sets][2N]
+  float* partials = nullptr;      // [max_partials][2N]
   double* coef = nullptr;         // [5][sets][N]
   float* gamma_f32 = nullptr;     // [sets][N]
   double* m = nullptr;            // [sets][N]
@@ -69,6 +69,16 @@ struct adacons_ctx {
   void* staging = nullptr;        // adacons_aggregate_host: N*pitch + d elements
   size_t staging_bytes = 0;
   size_t scratch_bytes = 0;
+
+  // more than 64 workers: column sums to scratch, then dot products per 64-row chunk
+  bool big_available = false;
+  int big_grid = 0, big_tiles = 0, big_stages = 0;
+  size_t big_smem = 0;
+  float* d_colsum = nullptr;            // [big_tiles * tile columns], zero past d
+  size_t colsum_bytes = 0;
+  CUtensorMap tmap_big;
+  const void* tmap_big_for = nullptr;
+  int last_launches = 3;
 
   // single-pass path for problems that fit in the grid's shared memory
   bool fused_available = false;
@@ -203,6 +213,57 @@ int plan_fast(adacons_ctx* c) {
   f.grid = per_sm * c->num_sms;
   if (f.grid > f.num_tiles) f.grid = f.num_tiles;
   f.available = true;
+  return ADACONS_OK;
+}
+
+// N > 64 on the aligned path: needs d floats of scratch for the column sums.
+int plan_big(adacons_ctx* c) {
+  c->big_available = false;
+  if (c->N <= kMaxFastN) return ADACONS_OK;
+  if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > 2147483647ll - 8192) return ADACONS_OK;
+  const int tile_cols = kBoxRowBytes / c->elem_bytes;
+  c->big_tiles = static_cast<int>((c->d + tile_cols - 1) / tile_cols);
+  const uint32_t stage_bytes = 64u * kBoxRowBytes;
+  const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
+  const size_t fixed = static_cast<size_t>(2) * 8 * 32 * vec * sizeof(float) + static_cast<size_t>(kWarps) * 8 * 2 * sizeof(float);
+  c->big_stages = 2;
+  c->big_smem = static_cast<size_t>(c->big_stages) * stage_bytes + fixed + static_cast<size_t>(c->big_stages) * 8;
+  const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_dot_kernel<0>)
+                                          : reinterpret_cast<const void*>(&pass1_dot_kernel<1>);
+  int per_sm = 0;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->big_smem)) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, c->big_smem) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  c->big_grid = per_sm * c->num_sms;
+  if (c->big_grid > c->big_tiles) c->big_grid = c->big_tiles;
+  const size_t need = static_cast<size_t>(c->big_tiles) * tile_cols * sizeof(float);
+  if (need > c->colsum_bytes) {
+    cudaFree(c->d_colsum);
+    c->d_colsum = nullptr;
+    c->colsum_bytes = 0;
+    if (cudaMalloc(&c->d_colsum, need) != cudaSuccess) { cudaGetLastError(); return ADACONS_ENOMEM; }
+    c->colsum_bytes = need;
+  }
+  if (cudaMemset(c->d_colsum, 0, c->colsum_bytes) != cudaSuccess) return ADACONS_ECUDA;
+  c->big_available = true;
+  return ADACONS_OK;
+}
+
+int encode_map_big(adacons_ctx* c, const void* grads) {
+  if (c->tmap_big_for == grads) return ADACONS_OK;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), 64u};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = c->encode(&c->tmap_big,
+                               c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                               2, const_cast<void*>(grads), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  c->tmap_big_for = grads;
   return ADACONS_OK;
 }
 
@@ -455,6 +516,9 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   if (c->fast.available && c->fast.grid > c->max_partials) c->max_partials = c->fast.grid;
   plan_fused(c);
   if (c->fused_available && c->fused_grid > c->max_partials) c->max_partials = c->fused_grid;
+  rc = plan_big(c);
+  if (rc != ADACONS_OK) { adacons_destroy(c); return rc; }
+  if (c->big_available && c->big_grid > c->max_partials) c->max_partials = c->big_grid;
 
   if (cudaMalloc(&c->flags, sizeof(uint32_t)) != cudaSuccess || cudaMalloc(&c->step, sizeof(long long)) != cudaSuccess ||
       cudaMalloc(&c->d_barrier, sizeof(unsigned long long)) != cudaSuccess) {
@@ -478,7 +542,7 @@ int adacons_destroy(adacons_ctx* c) {
   if (c == nullptr) return ADACONS_OK;
   DeviceGuard g(c->device);
   cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
-  cudaFree(c->flags); cudaFree(c->step); cudaFree(c->staging); cudaFree(c->d_barrier);
+  cudaFree(c->flags); cudaFree(c->step); cudaFree(c->staging); cudaFree(c->d_barrier); cudaFree(c->d_colsum);
   free_seg_plan(c);
   if (c->prof_ready)
     for (int s = 0; s < adacons_ctx::kProfSlots; ++s)
@@ -503,6 +567,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   const long long row_bytes = c->pitch * c->elem_bytes;
   const int N = c->N;
   int num_partials;
+  int extra_launches = 0;
   cudaEvent_t* ev = (c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
   if (ev) cudaEventRecord(ev[0], st);
 
@@ -530,6 +595,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); cudaEventRecord(ev[3], st); c->prof_calls += 1; }
     c->last_path = 3;
+    c->last_launches = 1;
     c->total_launches += 1;
     return ADACONS_OK;
   }
@@ -563,6 +629,29 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     num_partials = c->fast.grid;
     c->last_path = 1;
+  } else if (aligned && c->big_available) {
+    int rc = encode_map_big(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    const unsigned cblocks = static_cast<unsigned>((num_vec + kThreads - 1) / kThreads);
+    const unsigned char* g8 = static_cast<const unsigned char*>(grads);
+    if (c->dtype == ADACONS_F32) colsum_kernel<0><<<cblocks, kThreads, 0, st>>>(g8, c->d_colsum, N, row_bytes, num_vec, tail_elems);
+    else colsum_kernel<1><<<cblocks, kThreads, 0, st>>>(g8, c->d_colsum, N, row_bytes, num_vec, tail_elems);
+    if (!launch_ok()) return ADACONS_ECUDA;
+    const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_dot_kernel<0>)
+                                            : reinterpret_cast<const void*>(&pass1_dot_kernel<1>);
+    for (int r0 = 0; r0 < N; r0 += 64) {
+      Pass1DotParams p;
+      p.N = N; p.r0 = r0; p.rows = N - r0 < 64 ? N - r0 : 64; p.num_tiles = c->big_tiles; p.stages = c->big_stages;
+      p.stage_bytes = 64u * kBoxRowBytes; p.s = c->d_colsum; p.partials = c->partials; p.flags = c->flags;
+      void* args[2] = {&c->tmap_big, &p};
+      if (cudaLaunchKernel(k, dim3(c->big_grid), dim3(kThreads), args, c->big_smem, st) != cudaSuccess) {
+        cudaGetLastError();
+        return ADACONS_ECUDA;
+      }
+      extra_launches += 1;
+    }
+    num_partials = c->big_grid;
+    c->last_path = 4;
   } else {
     if (c->dtype == ADACONS_F32)
       pass1_generic_kernel<0><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->pitch, c->generic_tiles, c->partials);
@@ -615,7 +704,8 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   }
   if (e2 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
   if (ev) { cudaEventRecord(ev[3], st); c->prof_calls += 1; }
-  c->total_launches += 3;
+  c->last_launches = 3 + extra_launches;
+  c->total_launches += c->last_launches;
   return ADACONS_OK;
 }
 
@@ -701,9 +791,13 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       int rc = plan_fast(c);
       if (rc != ADACONS_OK) return rc;
       plan_fused(c);
+      c->tmap_big_for = nullptr;
+      rc = plan_big(c);
+      if (rc != ADACONS_OK) return rc;
       int need = c->generic_grid;
       if (c->fast.available && c->fast.grid > need) need = c->fast.grid;
       if (c->fused_available && c->fused_grid > need) need = c->fused_grid;
+      if (c->big_available && c->big_grid > need) need = c->big_grid;
       if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
         cudaFree(c->partials);
         c->partials = nullptr;
@@ -835,7 +929,7 @@ int adacons_get_info(adacons_ctx* c, int key, int64_t* value) {
     case ADACONS_INFO_COEFF_SETS: *value = c->sets(); return ADACONS_OK;
     case ADACONS_INFO_PASS1_BLOCKS: *value = c->fast.available ? c->fast.grid : c->generic_grid; return ADACONS_OK;
     case ADACONS_INFO_SCRATCH_BYTES: *value = static_cast<int64_t>(c->scratch_bytes); return ADACONS_OK;
-    case ADACONS_INFO_LAUNCHES_PER_CALL: *value = c->last_path == 3 ? 1 : 3; return ADACONS_OK;
+    case ADACONS_INFO_LAUNCHES_PER_CALL: *value = c->last_launches; return ADACONS_OK;
     case ADACONS_INFO_LAST_PATH: *value = c->last_path; return ADACONS_OK;
     case ADACONS_INFO_TOTAL_LAUNCHES: *value = c->total_launches; return ADACONS_OK;
     default: return ADACONS_EINVAL;

@@ -260,11 +260,11 @@ __device__ __forceinline__ void p1_accumulate_masked(const uint4 (&v)[C::NR], co
     }
 }
 // Block partial of the accumulators: lanes (fixed xor tree), then the WC warps that share a row
-// (fixed order).  dst[0..N) = N p_i (un-divided), dst[N..2N) = q_i.  Contains two barriers; the
-// accumulators are reset.
+// (fixed order).  dst_p[0..rows) = N p_i (un-divided), dst_q[0..rows) = q_i.  Contains two
+// barriers; the accumulators are reset.
 template <class C>
 __device__ __forceinline__ void p1_block_store(float2 (&pacc)[C::NR], float2 (&qacc)[C::NR], float* red,
-                                               float* dst, int N) {
+                                               float* dst_p, float* dst_q, int rows) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 #pragma unroll
   for (int j = 0; j < C::NR; ++j) {
@@ -281,7 +281,7 @@ __device__ __forceinline__ void p1_block_store(float2 (&pacc)[C::NR], float2 (&q
     pacc[j] = qacc[j] = make_float2(0.f, 0.f);
   }
   __syncthreads();
-  if (tid < N) {
+  if (tid < rows) {
     const int r_w = tid % C::WR, j = tid / C::WR;
     float p = 0.f, q = 0.f;
 #pragma unroll
@@ -289,8 +289,8 @@ __device__ __forceinline__ void p1_block_store(float2 (&pacc)[C::NR], float2 (&q
       p += red[((c * C::WR + r_w) * C::NR + j) * 2 + 0];
       q += red[((c * C::WR + r_w) * C::NR + j) * 2 + 1];
     }
-    dst[tid] = p;
-    dst[N + tid] = q;
+    dst_p[tid] = p;
+    dst_q[tid] = q;
   }
   __syncthreads();
 }
@@ -388,7 +388,133 @@ pass1_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm
     if (tid < 2 * N) dst[tid] = 0.f;
     return;
   }
-  p1_block_store<C>(pacc, qacc, sm.red, dst, N);
+  p1_block_store<C>(pacc, qacc, sm.red, dst, dst + N, N);
+}
+
+// ---- pass 1 for more than 64 workers: column sums first, then dot products per 64-row chunk -----
+// With N > 64 a tile of all rows no longer fits the ring.  colsum_kernel streams the matrix once
+// and leaves the column sums s (fp32) in scratch; pass1_dot_kernel then runs once per chunk of 64
+// rows with the same boxes, ring and warp grid as pass1_tma_kernel<DT, 8, 8>, reading s instead of
+// exchanging partial sums, and writes its rows' slice of the block partial.  Pass 1 costs two
+// reads of the matrix instead of one.
+template <int DT>
+__global__ void __launch_bounds__(kThreads)
+colsum_kernel(const unsigned char* __restrict__ grads, float* __restrict__ s_out, int N, long long row_bytes,
+              long long num_vec, int tail_elems) {
+  constexpr int VEC = Elem<DT>::kVec;
+  constexpr int NP = VEC / 2;
+  constexpr int U = 8;
+  const long long v = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+  if (v >= num_vec) return;
+  const unsigned char* col = grads + v * 16;
+  float2 acc[NP];
+#pragma unroll
+  for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+  int i0 = 0;
+  for (; i0 + U <= N; i0 += U) {
+    uint4 x[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) x[u] = ld_stream_v4(col + static_cast<long long>(i0 + u) * row_bytes);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int h = 0; h < NP; ++h) acc[h] = __fadd2_rn(acc[h], unpack_pair<DT>(x[u], h));
+  }
+  for (; i0 < N; ++i0) {
+    const uint4 x = ld_stream_v4(col + static_cast<long long>(i0) * row_bytes);
+#pragma unroll
+    for (int h = 0; h < NP; ++h) acc[h] = __fadd2_rn(acc[h], unpack_pair<DT>(x, h));
+  }
+  float* dst = s_out + v * VEC;
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    float x = (e & 1) ? acc[e / 2].y : acc[e / 2].x;
+    if (tail_elems != 0 && v == num_vec - 1 && e >= tail_elems) x = 0.f;   // row padding is not data
+    dst[e] = x;
+  }
+}
+
+struct Pass1DotParams {
+  int N;                // all workers (row pitch of the partials)
+  int r0;               // first row of this chunk
+  int rows;             // rows in this chunk (<= 64)
+  int num_tiles;
+  int stages;
+  uint32_t stage_bytes; // 64 * 512
+  const float* s;       // column sums, zero past d, padded to a whole tile
+  float* partials;      // [gridDim.x][2N]
+  uint32_t* flags;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 2)
+pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams prm) {
+  using C = P1<DT, 8, 8>;
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int s_abort;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rw = warp;                               // WR = 8, WC = 1
+  const P1Smem sm = p1_carve<C>(smem_raw, prm.stages, prm.stage_bytes);
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < prm.stages; ++s) mbar_init(&sm.full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+  const int first = blockIdx.x, stride = gridDim.x;
+  const int my_tiles = first < prm.num_tiles ? (prm.num_tiles - first + stride - 1) / stride : 0;
+  auto issue = [&](int k, int s) {
+    mbar_expect_tx(&sm.full[s], prm.stage_bytes);
+    tma_load_2d(sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes, &tmap, &sm.full[s],
+                (first + k * stride) * C::TILEC, prm.r0);
+  };
+  int issued = 0;
+  if (tid == 0) {
+    const int pre = my_tiles < prm.stages ? my_tiles : prm.stages;
+    for (int k = 0; k < pre; ++k) issue(k, k);
+    issued = pre;
+  }
+  float2 pacc[8], qacc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  int s = 0;
+  uint32_t parity = 0;
+  for (int k = 0; k < my_tiles; ++k) {
+    // column sums of this thread's 16-byte group (in flight while the tile lands)
+    float2 sp[C::NP];
+    const float* sv = prm.s + static_cast<long long>(first + k * stride) * C::TILEC + lane * C::VEC;
+#pragma unroll
+    for (int h2 = 0; h2 < C::VEC / 4; ++h2) {
+      const float4 w4 = __ldg(reinterpret_cast<const float4*>(sv) + h2);
+      sp[2 * h2] = make_float2(w4.x, w4.y);
+      sp[2 * h2 + 1] = make_float2(w4.z, w4.w);
+    }
+    uint4 v[8];
+    if (mbar_wait_bounded(&sm.full[s], parity)) {
+      p1_load_rows<C>(v, sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes + lane * 16, rw, 64);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
+      atomicOr(&s_abort, 1);
+    }
+    __syncthreads();                                   // the stage is in registers
+    if (s_abort) break;
+    if (tid == 0 && k + prm.stages < my_tiles) {
+      fence_proxy_async_smem();
+      issue(k + prm.stages, s);
+      issued = k + prm.stages + 1;
+    }
+    p1_accumulate<DT, C>(v, sp, pacc, qacc);
+    if (++s == prm.stages) { s = 0; parity ^= 1u; }
+  }
+  float* dst = prm.partials + static_cast<size_t>(blockIdx.x) * 2 * prm.N;
+  if (s_abort) {
+    if (tid == 0) p1_drain_after_timeout(sm.full, prm.stages, issued, prm.flags);
+    if (tid < prm.rows) { dst[prm.r0 + tid] = 0.f; dst[prm.N + prm.r0 + tid] = 0.f; }
+    return;
+  }
+  p1_block_store<C>(pacc, qacc, sm.red, dst + prm.r0, dst + prm.N + prm.r0, prm.rows);
 }
 
 // ---- per-segment ("layer-wise") pass 1 ----------------------------------------------------------
@@ -500,7 +626,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
         const long long hi = seg_end < tile_hi ? seg_end : tile_hi;
         if (hi > lo) p1_accumulate_masked<DT, C>(v, sp, pacc, qacc, col0, lo, hi);
         if (seg_end <= tile_hi && seg < last_seg) {
-          p1_block_store<C>(pacc, qacc, sm.red, record(seg), N);
+          p1_block_store<C>(pacc, qacc, sm.red, record(seg), record(seg) + N, N);
           ++seg;
           seg_end = prm.seg_off[seg + 1];
           lo = hi;                                              // empty segments fall through here
@@ -516,7 +642,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
     if (tid == 0) p1_drain_after_timeout(sm.full, prm.stages, issued, prm.flags);
     return;   // the records keep whatever they held; the status word says the result is invalid
   }
-  p1_block_store<C>(pacc, qacc, sm.red, record(seg), N);
+  p1_block_store<C>(pacc, qacc, sm.red, record(seg), record(seg) + N, N);
 }
 
 // ----------------------------------------------------------------------------------------------

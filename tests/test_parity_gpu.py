@@ -648,7 +648,22 @@ def test_config3_full_size_streamed_oracle(ac):
 @pytest.mark.parametrize("N", [512, 600, 1024])
 def test_many_workers(ac, N):
     w = wl.Workload(f"many{N}", N, 3_000, "f32", 2, "gauss", seed=N)
+    run_case(ac, w, 2, beta=0.9, expect_path=4)
+    w = wl.Workload(f"manyodd{N}", N, 3_001, "f32", 2, "gauss", seed=N)      # unaligned: generic path
     run_case(ac, w, 2, beta=0.9, expect_path=2)
+
+
+@pytest.mark.parametrize("N,d,dtype", [(65, 400_008, "bf16"), (100, 300_004, "f32"), (128, 500_000, "bf16"),
+                                       (200, 150_000, "f32"), (257, 100_008, "bf16")])
+def test_more_than_64_workers_column_sum_then_dot_path(ac, N, d, dtype):
+    """N > 64 on aligned buffers: column sums to scratch, then one dot-product launch per 64 rows
+    (the last chunk is ragged)."""
+    w = wl.Workload(f"big{N}", N, d, dtype, 2, "gauss", seed=N)
+    h = run_case(ac, w, 2, beta=0.8, expect_path=4)
+
+
+def test_more_than_64_workers_with_padded_rows(ac):
+    _padded_case(ac, 96, 123_457, "bf16", 123_464, 2, fused=False, expect_path=4)
 
 
 # ---- the call neither allocates nor synchronises: it can be recorded once and replayed -----------
