@@ -48,7 +48,7 @@ def parse_args(argv=None):
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--d", type=int, default=0, help="override the gradient length (debugging)")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--overlap-launch", action="store_true", help="programmatic dependent launch between the kernels")
+    ap.add_argument("--no-overlap-launch", action="store_true", help="plain stream order for the coefficient kernel too")
     ap.add_argument("--per-segment", action="store_true", help="layer-wise coefficients (workloads with segments)")
     ap.add_argument("--no-profile", action="store_true",
                     help="keep the per-kernel CUDA events out of the timed region (they are taken in a second loop)")
@@ -248,8 +248,8 @@ def run_ours(args):
     h = ac.AdaCons(w.N, w.d, w.dtype, seg_offsets=wl.segment_offsets(w))
     if args.per_segment:
         h.set_option(ac.OPT_PER_SEGMENT, 1)
-    if args.overlap_launch:
-        h.set_option(ac.OPT_OVERLAP_LAUNCH, 1)
+    if args.no_overlap_launch:
+        h.set_option(ac.OPT_OVERLAP_LAUNCH, 0)
     stream = torch.cuda.current_stream()
 
     for t in range(max(args.warmup, 3)):

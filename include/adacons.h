@@ -80,12 +80,12 @@ enum adacons_option {
   ADACONS_OPT_PROFILE = 5,     /* 0 (default) / 1: record CUDA events around each of the three
                                   kernels of every aggregate call (see adacons_get_profile).
                                   Setting it (to either value) clears the recorded samples.      */
-  ADACONS_OPT_OVERLAP_LAUNCH = 6, /* 0 (default): plain stream order between the three kernels;
-                                  1: the coefficient step and pass 2 are launched with
-                                  programmatic stream serialisation (their blocks may become
-                                  resident while the kernel before them still runs).  Measured
-                                  slower on B200 for every workload tried, hence off; no effect
-                                  on results.                                                    */
+  ADACONS_OPT_OVERLAP_LAUNCH = 6, /* 1 (default): the one-block coefficient kernel is launched with
+                                  programmatic stream serialisation, so its launch latency hides
+                                  behind pass 1 (it waits for pass 1 on the device); 0: plain
+                                  stream order.  Pass 2 is always launched in plain stream order
+                                  (letting its blocks become resident early measured slower).
+                                  No effect on results.                                          */
   ADACONS_OPT_FUSED_SMALL = 7, /* 1 (default): when the whole matrix fits in the shared memory of
                                   the grid (about 148 x 160 KB) and the buffers are 16-byte
                                   aligned, one cooperative kernel reads it from HBM once and does

@@ -50,7 +50,7 @@ struct adacons_ctx {
 
   // options
   double beta = 0.99;
-  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0, overlap_launch = 0, fused_small = 1;
+  int momentum = 1, sorted = 1, normalize = 1, per_segment = 0, overlap_launch = 1, fused_small = 1;
 
   // plans
   Pass1Plan fast;
@@ -571,7 +571,9 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   cudaEvent_t* ev = (c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
   if (ev) cudaEventRecord(ev[0], st);
 
-  const bool pdl = (ev == nullptr) && c->overlap_launch;   // event records between the kernels would defeat the overlap
+  // the coefficient kernel may be launched while pass 1 still runs (it waits for it on the device);
+  // event records between the kernels would defeat that
+  const bool pdl = (ev == nullptr) && c->overlap_launch;
   const bool seg = c->per_segment != 0;
   if (seg && !(aligned && c->fast.available && c->seg_kernel != nullptr)) return ADACONS_EALIGN;
 
@@ -690,17 +692,17 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     const int* bs = c->d_pass2_blk_seg;
     const long long* so = c->d_seg_off;
     if (c->dtype == ADACONS_F32)
-      e2 = seg ? launch_kernel(pass2_vec_kernel<0, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
-               : launch_kernel(pass2_vec_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
+      e2 = seg ? launch_kernel(pass2_vec_kernel<0, true>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
+               : launch_kernel(pass2_vec_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
     else
-      e2 = seg ? launch_kernel(pass2_vec_kernel<1, true>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
-               : launch_kernel(pass2_vec_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, pdl, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
+      e2 = seg ? launch_kernel(pass2_vec_kernel<1, true>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
+               : launch_kernel(pass2_vec_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
   } else {
     const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);
     if (c->dtype == ADACONS_F32)
-      e2 = launch_kernel(pass2_generic_kernel<0>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d, c->pitch);
+      e2 = launch_kernel(pass2_generic_kernel<0>, dim3(blocks), dim3(kThreads), 0, st, false, grads, out, c->gamma_f32, N, c->d, c->pitch);
     else
-      e2 = launch_kernel(pass2_generic_kernel<1>, dim3(blocks), dim3(kThreads), 0, st, pdl, grads, out, c->gamma_f32, N, c->d, c->pitch);
+      e2 = launch_kernel(pass2_generic_kernel<1>, dim3(blocks), dim3(kThreads), 0, st, false, grads, out, c->gamma_f32, N, c->d, c->pitch);
   }
   if (e2 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
   if (ev) { cudaEventRecord(ev[3], st); c->prof_calls += 1; }
