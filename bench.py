@@ -255,24 +255,30 @@ def run_ours(args):
     for t in range(max(args.warmup, 3)):
         h.aggregate(Gs[t % nbuf], out)
     torch.cuda.synchronize()
-    if not args.no_profile:
-        h.set_option(ac.OPT_PROFILE, 1)
-    launches0 = h.info(ac.INFO_TOTAL_LAUNCHES)
-
-    sampler = ClockSampler(physical_gpu_index(local))
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    ev0.record(stream)
-    for t in range(args.steps):
-        h.aggregate(Gs[t % nbuf], out)
-    ev1.record(stream)
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    barrier()
-    ms_local = ev0.elapsed_time(ev1)
-    launches = h.info(ac.INFO_TOTAL_LAUNCHES) - launches0
+    # A timed region that saw a thermal or hardware slowdown is measured once more.
+    for attempt in range(2):
+        if not args.no_profile:
+            h.set_option(ac.OPT_PROFILE, 1)          # also clears the recorded samples
+        launches0 = h.info(ac.INFO_TOTAL_LAUNCHES)
+        sampler = ClockSampler(physical_gpu_index(local))
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        ev0.record(stream)
+        for t in range(args.steps):
+            h.aggregate(Gs[t % nbuf], out)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        barrier()
+        ms_local = ev0.elapsed_time(ev1)
+        launches = h.info(ac.INFO_TOTAL_LAUNCHES) - launches0
+        slowed = any(r in clocks["reasons"] for r in ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"))
+        slowed_anywhere = reduce_over_ranks(1.0 if slowed else 0.0, 0.0, device=dev)[0] > 0.0
+        clocks["remeasured"] = attempt > 0
+        if not slowed_anywhere:
+            break
     if args.no_profile:
         h.set_option(ac.OPT_PROFILE, 1)
         for t in range(args.steps):
