@@ -126,7 +126,7 @@ enum adacons_info {
  * (problem statement: Eq. 4, psi_t : {g_i}_{i=1..N} -> R^d, stateful in t).
  *   out          receives the context (host pointer, must not be NULL).
  *   N            1 <= N <= 1024.
- *   d            1 <= d < 2^31.
+ *   d            1 <= d < 2^40 (per-segment mode and the N > 64 fast path: d <= 2^30).
  *   seg_offsets  host pointer to num_segments+1 ascending offsets with seg_offsets[0] = 0 and
  *                seg_offsets[num_segments] = d (segments may be empty and need no alignment);
  *                NULL / num_segments = 0 means one segment [0, d).  Copied; the caller keeps

@@ -23,6 +23,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// TMA coordinates are 32-bit: longer vectors are walked in column chunks of this many elements,
+// each with its own tensor map and its own slice of the partial records.
+constexpr long long kChunkCols = 1ll << 30;
+
 struct Pass1Plan {            // TMA-staged pass 1 for this (N, dtype)
   bool available = false;
   int NR = 0, WR = 0;
@@ -101,7 +105,8 @@ struct adacons_ctx {
   size_t seg_bytes = 0;
 
   EncodeTiledFn encode = nullptr;
-  CUtensorMap tmap;
+  int num_chunks = 1;                   // ceil(d / kChunkCols)
+  std::vector<CUtensorMap> tmaps;       // one per column chunk; tmaps[0] covers everything when d <= 2^30
   const void* tmap_for = nullptr;
 
   int last_path = 0;
@@ -177,8 +182,11 @@ int plan_fast(adacons_ctx* c) {
   const int N = c->N;
   if (N > kMaxFastN) return ADACONS_OK;
   if ((c->pitch * c->elem_bytes) % 16 != 0) return ADACONS_OK;
-  if (c->d > 2147483647ll - 8192) return ADACONS_OK;
   if (c->encode == nullptr) return ADACONS_OK;
+  c->num_chunks = static_cast<int>((c->d + kChunkCols - 1) / kChunkCols);
+  c->tmaps.resize(static_cast<size_t>(c->num_chunks));
+  c->tmap_for = nullptr;
+  const long long first_cols = c->d < kChunkCols ? c->d : kChunkCols;   // columns of the first (largest) chunk
   int WR, NR;
   if (N <= 8) { WR = 1; NR = N <= 1 ? 1 : N <= 2 ? 2 : N <= 4 ? 4 : 8; }
   else if (N <= 16) { WR = 2; NR = 8; }
@@ -188,7 +196,7 @@ int plan_fast(adacons_ctx* c) {
   const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
   f.NR = NR; f.WR = WR;
   f.tile_cols = WC * (kBoxRowBytes / c->elem_bytes);
-  f.num_tiles = static_cast<int>((c->d + f.tile_cols - 1) / f.tile_cols);
+  f.num_tiles = static_cast<int>((first_cols + f.tile_cols - 1) / f.tile_cols);
   f.stage_bytes = static_cast<uint32_t>(WC) * N * kBoxRowBytes;
   const size_t xch = WR > 1 ? static_cast<size_t>(2) * WR * WC * 32 * vec * sizeof(float) : 0;
   const size_t fixed = xch + static_cast<size_t>(kWarps) * NR * 2 * sizeof(float);
@@ -220,7 +228,7 @@ int plan_fast(adacons_ctx* c) {
 int plan_big(adacons_ctx* c) {
   c->big_available = false;
   if (c->N <= kMaxFastN) return ADACONS_OK;
-  if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > 2147483647ll - 8192) return ADACONS_OK;
+  if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > kChunkCols) return ADACONS_OK;
   const int tile_cols = kBoxRowBytes / c->elem_bytes;
   c->big_tiles = static_cast<int>((c->d + tile_cols - 1) / tile_cols);
   const uint32_t stage_bytes = 64u * kBoxRowBytes;
@@ -300,16 +308,21 @@ int plan_fused(adacons_ctx* c) {
 
 int encode_map(adacons_ctx* c, const void* grads) {
   if (c->tmap_for == grads) return ADACONS_OK;
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(c->N)};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = c->encode(&c->tmap,
-                               c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                               2, const_cast<void*>(grads), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  for (int ch = 0; ch < c->num_chunks; ++ch) {
+    const long long col0 = static_cast<long long>(ch) * kChunkCols;
+    const long long cols = c->d - col0 < kChunkCols ? c->d - col0 : kChunkCols;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(c->N)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(c->N)};
+    const cuuint32_t estr[2] = {1, 1};
+    void* base = const_cast<unsigned char*>(static_cast<const unsigned char*>(grads)) + col0 * c->elem_bytes;
+    const CUresult r = c->encode(&c->tmaps[static_cast<size_t>(ch)],
+                                 c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  }
   c->tmap_for = grads;
   return ADACONS_OK;
 }
@@ -374,7 +387,7 @@ int upload(T** dst, const std::vector<T>& src, size_t* bytes) {
 // Host plan of the per-segment mode: which block meets which segments, where each (set, block)
 // partial record lives, and which segment each pass-2 block works in.
 int build_seg_plan(adacons_ctx* c) {
-  if (!c->fast.available) return ADACONS_EALIGN;   // needs the TMA path: N <= 64, 16-byte row pitch
+  if (!c->fast.available || c->num_chunks != 1) return ADACONS_EALIGN;   // needs the TMA path: N <= 64, 16-byte row pitch, d <= 2^30
   free_seg_plan(c);
   const int S = c->num_segments;
   const std::vector<long long>& off = c->seg_offsets;
@@ -461,7 +474,7 @@ const char* adacons_strerror(int code) {
 int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t* seg_offsets, int num_segments) {
   if (out == nullptr) return ADACONS_EINVAL;
   *out = nullptr;
-  if (N < 1 || N > kMaxN || d < 1 || d >= (1ll << 31)) return ADACONS_EINVAL;
+  if (N < 1 || N > kMaxN || d < 1 || d >= (1ll << 40)) return ADACONS_EINVAL;
   if (dtype != ADACONS_F32 && dtype != ADACONS_BF16) return ADACONS_EINVAL;
   if (num_segments < 0 || (num_segments > 0 && seg_offsets == nullptr)) return ADACONS_EINVAL;
   if (num_segments > 0) {
@@ -513,7 +526,7 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   c->generic_grid = sms * 4;
   if (c->generic_grid > c->generic_tiles) c->generic_grid = c->generic_tiles;
   c->max_partials = c->generic_grid;
-  if (c->fast.available && c->fast.grid > c->max_partials) c->max_partials = c->fast.grid;
+  if (c->fast.available && c->fast.grid * c->num_chunks > c->max_partials) c->max_partials = c->fast.grid * c->num_chunks;
   plan_fused(c);
   if (c->fused_available && c->fused_grid > c->max_partials) c->max_partials = c->fused_grid;
   rc = plan_big(c);
@@ -611,7 +624,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     p.d = c->d; p.seg_off = c->d_seg_off; p.blk_first_seg = c->d_blk_first_seg; p.blk_last_seg = c->d_blk_last_seg;
     p.rec_begin = c->d_rec_begin; p.set_first_block = c->d_set_first_block; p.records = c->d_records;
     p.flags = c->flags;
-    void* args[2] = {&c->tmap, &p};
+    void* args[2] = {&c->tmaps[0], &p};
     if (cudaLaunchKernel(c->seg_kernel, dim3(c->seg_grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
       cudaGetLastError();
       return ADACONS_ECUDA;
@@ -621,15 +634,21 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   } else if (aligned && c->fast.available) {
     int rc = encode_map(c, grads);
     if (rc != ADACONS_OK) return rc;
-    Pass1Params p;
-    p.N = N; p.num_tiles = c->fast.num_tiles; p.stages = c->fast.stages; p.stage_bytes = c->fast.stage_bytes;
-    p.partials = c->partials; p.flags = c->flags;
-    void* args[2] = {&c->tmap, &p};
-    if (cudaLaunchKernel(c->fast.kernel, dim3(c->fast.grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
-      cudaGetLastError();
-      return ADACONS_ECUDA;
+    for (int ch = 0; ch < c->num_chunks; ++ch) {      // one launch per column chunk of 2^30 (normally one)
+      const long long col0 = static_cast<long long>(ch) * kChunkCols;
+      const long long cols = c->d - col0 < kChunkCols ? c->d - col0 : kChunkCols;
+      Pass1Params p;
+      p.N = N; p.num_tiles = static_cast<int>((cols + c->fast.tile_cols - 1) / c->fast.tile_cols);
+      p.stages = c->fast.stages; p.stage_bytes = c->fast.stage_bytes;
+      p.partials = c->partials + static_cast<size_t>(ch) * c->fast.grid * 2 * N; p.flags = c->flags;
+      void* args[2] = {&c->tmaps[static_cast<size_t>(ch)], &p};
+      if (cudaLaunchKernel(c->fast.kernel, dim3(c->fast.grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
+        cudaGetLastError();
+        return ADACONS_ECUDA;
+      }
+      if (ch > 0) extra_launches += 1;
     }
-    num_partials = c->fast.grid;
+    num_partials = c->fast.grid * c->num_chunks;
     c->last_path = 1;
   } else if (aligned && c->big_available) {
     int rc = encode_map_big(c, grads);
@@ -797,7 +816,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       rc = plan_big(c);
       if (rc != ADACONS_OK) return rc;
       int need = c->generic_grid;
-      if (c->fast.available && c->fast.grid > need) need = c->fast.grid;
+      if (c->fast.available && c->fast.grid * c->num_chunks > need) need = c->fast.grid * c->num_chunks;
       if (c->fused_available && c->fused_grid > need) need = c->fused_grid;
       if (c->big_available && c->big_grid > need) need = c->big_grid;
       if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
@@ -1039,15 +1058,22 @@ extern "C" int adacons_stats_noalloc(const void* grads, int N, int64_t d, int dt
   if (aligned && plan.fast.available) {
     rc = encode_map(&plan, grads);
     if (rc != ADACONS_OK) return rc;
-    blocks = plan.fast.grid < ADACONS_NOALLOC_MAX_BLOCKS ? plan.fast.grid : ADACONS_NOALLOC_MAX_BLOCKS;
-    Pass1Params p;
-    p.N = N; p.num_tiles = plan.fast.num_tiles; p.stages = plan.fast.stages; p.stage_bytes = plan.fast.stage_bytes;
-    p.partials = partials; p.flags = flag;
-    void* args[2] = {&plan.tmap, &p};
-    if (cudaLaunchKernel(plan.fast.kernel, dim3(blocks), dim3(kThreads), args, plan.fast.smem_bytes, st) != cudaSuccess) {
-      cudaGetLastError();
-      return ADACONS_ECUDA;
+    int grid = plan.fast.grid;
+    if (grid * plan.num_chunks > ADACONS_NOALLOC_MAX_BLOCKS) grid = ADACONS_NOALLOC_MAX_BLOCKS / plan.num_chunks;
+    for (int ch = 0; ch < plan.num_chunks; ++ch) {      // column chunks of 2^30 (32-bit TMA coordinates)
+      const long long col0 = static_cast<long long>(ch) * kChunkCols;
+      const long long cols = d - col0 < kChunkCols ? d - col0 : kChunkCols;
+      Pass1Params p;
+      p.N = N; p.num_tiles = static_cast<int>((cols + plan.fast.tile_cols - 1) / plan.fast.tile_cols);
+      p.stages = plan.fast.stages; p.stage_bytes = plan.fast.stage_bytes;
+      p.partials = partials + static_cast<size_t>(ch) * grid * 2 * N; p.flags = flag;
+      void* args[2] = {&plan.tmaps[static_cast<size_t>(ch)], &p};
+      if (cudaLaunchKernel(plan.fast.kernel, dim3(grid), dim3(kThreads), args, plan.fast.smem_bytes, st) != cudaSuccess) {
+        cudaGetLastError();
+        return ADACONS_ECUDA;
+      }
     }
+    blocks = grid * plan.num_chunks;
   } else {
     const int tiles = static_cast<int>((d + kThreads * 4 - 1) / (kThreads * 4));
     blocks = nd->sms * 4;

@@ -857,3 +857,35 @@ def test_profile_and_info_getters(ac):
     assert h.get_option(ac.OPT_BETA) == 0.99 and h.get_option(ac.OPT_ROW_PITCH) == w.d
     with pytest.raises(ac.AdaConsError):
         h.info(99)
+
+
+def test_vector_longer_than_2_to_the_31(ac):
+    """d = 2^31 + 98,760 (N = 2, bf16, 8.6 GB): the TMA coordinates are 32-bit, so pass 1 walks the
+    vector in chunks of 2^30 columns.  Statistics from the oracle over all columns; output on
+    sampled columns including both sides of every chunk boundary and the very end."""
+    N, d = 2, (1 << 31) + 98_760
+    free, _ = torch.cuda.mem_get_info()
+    if free < 24e9:
+        pytest.skip("needs 24 GB of free device memory")
+    dev = torch.device("cuda:0")
+    w = wl.Workload("long", N, d, "bf16", 1, "gauss", seed=17)
+    G = wl.generate(w, 0, dev, row_block=64_000_000)
+    out = torch.empty(d, dtype=torch.bfloat16, device=dev)
+    h = ac.AdaCons(N, d, "bf16")
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 1 and h.status() == 0
+    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 5                      # three chunks of pass 1
+    p, q = streamed_statistics(G, slab=64_000_000, threads=4)
+    c = oc.coefficients(p, q, np.zeros(N), 0.99)
+    assert_coeffs(h.coeffs(ac.COEFF_P), p, "p")
+    assert_coeffs(h.coeffs(ac.COEFF_Q), q, "q")
+    assert_coeffs(h.coeffs(ac.COEFF_GAMMA), c["gamma"], "gamma")
+    gcpu = torch.Generator().manual_seed(9)
+    edges = torch.cat([torch.arange(b - 300, b + 300) for b in (1 << 30, 1 << 31)])
+    cols = torch.cat([torch.arange(0, 256), torch.arange(d - 256, d), edges, torch.randint(0, d, (100_000,), generator=gcpu)]).to(dev)
+    Gs = to_f64(G[:, cols])
+    psi = oc.combine(Gs, c["gamma"])
+    got = to_f64(out[cols])
+    tight = 1e-5 * (np.abs(c["gamma"])[:, None] * np.abs(Gs)).sum(0) + ULP["bf16"] * np.abs(psi) + 1e-45
+    assert np.all(np.abs(got - psi) <= tight)

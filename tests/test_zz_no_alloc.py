@@ -61,6 +61,26 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
     np.testing.assert_allclose(got[w.N:2 * w.N], q, rtol=COEFF_RTOL)
 
 
+def test_noalloc_vector_longer_than_one_tma_chunk():
+    """Beyond 2^30 columns pass 1 runs once per column chunk; the scratch then holds the partial
+    sums of every chunk.  Same comparison as above, N = 2, d = 2^30 + 32,768 (4.3 GB)."""
+    from paper_2411_03742_b200 import binding as ac
+    dev = torch.device("cuda:0")
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12e9:
+        pytest.skip("needs 12 GB of free device memory")
+    w = wl.Workload("nalong", 2, (1 << 30) + 32_768, "bf16", 1, "gauss", seed=12)
+    G = wl.generate(w, 0, dev, row_block=64_000_000)
+    pq = torch.zeros(4, dtype=torch.float64, device=dev)
+    for _ in range(2):
+        ac.stats_noalloc(G, pq)
+    torch.cuda.synchronize()
+    p, q = _reference(ac, G)
+    got = pq.cpu().numpy()
+    np.testing.assert_allclose(got[:2], p, rtol=COEFF_RTOL)
+    np.testing.assert_allclose(got[2:], q, rtol=COEFF_RTOL)
+
+
 def test_noalloc_rejects_sizes_beyond_its_scratch():
     from paper_2411_03742_b200 import binding as ac
     G = torch.zeros(ac.NOALLOC_MAX_N + 1, 256, device="cuda:0")
