@@ -185,6 +185,14 @@ int adacons_get_option(adacons_ctx *ctx, int key, double *value);
 int adacons_get_coeffs(adacons_ctx *ctx, int which, double *host, void *cuda_stream);
 
 /*
+ * The normaliser Z = sum_i u_i of Eq. 13 (u_i = a~_i / ||g_i||) of the most recent aggregate call,
+ * one double per coefficient set.  |Z| small against sum_i |u_i| means weights of both signs with
+ * large magnitude (an ill-conditioned step).  NaN after a non-finite input.  Synchronises
+ * `cuda_stream`.
+ */
+int adacons_get_normaliser(adacons_ctx *ctx, double *host_z, void *cuda_stream);
+
+/*
  * Momentum state for checkpoint / resume (Eq. 11): host_m receives / provides sets*N doubles,
  * slot k of a set = EMA of the k-th smallest coefficient; *step = number of aggregations since
  * the last reset.  Either pointer of get may be NULL.  Both synchronise `cuda_stream`.

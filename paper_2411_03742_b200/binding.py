@@ -63,6 +63,7 @@ def load_library() -> ctypes.CDLL:
         "adacons_set_option": [vp, i32, dbl],
         "adacons_get_option": [vp, i32, P(dbl)],
         "adacons_get_coeffs": [vp, i32, P(dbl), vp],
+        "adacons_get_normaliser": [vp, P(dbl), vp],
         "adacons_get_state": [vp, P(dbl), P(i64), vp],
         "adacons_set_state": [vp, P(dbl), i64, vp],
         "adacons_get_status": [vp, P(ctypes.c_uint32), vp],
@@ -183,6 +184,13 @@ class AdaCons:
         buf = np.empty((sets, self.N), dtype=np.float64)
         _check(self._lib.adacons_get_coeffs(self._ctx, which, buf.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
                                             _stream_handle(stream)), "adacons_get_coeffs")
+        return buf
+
+    def normaliser(self, stream=None) -> np.ndarray:
+        """Z = sum_i u_i of the last call, one value per coefficient set."""
+        buf = np.empty(self.info(INFO_COEFF_SETS), dtype=np.float64)
+        _check(self._lib.adacons_get_normaliser(self._ctx, buf.ctypes.data_as(ctypes.POINTER(ctypes.c_double)),
+                                                _stream_handle(stream)), "adacons_get_normaliser")
         return buf
 
     def state(self, stream=None):

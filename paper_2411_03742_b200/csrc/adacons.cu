@@ -68,6 +68,7 @@ struct adacons_ctx {
   double* coef = nullptr;         // [5][sets][N]
   float* gamma_f32 = nullptr;     // [sets][N]
   double* m = nullptr;            // [sets][N]
+  double* z = nullptr;            // [sets]
   uint32_t* flags = nullptr;
   long long* step = nullptr;
   void* staging = nullptr;        // adacons_aggregate_host: N*pitch + d elements
@@ -343,20 +344,20 @@ struct DeviceGuard {   // make the context's device current for the duration of 
 };
 
 int alloc_sets(adacons_ctx* c) {   // (re)allocate everything whose size depends on sets()
-  cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
-  c->coef = nullptr; c->gamma_f32 = nullptr; c->m = nullptr;
+  cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m); cudaFree(c->z);
+  c->coef = nullptr; c->gamma_f32 = nullptr; c->m = nullptr; c->z = nullptr;
   const size_t sets = static_cast<size_t>(c->sets());
   const size_t N = static_cast<size_t>(c->N);
   const size_t b_coef = 5 * sets * N * sizeof(double);
   const size_t b_gam = sets * N * sizeof(float);
   const size_t b_m = sets * N * sizeof(double);
   if (cudaMalloc(&c->coef, b_coef) != cudaSuccess || cudaMalloc(&c->gamma_f32, b_gam) != cudaSuccess ||
-      cudaMalloc(&c->m, b_m) != cudaSuccess) {
+      cudaMalloc(&c->m, b_m) != cudaSuccess || cudaMalloc(&c->z, sets * sizeof(double)) != cudaSuccess) {
     cudaGetLastError();
     return ADACONS_ENOMEM;
   }
   if (cudaMemset(c->coef, 0, b_coef) != cudaSuccess || cudaMemset(c->gamma_f32, 0, b_gam) != cudaSuccess ||
-      cudaMemset(c->m, 0, b_m) != cudaSuccess)
+      cudaMemset(c->m, 0, b_m) != cudaSuccess || cudaMemset(c->z, 0, sets * sizeof(double)) != cudaSuccess)
     return ADACONS_ECUDA;
   const size_t b_part = static_cast<size_t>(c->max_partials) * 2 * N * sizeof(float);
   c->scratch_bytes = b_part + b_coef + b_gam + b_m + sizeof(uint32_t) + sizeof(long long) + c->seg_bytes;
@@ -554,7 +555,7 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
 int adacons_destroy(adacons_ctx* c) {
   if (c == nullptr) return ADACONS_OK;
   DeviceGuard g(c->device);
-  cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m);
+  cudaFree(c->partials); cudaFree(c->coef); cudaFree(c->gamma_f32); cudaFree(c->m); cudaFree(c->z);
   cudaFree(c->flags); cudaFree(c->step); cudaFree(c->staging); cudaFree(c->d_barrier); cudaFree(c->d_colsum);
   free_seg_plan(c);
   if (c->prof_ready)
@@ -600,7 +601,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     q.N = N; q.num_partials = c->fused_grid; q.sets = 1; q.beta = c->beta;
     q.momentum = c->momentum; q.sorted = c->sorted; q.normalize = c->normalize;
     q.partials = c->partials; q.rec_begin = nullptr; q.rec_count = nullptr;
-    q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.flags = c->flags; q.step = c->step;
+    q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.z = c->z; q.flags = c->flags; q.step = c->step;
     const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&fused_small_kernel<0>)
                                             : reinterpret_cast<const void*>(&fused_small_kernel<1>);
     void* args[1] = {&f};
@@ -691,7 +692,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   q.partials = seg ? c->d_records : c->partials;
   q.rec_begin = seg ? c->d_rec_begin : nullptr;
   q.rec_count = seg ? c->d_rec_count : nullptr;
-  q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m;
+  q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.z = c->z;
   q.flags = c->flags; q.step = c->step;
   int cthreads = 1024;
   if (seg) { cthreads = ((2 * N + 31) / 32) * 32; if (cthreads > 1024) cthreads = 1024; }
@@ -873,6 +874,16 @@ int adacons_get_coeffs(adacons_ctx* c, int which, double* host, void* cuda_strea
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t n = static_cast<size_t>(c->sets()) * c->N;
   if (cudaMemcpyAsync(host, c->coef + static_cast<size_t>(which) * n, n * sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+  return ADACONS_OK;
+}
+
+int adacons_get_normaliser(adacons_ctx* c, double* host_z, void* cuda_stream) {
+  if (c == nullptr || host_z == nullptr) return ADACONS_EINVAL;
+  DeviceGuard guard(c->device);
+  if (!guard.ok) return ADACONS_ECUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(host_z, c->z, static_cast<size_t>(c->sets()) * sizeof(double), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
   return ADACONS_OK;
 }

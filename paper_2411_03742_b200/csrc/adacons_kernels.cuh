@@ -732,6 +732,7 @@ struct CoeffParams {
   double* coef;          // [5][sets][N]: a, a~, gamma, p, q   (enum adacons_coeff order)
   float* gamma_f32;      // [sets][N]   weights as pass 2 reads them
   double* m;             // [sets][N]   momentum state, in place
+  double* z;             // [sets]      normaliser Z = sum_i u_i of the last call (NaN if not computed)
   uint32_t* flags;       // device status word (OR)
   long long* step;       // aggregation counter
 };
@@ -803,6 +804,7 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
     }
     if (i == 0) {
       atomicOr(prm.flags, flags | kFlagNonfinite);
+      prm.z[set] = __longlong_as_double(0x7ff8000000000000ll);
       if (set == 0) *prm.step += 1;
     }
     return;
@@ -832,6 +834,7 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
     double Z = 0.0, A = 0.0;
     for (int j = 0; j < N; ++j) { Z += sh_u[j]; A += fabs(sh_u[j]); }
     sh_Z = Z;
+    prm.z[set] = Z;
     sh_uniform = 0;
     if (prm.normalize) {
       if (!isfinite(Z) || fabs(Z) <= 1e-12 * A) { sh_uniform = 1; flags |= kFlagDegenerateZ; }

@@ -132,6 +132,10 @@ def run_case(ac, w, steps, *, beta=0.99, options=None, oracle_kw=None, offsets=N
         assert_coeffs_by_set(h.coeffs(ac.COEFF_A), res["a"], f"{w.name} step {t} a")
         assert_coeffs_by_set(h.coeffs(ac.COEFF_A_TILDE), res["a_tilde"], f"{w.name} step {t} a~")
         assert_coeffs_by_set(h.coeffs(ac.COEFF_GAMMA), res["gamma"], f"{w.name} step {t} gamma")
+        if oracle_kw.get("normalize", True):
+            zg, zo = h.normaliser(), res["Z"]
+            ok = np.isfinite(zo)
+            assert np.all(np.abs(zg[ok] - zo[ok]) <= COEFF_RTOL * np.abs(res["u"][ok]).sum(axis=1) + 1e-300), "Z"
         m, step = h.state()
         assert step == t + 1
         assert_coeffs_by_set(m, res["m"], f"{w.name} step {t} m")
