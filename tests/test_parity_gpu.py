@@ -893,3 +893,63 @@ def test_vector_longer_than_2_to_the_31(ac):
     got = to_f64(out[cols])
     tight = 1e-5 * (np.abs(c["gamma"])[:, None] * np.abs(Gs)).sum(0) + ULP["bf16"] * np.abs(psi) + 1e-45
     assert np.all(np.abs(got - psi) <= tight)
+
+
+# ---- seeded random sweep over shapes, types, pitches, segment layouts and paths -------------------
+def _random_case(seed):
+    r = np.random.default_rng(seed)
+    dtype = ["f32", "bf16"][int(r.integers(2))]
+    vec = 4 if dtype == "f32" else 8
+    N = int(r.choice([1, 2, 3, 5, 8, 9, 16, 17, 31, 32, 33, 48, 64, 65, 70, 130]))
+    d = int(r.choice([r.integers(1, 64), r.integers(64, 5_000), r.integers(5_000, 120_000), r.integers(120_000, 400_000)]))
+    pad = int(r.choice([0, 0, 1, vec, 3 * vec + 1]))
+    pitch = d + pad
+    if r.random() < 0.7:                              # most cases: a 16-byte pitch (fast paths)
+        pitch = (pitch + vec - 1) // vec * vec
+    S = int(r.choice([1, 1, 2, 5, 40]))
+    cuts = np.sort(r.integers(0, d + 1, size=S - 1)) if S > 1 else np.array([], dtype=np.int64)
+    offsets = [0] + [int(c) for c in cuts] + [d]
+    fused = bool(r.random() < 0.5)
+    aligned = (pitch * (4 if dtype == "f32" else 2)) % 16 == 0
+    per_segment = bool(S > 1 and aligned and N <= 64 and r.random() < 0.7)
+    return dict(N=N, d=d, dtype=dtype, pitch=pitch, offsets=offsets, fused=fused, per_segment=per_segment,
+                beta=float(r.choice([0.0, 0.5, 0.99])), kind=str(r.choice(["gauss", "gauss_outlier", "student_flip"])))
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_shapes(ac, seed):
+    c = _random_case(1000 + seed)
+    dev = torch.device("cuda:0")
+    tdt = torch.float32 if c["dtype"] == "f32" else torch.bfloat16
+    N, d, pitch = c["N"], c["d"], c["pitch"]
+    w = wl.Workload(f"rnd{seed}", N, d, c["dtype"], 2, c["kind"], seed=seed)
+    buf = torch.full((N, pitch), float("nan"), dtype=tdt, device=dev)
+    obuf = torch.full((d + 32,), 7.0, dtype=tdt, device=dev)
+    out = obuf[:d]
+    h = ac.AdaCons(N, d, c["dtype"], seg_offsets=c["offsets"])
+    h.set_option(ac.OPT_ROW_PITCH, pitch)
+    h.set_option(ac.OPT_FUSED_SMALL, 1 if c["fused"] else 0)
+    h.set_option(ac.OPT_BETA, c["beta"])
+    okw = {}
+    if c["per_segment"]:
+        h.set_option(ac.OPT_PER_SEGMENT, 1)
+        okw = dict(seg_offsets=c["offsets"], per_segment=True)
+    orc = oc.AdaConsOracle(N, d, beta=c["beta"], **okw)
+    flags = 0
+    for t in range(2):
+        G = wl.generate(w, t, dev)
+        buf[:, :d] = G
+        h.aggregate(buf, out)
+        torch.cuda.synchronize()
+        G64 = to_f64(G)
+        res = oracle_step_with_kernel_ranks(orc, G64, c["dtype"], h.coeffs(ac.COEFF_A))
+        flags |= int(np.bitwise_or.reduce(res["flags"]))
+        assert h.status() == flags, c
+        well = np.abs(res["Z"]) > 1e-4 * np.abs(res["u"]).sum(axis=1)       # sets with a sane normaliser
+        for s_ in np.nonzero(well)[0]:
+            assert_coeffs(h.coeffs(ac.COEFF_GAMMA)[s_], res["gamma"][s_], f"gamma set {s_} {c}")
+        assert_coeffs_by_set(h.coeffs(ac.COEFF_A), res["a"], f"a {c}")
+        assert_coeffs_by_set(h.state()[0], res["m"], f"m {c}")
+        if well.all():
+            assert_output(out, res, G64, c["dtype"], f"out {c}", c["offsets"] if c["per_segment"] else None)
+        assert bool((obuf[d:] == 7.0).all()), "wrote past the end of out"
