@@ -185,7 +185,6 @@ int plan_fast(adacons_ctx* c) {
   if ((c->pitch * c->elem_bytes) % 16 != 0) return ADACONS_OK;
   if (c->encode == nullptr) return ADACONS_OK;
   c->num_chunks = static_cast<int>((c->d + kChunkCols - 1) / kChunkCols);
-  c->tmaps.resize(static_cast<size_t>(c->num_chunks));
   c->tmap_for = nullptr;
   const long long first_cols = c->d < kChunkCols ? c->d : kChunkCols;   // columns of the first (largest) chunk
   int WR, NR;
@@ -307,22 +306,28 @@ int plan_fused(adacons_ctx* c) {
   return ADACONS_OK;
 }
 
+// Tensor map of column chunk `ch` (columns [ch * 2^30, ...)) of the matrix at `grads`.
+int encode_chunk_map(const adacons_ctx* c, const void* grads, int ch, CUtensorMap* out) {
+  const long long col0 = static_cast<long long>(ch) * kChunkCols;
+  const long long cols = c->d - col0 < kChunkCols ? c->d - col0 : kChunkCols;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(c->N)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(c->N)};
+  const cuuint32_t estr[2] = {1, 1};
+  void* base = const_cast<unsigned char*>(static_cast<const unsigned char*>(grads)) + col0 * c->elem_bytes;
+  const CUresult r = c->encode(out, c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                               2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ADACONS_OK : ADACONS_ECUDA;
+}
+
+// All chunk maps of a context (its vector was sized when the plan was made).
 int encode_map(adacons_ctx* c, const void* grads) {
   if (c->tmap_for == grads) return ADACONS_OK;
   for (int ch = 0; ch < c->num_chunks; ++ch) {
-    const long long col0 = static_cast<long long>(ch) * kChunkCols;
-    const long long cols = c->d - col0 < kChunkCols ? c->d - col0 : kChunkCols;
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(c->N)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
-    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(c->N)};
-    const cuuint32_t estr[2] = {1, 1};
-    void* base = const_cast<unsigned char*>(static_cast<const unsigned char*>(grads)) + col0 * c->elem_bytes;
-    const CUresult r = c->encode(&c->tmaps[static_cast<size_t>(ch)],
-                                 c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                                 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+    const int rc = encode_chunk_map(c, grads, ch, &c->tmaps[static_cast<size_t>(ch)]);
+    if (rc != ADACONS_OK) return rc;
   }
   c->tmap_for = grads;
   return ADACONS_OK;
@@ -515,6 +520,7 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
 
   int rc = plan_fast(c);
   if (rc != ADACONS_OK) { delete c; return rc; }
+  c->tmaps.resize(static_cast<size_t>(c->num_chunks));
 
   // generic path: always available
   c->generic_tiles = static_cast<int>((d + kThreads * 4 - 1) / (kThreads * 4));
@@ -812,6 +818,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       c->tmap_for = nullptr;
       int rc = plan_fast(c);
       if (rc != ADACONS_OK) return rc;
+      c->tmaps.resize(static_cast<size_t>(c->num_chunks));
       plan_fused(c);
       c->tmap_big_for = nullptr;
       rc = plan_big(c);
@@ -1067,8 +1074,12 @@ extern "C" int adacons_stats_noalloc(const void* grads, int N, int64_t d, int dt
   const bool aligned = (reinterpret_cast<uintptr_t>(grads) % 16 == 0) && ((d * plan.elem_bytes) % 16 == 0);
   int blocks;
   if (aligned && plan.fast.available) {
-    rc = encode_map(&plan, grads);
-    if (rc != ADACONS_OK) return rc;
+    CUtensorMap maps[2];                                // d < 2^31: at most two chunks; nothing is allocated
+    if (plan.num_chunks > 2) return ADACONS_EINVAL;
+    for (int ch = 0; ch < plan.num_chunks; ++ch) {
+      rc = encode_chunk_map(&plan, grads, ch, &maps[ch]);
+      if (rc != ADACONS_OK) return rc;
+    }
     int grid = plan.fast.grid;
     if (grid * plan.num_chunks > ADACONS_NOALLOC_MAX_BLOCKS) grid = ADACONS_NOALLOC_MAX_BLOCKS / plan.num_chunks;
     for (int ch = 0; ch < plan.num_chunks; ++ch) {      // column chunks of 2^30 (32-bit TMA coordinates)
@@ -1078,7 +1089,7 @@ extern "C" int adacons_stats_noalloc(const void* grads, int N, int64_t d, int dt
       p.N = N; p.num_tiles = static_cast<int>((cols + plan.fast.tile_cols - 1) / plan.fast.tile_cols);
       p.stages = plan.fast.stages; p.stage_bytes = plan.fast.stage_bytes;
       p.partials = partials + static_cast<size_t>(ch) * grid * 2 * N; p.flags = flag;
-      void* args[2] = {&plan.tmaps[static_cast<size_t>(ch)], &p};
+      void* args[2] = {&maps[ch], &p};
       if (cudaLaunchKernel(plan.fast.kernel, dim3(grid), dim3(kThreads), args, plan.fast.smem_bytes, st) != cudaSuccess) {
         cudaGetLastError();
         return ADACONS_ECUDA;
