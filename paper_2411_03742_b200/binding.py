@@ -112,6 +112,34 @@ def stats_noalloc(grads, pq_out, stream=None) -> None:
            "adacons_stats_noalloc")
 
 
+def check_tensors(N: int, d: int, dtype: str, pitch: int, grads, out, want_cuda: bool = True) -> None:
+    """Raise ValueError unless `grads` is an N x d matrix of `dtype` whose rows are `pitch` elements
+    apart with unit column stride and `out` is a contiguous d-vector of the same type (and, with
+    want_cuda, both live on one CUDA device).  The library trusts its pointers; this is the guard."""
+    import torch
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16}[dtype]
+    if grads.dtype != tdt or out.dtype != tdt:
+        raise ValueError(f"expected {tdt} tensors, got grads {grads.dtype} and out {out.dtype}")
+    if grads.dim() != 2 or tuple(grads.shape) != (N, d):
+        raise ValueError(f"grads must have shape ({N}, {d}), got {tuple(grads.shape)}")
+    if out.dim() != 1 or out.shape[0] != d:
+        raise ValueError(f"out must have shape ({d},), got {tuple(out.shape)}")
+    if d > 1 and grads.stride(1) != 1:
+        raise ValueError("grads must have unit stride along the gradient dimension")
+    if N > 1 and grads.stride(0) != pitch:
+        raise ValueError(f"rows of grads are {grads.stride(0)} elements apart, the context expects {pitch} "
+                         "(set OPT_ROW_PITCH or pass a contiguous matrix)")
+    if d > 1 and out.stride(0) != 1:
+        raise ValueError("out must be contiguous")
+    if want_cuda:
+        if not (grads.is_cuda and out.is_cuda):
+            raise ValueError("grads and out must be CUDA tensors (use aggregate_host for host memory)")
+        if grads.device != out.device:
+            raise ValueError("grads and out must be on the same device")
+    elif grads.is_cuda or out.is_cuda:
+        raise ValueError("aggregate_host takes host tensors")
+
+
 class AdaCons:
     """One aggregation context: N workers, gradients of d elements of `dtype` ("f32"/"bf16").
 
@@ -151,13 +179,17 @@ class AdaCons:
 
     # -- hot path ---------------------------------------------------------------------------
     def aggregate(self, grads, out, stream=None) -> None:
+        check_tensors(self.N, self.d, self.dtype, int(self.get_option(OPT_ROW_PITCH)), grads, out)
         self.aggregate_ptr(grads.data_ptr(), out.data_ptr(), _stream_handle(stream))
 
     def aggregate_ptr(self, grads_ptr: int, out_ptr: int, stream_handle: int) -> None:
         _check(self._lib.adacons_aggregate(self._ctx, grads_ptr, out_ptr, stream_handle), "adacons_aggregate")
 
     def aggregate_host(self, host_grads, host_out, stream=None) -> None:
-        """host_grads / host_out: CPU tensors or numpy arrays (contiguous)."""
+        """host_grads / host_out: CPU tensors (checked) or numpy arrays (contiguous, unchecked)."""
+        if hasattr(host_grads, "data_ptr") and hasattr(host_out, "data_ptr"):
+            check_tensors(self.N, self.d, self.dtype, int(self.get_option(OPT_ROW_PITCH)), host_grads, host_out,
+                          want_cuda=False)
         gp = host_grads.data_ptr() if hasattr(host_grads, "data_ptr") else host_grads.ctypes.data
         op = host_out.data_ptr() if hasattr(host_out, "data_ptr") else host_out.ctypes.data
         _check(self._lib.adacons_aggregate_host(self._ctx, gp, op, _stream_handle(stream)), "adacons_aggregate_host")

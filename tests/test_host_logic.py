@@ -75,3 +75,21 @@ def test_product_does_not_import_the_oracle():
     for f in os.listdir(os.path.join(ROOT, "oracle")):
         if f.endswith(".py"):
             assert "paper_2411_03742_b200" not in open(os.path.join(ROOT, "oracle", f)).read(), f
+
+
+def test_binding_rejects_tensors_that_do_not_match_the_context():
+    """The kernels trust their pointers, so the binding checks shape, type, strides and device."""
+    import torch
+    from paper_2411_03742_b200.binding import check_tensors
+    G, out = torch.zeros(4, 100), torch.zeros(100)
+    check_tensors(4, 100, "f32", 100, G, out, want_cuda=False)
+    for bad_G, bad_out, pitch in [(torch.zeros(4, 99), out, 100), (torch.zeros(5, 100), out, 100),
+                                  (G.to(torch.bfloat16), out, 100), (G, torch.zeros(101), 100),
+                                  (torch.zeros(100, 4).t(), out, 100), (torch.zeros(4, 200)[:, ::2], out, 100),
+                                  (G, torch.zeros(200)[::2], 100), (G, out, 104), (G, out.double(), 100)]:
+        with pytest.raises(ValueError):
+            check_tensors(4, 100, "f32", pitch, bad_G, bad_out, want_cuda=False)
+    padded = torch.zeros(4, 104)[:, :100]
+    check_tensors(4, 100, "f32", 104, padded, out, want_cuda=False)          # padded rows are fine
+    with pytest.raises(ValueError):
+        check_tensors(4, 100, "f32", 100, G, out, want_cuda=True)             # host tensors on the device path

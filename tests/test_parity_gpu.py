@@ -727,7 +727,7 @@ def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=
     for t in range(steps):
         G = wl.generate(w, t, dev)
         buf[:, :d] = G
-        h.aggregate(buf, out)
+        h.aggregate(buf[:, :d], out)
         torch.cuda.synchronize()
         if expect_path is not None:
             assert h.info(ac.INFO_LAST_PATH) == expect_path
@@ -771,7 +771,7 @@ def test_host_entry_point_with_padded_rows(ac):
     out = torch.empty(d, dtype=torch.bfloat16).pin_memory()
     h = ac.AdaCons(N, d, "bf16")
     h.set_option(ac.OPT_ROW_PITCH, pitch)
-    h.aggregate_host(buf, out)
+    h.aggregate_host(buf[:, :d], out)
     res = oc.AdaConsOracle(N, d).step(to_f64(G), storage="bf16")
     assert_coeffs(h.coeffs(), res["gamma"], "gamma host padded")
     assert_output(out, res, to_f64(G), "bf16", "host padded")
@@ -940,7 +940,7 @@ def test_random_shapes(ac, seed):
     for t in range(2):
         G = wl.generate(w, t, dev)
         buf[:, :d] = G
-        h.aggregate(buf, out)
+        h.aggregate(buf[:, :d], out)
         torch.cuda.synchronize()
         G64 = to_f64(G)
         res = oracle_step_with_kernel_ranks(orc, G64, c["dtype"], h.coeffs(ac.COEFF_A))
