@@ -158,6 +158,8 @@ class AdaCons:
         else:
             rc = self._lib.adacons_create(ctypes.byref(self._ctx), N, d, dt, None, 0)
         _check(rc, "adacons_create")
+        self._pitch = self.d          # mirrors OPT_ROW_PITCH
+        self._checked = None          # signature of the last tensor layout that passed check_tensors
 
     # -- lifetime ---------------------------------------------------------------------------
     def close(self) -> None:
@@ -179,7 +181,11 @@ class AdaCons:
 
     # -- hot path ---------------------------------------------------------------------------
     def aggregate(self, grads, out, stream=None) -> None:
-        check_tensors(self.N, self.d, self.dtype, int(self.get_option(OPT_ROW_PITCH)), grads, out)
+        # the full check runs once per distinct layout; repeats are recognised by their signature
+        sig = (grads.dtype, grads.shape, grads.stride(), grads.device, out.dtype, out.shape, out.stride(), out.device)
+        if sig != self._checked:
+            check_tensors(self.N, self.d, self.dtype, self._pitch, grads, out)
+            self._checked = sig
         self.aggregate_ptr(grads.data_ptr(), out.data_ptr(), _stream_handle(stream))
 
     def aggregate_ptr(self, grads_ptr: int, out_ptr: int, stream_handle: int) -> None:
@@ -188,8 +194,7 @@ class AdaCons:
     def aggregate_host(self, host_grads, host_out, stream=None) -> None:
         """host_grads / host_out: CPU tensors (checked) or numpy arrays (contiguous, unchecked)."""
         if hasattr(host_grads, "data_ptr") and hasattr(host_out, "data_ptr"):
-            check_tensors(self.N, self.d, self.dtype, int(self.get_option(OPT_ROW_PITCH)), host_grads, host_out,
-                          want_cuda=False)
+            check_tensors(self.N, self.d, self.dtype, self._pitch, host_grads, host_out, want_cuda=False)
         gp = host_grads.data_ptr() if hasattr(host_grads, "data_ptr") else host_grads.ctypes.data
         op = host_out.data_ptr() if hasattr(host_out, "data_ptr") else host_out.ctypes.data
         _check(self._lib.adacons_aggregate_host(self._ctx, gp, op, _stream_handle(stream)), "adacons_aggregate_host")
@@ -200,6 +205,9 @@ class AdaCons:
     # -- options, state, diagnostics -----------------------------------------------------------
     def set_option(self, key: int, value: float) -> None:
         _check(self._lib.adacons_set_option(self._ctx, key, float(value)), "adacons_set_option")
+        if key == OPT_ROW_PITCH:
+            self._pitch = int(value)
+            self._checked = None
 
     def get_option(self, key: int) -> float:
         v = ctypes.c_double()
