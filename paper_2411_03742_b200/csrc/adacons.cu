@@ -199,7 +199,8 @@ int plan_fast(adacons_ctx* c) {
   f.num_tiles = static_cast<int>((first_cols + f.tile_cols - 1) / f.tile_cols);
   f.stage_bytes = static_cast<uint32_t>(WC) * N * kBoxRowBytes;
   const size_t xch = WR > 1 ? static_cast<size_t>(2) * WR * WC * 32 * vec * sizeof(float) : 0;
-  const size_t fixed = xch + static_cast<size_t>(kWarps) * NR * 2 * sizeof(float);
+  const size_t fixed = xch + static_cast<size_t>(kWarps) * NR * 2 * sizeof(float) +
+                       static_cast<size_t>(2) * NR * kThreads * sizeof(float);   // exchange, block reduce, second-level sums
   const size_t budget = 110 * 1024;   // two blocks per SM
   int stages = static_cast<int>((budget - fixed - 64) / f.stage_bytes);
   if (stages > 8) stages = 8;
@@ -233,7 +234,8 @@ int plan_big(adacons_ctx* c) {
   c->big_tiles = static_cast<int>((c->d + tile_cols - 1) / tile_cols);
   const uint32_t stage_bytes = 64u * kBoxRowBytes;
   const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
-  const size_t fixed = static_cast<size_t>(2) * 8 * 32 * vec * sizeof(float) + static_cast<size_t>(kWarps) * 8 * 2 * sizeof(float);
+  const size_t fixed = static_cast<size_t>(2) * 8 * 32 * vec * sizeof(float) + static_cast<size_t>(kWarps) * 8 * 2 * sizeof(float) +
+                       static_cast<size_t>(2) * 8 * kThreads * sizeof(float);
   c->big_stages = 2;
   c->big_smem = static_cast<size_t>(c->big_stages) * stage_bytes + fixed + static_cast<size_t>(c->big_stages) * 8;
   const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_dot_kernel<0>)

@@ -141,12 +141,14 @@ struct P1 {
   static constexpr int kXchOne = WR * WC * 32 * VEC;             // floats of one exchange buffer
   static constexpr int kXchFloats = (WR > 1) ? 2 * kXchOne : 0;
   static constexpr int kRedFloats = kWarps * NR * 2;
+  static constexpr int kOuterFloats = 2 * NR * kThreads;        // second-level accumulators, [2][NR][thread]
 };
 
 struct P1Smem {            // carve-up of the dynamic shared memory of both pass-1 kernels
   unsigned char* stage_base;
   float* xch;
   float* red;
+  float* outer;
   uint64_t* full;
 };
 template <class C>
@@ -155,7 +157,8 @@ __device__ __forceinline__ P1Smem p1_carve(unsigned char* raw, int stages, uint3
   s.stage_base = raw;
   s.xch = reinterpret_cast<float*>(raw + static_cast<size_t>(stages) * stage_bytes);
   s.red = s.xch + C::kXchFloats;
-  s.full = reinterpret_cast<uint64_t*>(s.red + C::kRedFloats);
+  s.outer = s.red + C::kRedFloats;
+  s.full = reinterpret_cast<uint64_t*>(s.outer + C::kOuterFloats);
   return s;
 }
 
@@ -259,16 +262,40 @@ __device__ __forceinline__ void p1_accumulate_masked(const uint4 (&v)[C::NR], co
       qacc[j] = __ffma2_rn(x, x, qacc[j]);
     }
 }
-// Block partial of the accumulators: lanes (fixed xor tree), then the WC warps that share a row
-// (fixed order).  dst_p[0..rows) = N p_i (un-divided), dst_q[0..rows) = q_i.  Contains two
-// barriers; the accumulators are reset.
+// Two-level accumulation.  A thread's fp32 sums are folded into second-level accumulators (in
+// shared memory, one slot per thread and row) every kFoldTiles tiles.  Long fp32 sums of squares of
+// bf16 values are not merely noisy but biased: such squares have few, structured significant bits,
+// so once the running sum is large they round down more often than up (q was 9e-6 low after 18k
+// terms per accumulator at d = 340M).  Kept below ~128 terms the first level is exact for typical
+// data, and the second level adds full-width values, whose rounding is unbiased.
+constexpr int kFoldTiles = 32;
 template <class C>
-__device__ __forceinline__ void p1_block_store(float2 (&pacc)[C::NR], float2 (&qacc)[C::NR], float* red,
-                                               float* dst_p, float* dst_q, int rows) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+__device__ __forceinline__ void p1_outer_clear(float* outer) {
+#pragma unroll
+  for (int j = 0; j < 2 * C::NR; ++j) outer[j * kThreads + threadIdx.x] = 0.f;
+}
+template <class C>
+__device__ __forceinline__ void p1_fold(float2 (&pacc)[C::NR], float2 (&qacc)[C::NR], float* outer) {
 #pragma unroll
   for (int j = 0; j < C::NR; ++j) {
-    float p = pacc[j].x + pacc[j].y, q = qacc[j].x + qacc[j].y;
+    outer[j * kThreads + threadIdx.x] += pacc[j].x + pacc[j].y;
+    outer[(C::NR + j) * kThreads + threadIdx.x] += qacc[j].x + qacc[j].y;
+    pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  }
+}
+// Block partial of the accumulators (both levels): lanes (fixed xor tree), then the WC warps that
+// share a row (fixed order).  dst_p[0..rows) = N p_i (un-divided), dst_q[0..rows) = q_i.  Contains
+// two barriers; both levels are reset.
+template <class C>
+__device__ __forceinline__ void p1_block_store(float2 (&pacc)[C::NR], float2 (&qacc)[C::NR], float* outer, float* red,
+                                               float* dst_p, float* dst_q, int rows) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  p1_fold<C>(pacc, qacc, outer);
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j) {
+    float p = outer[j * kThreads + tid], q = outer[(C::NR + j) * kThreads + tid];
+    outer[j * kThreads + tid] = 0.f;
+    outer[(C::NR + j) * kThreads + tid] = 0.f;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       p += __shfl_xor_sync(0xffffffffu, p, o);
@@ -278,7 +305,6 @@ __device__ __forceinline__ void p1_block_store(float2 (&pacc)[C::NR], float2 (&q
       red[(warp * C::NR + j) * 2 + 0] = p;
       red[(warp * C::NR + j) * 2 + 1] = q;
     }
-    pacc[j] = qacc[j] = make_float2(0.f, 0.f);
   }
   __syncthreads();
   if (tid < rows) {
@@ -353,6 +379,7 @@ pass1_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm
   float2 pacc[NR], qacc[NR];
 #pragma unroll
   for (int j = 0; j < NR; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  p1_outer_clear<C>(sm.outer);
 
   int s = 0;
   uint32_t parity = 0;
@@ -379,6 +406,7 @@ pass1_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm
     }
     p1_xch_finish<C>(sm.xch, k, sp, cw, lane);
     p1_accumulate<DT, C>(v, sp, pacc, qacc);
+    if ((k & (kFoldTiles - 1)) == kFoldTiles - 1) p1_fold<C>(pacc, qacc, sm.outer);
     if (++s == prm.stages) { s = 0; parity ^= 1u; }
   }
 
@@ -388,7 +416,7 @@ pass1_tma_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm
     if (tid < 2 * N) dst[tid] = 0.f;
     return;
   }
-  p1_block_store<C>(pacc, qacc, sm.red, dst, dst + N, N);
+  p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst, dst + N, N);
 }
 
 // ---- pass 1 for more than 64 workers: column sums first, then dot products per 64-row chunk -----
@@ -478,6 +506,7 @@ pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams 
   float2 pacc[8], qacc[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  p1_outer_clear<C>(sm.outer);
   int s = 0;
   uint32_t parity = 0;
   for (int k = 0; k < my_tiles; ++k) {
@@ -506,6 +535,7 @@ pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams 
       issued = k + prm.stages + 1;
     }
     p1_accumulate<DT, C>(v, sp, pacc, qacc);
+    if ((k & (kFoldTiles - 1)) == kFoldTiles - 1) p1_fold<C>(pacc, qacc, sm.outer);
     if (++s == prm.stages) { s = 0; parity ^= 1u; }
   }
   float* dst = prm.partials + static_cast<size_t>(blockIdx.x) * 2 * prm.N;
@@ -514,7 +544,7 @@ pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams 
     if (tid < prm.rows) { dst[prm.r0 + tid] = 0.f; dst[prm.N + prm.r0 + tid] = 0.f; }
     return;
   }
-  p1_block_store<C>(pacc, qacc, sm.red, dst + prm.r0, dst + prm.N + prm.r0, prm.rows);
+  p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst + prm.r0, dst + prm.N + prm.r0, prm.rows);
 }
 
 // ---- per-segment ("layer-wise") pass 1 ----------------------------------------------------------
@@ -582,6 +612,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
   float2 pacc[NR], qacc[NR];
 #pragma unroll
   for (int j = 0; j < NR; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  p1_outer_clear<C>(sm.outer);
 
   int seg = prm.blk_first_seg[b];
   const int last_seg = prm.blk_last_seg[b];
@@ -626,7 +657,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
         const long long hi = seg_end < tile_hi ? seg_end : tile_hi;
         if (hi > lo) p1_accumulate_masked<DT, C>(v, sp, pacc, qacc, col0, lo, hi);
         if (seg_end <= tile_hi && seg < last_seg) {
-          p1_block_store<C>(pacc, qacc, sm.red, record(seg), record(seg) + N, N);
+          p1_block_store<C>(pacc, qacc, sm.outer, sm.red, record(seg), record(seg) + N, N);
           ++seg;
           seg_end = prm.seg_off[seg + 1];
           lo = hi;                                              // empty segments fall through here
@@ -635,6 +666,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
         }
       }
     }
+    if ((k & (kFoldTiles - 1)) == kFoldTiles - 1) p1_fold<C>(pacc, qacc, sm.outer);
     if (++s == prm.stages) { s = 0; parity ^= 1u; }
   }
 
@@ -642,7 +674,7 @@ pass1_seg_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1SegParams 
     if (tid == 0) p1_drain_after_timeout(sm.full, prm.stages, issued, prm.flags);
     return;   // the records keep whatever they held; the status word says the result is invalid
   }
-  p1_block_store<C>(pacc, qacc, sm.red, record(seg), record(seg) + N, N);
+  p1_block_store<C>(pacc, qacc, sm.outer, sm.red, record(seg), record(seg) + N, N);
 }
 
 // ----------------------------------------------------------------------------------------------
