@@ -36,7 +36,7 @@ CPU_BASELINE_COLUMNS = 4_000_000       # cpu_baseline leg of the CUDA arm: 3 ste
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/, as a multiple of the algorithmic bytes of that kernel (None = no capture for the
 # current kernel).
-NCU_TRAFFIC_RATIO = {"pass1": 1.0023, "pass2": 0.9881}
+NCU_TRAFFIC_RATIO = {"pass1": 1.0015, "pass2": 0.9876}
 
 
 def parse_args(argv=None):
