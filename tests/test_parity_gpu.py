@@ -973,3 +973,24 @@ def test_random_shapes(ac, seed):
         if well_so_far.all():
             assert_output(out, res, G64, c["dtype"], f"out {c}", c["offsets"] if c["per_segment"] else None)
         assert bool((obuf[d:] == 7.0).all()), "wrote past the end of out"
+
+
+def test_identical_bf16_gradients_at_scale_are_returned_bit_exactly(ac):
+    """64 identical bf16 gradients of 20M elements: every product x*s and x*x has few, structured
+    significant bits -- the case in which a single long fp32 sum would drift.  The statistics must
+    match the exact sum of squares, the weights must be 1/64, and out must equal g bit for bit."""
+    N, d = 64, 20_000_008
+    dev = torch.device("cuda:0")
+    gen = torch.Generator(device=dev).manual_seed(4)
+    g = (torch.randn(d, generator=gen, device=dev) * 0.01 + 0.003).to(torch.bfloat16)
+    G = g.unsqueeze(0).expand(N, d).contiguous()
+    out = torch.empty(d, dtype=torch.bfloat16, device=dev)
+    h = ac.AdaCons(N, d, "bf16")
+    for _ in range(2):                                    # the second step goes through the momentum
+        h.aggregate(G, out)
+    torch.cuda.synchronize()
+    _, q_ref = oc.consensus_statistics(to_f64(g.unsqueeze(0)))
+    q, p = h.coeffs(ac.COEFF_Q)[0], h.coeffs(ac.COEFF_P)[0]
+    assert np.all(np.abs(q - q_ref[0]) <= 1e-6 * q_ref[0]) and np.all(np.abs(p - q_ref[0]) <= 1e-6 * q_ref[0])
+    np.testing.assert_allclose(h.coeffs()[0], np.full(N, 1.0 / N), rtol=1e-12)
+    assert torch.equal(out.view(torch.int16), g.view(torch.int16))
