@@ -93,3 +93,18 @@ def test_binding_rejects_tensors_that_do_not_match_the_context():
     check_tensors(4, 100, "f32", 104, padded, out, want_cuda=False)          # padded rows are fine
     with pytest.raises(ValueError):
         check_tensors(4, 100, "f32", 100, G, out, want_cuda=True)             # host tensors on the device path
+
+
+def test_public_header_is_plain_c(tmp_path):
+    """include/adacons.h must compile as strict C99 (it is the C ABI) and as C++."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no gcc")
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "adacons.h"\nint use(void) { adacons_ctx *c = 0; (void)c; return ADACONS_NOALLOC_SCRATCH_BYTES > 0; }\n')
+    inc = os.path.join(ROOT, "include")
+    for cmd in (["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only"],
+                ["g++", "-std=c++17", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c++"]):
+        res = subprocess.run(cmd + ["-I", inc, str(src)], capture_output=True, text=True)
+        assert res.returncode == 0, res.stderr
