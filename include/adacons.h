@@ -26,6 +26,12 @@
  *   - Numerical degeneracies (a zero gradient, a vanishing or negative normaliser, Inf/NaN in
  *     the input) are not errors: the call completes with the documented fallback and raises a
  *     flag that adacons_get_status returns.
+ *   - Magnitudes.  Products g*g and g*s (s = the column sum) are accumulated in fp32, block
+ *     totals in fp64.  The result is scale-equivariant (exactly so for powers of two) while
+ *     those products stay normal fp32 numbers and a block's share of a row's sum does not
+ *     overflow: roughly 1e-15 <= |g| <= 1e15 for every element that matters to a norm.
+ *     Smaller elements lose relative accuracy in q_i (a row made only of such elements is
+ *     reported as a zero row); larger ones overflow to Inf and raise ADACONS_FLAG_NONFINITE.
  */
 #ifndef ADACONS_H_
 #define ADACONS_H_
@@ -150,7 +156,9 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  *   slower generic path with the same results.
  * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
  * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.
- * Errors: EINVAL (NULL pointers, overlap), ECUDA (launch failure).
+ * Errors: EINVAL (NULL pointers, overlap), ECUDA (launch failure), EALIGN (per-segment mode with
+ * misaligned buffers), ENOMEM (an earlier adacons_set_option ran out of memory and left the
+ * context without its buffers; destroy it).
  */
 int adacons_aggregate(adacons_ctx *ctx, const void *grads, void *out, void *cuda_stream);
 

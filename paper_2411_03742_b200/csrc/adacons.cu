@@ -576,6 +576,9 @@ int adacons_destroy(adacons_ctx* c) {
 
 int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_stream) {
   if (c == nullptr || grads == nullptr || out == nullptr) return ADACONS_EINVAL;
+  // an option change that ran out of memory half-way leaves the context without its buffers
+  if (c->partials == nullptr || c->coef == nullptr || c->gamma_f32 == nullptr || c->m == nullptr || c->z == nullptr)
+    return ADACONS_ENOMEM;
   const size_t gbytes = (static_cast<size_t>(c->N - 1) * c->pitch + c->d) * c->elem_bytes;
   const size_t obytes = static_cast<size_t>(c->d) * c->elem_bytes;
   const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads), o0 = reinterpret_cast<uintptr_t>(out);
@@ -769,6 +772,7 @@ int adacons_aggregate_host(adacons_ctx* c, const void* host_grads, void* host_ou
 
 int adacons_reset(adacons_ctx* c, void* cuda_stream) {
   if (c == nullptr) return ADACONS_EINVAL;
+  if (c->m == nullptr) return ADACONS_ENOMEM;
   DeviceGuard guard(c->device);
   if (!guard.ok) return ADACONS_ECUDA;
   const long long n = static_cast<long long>(c->sets()) * c->N;

@@ -71,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     if (global_timer_ns() - t0 > kWaitLimitNs) return false;
   }
 }
-// 2-D tiled TMA load global -> shared, completion reported on an mbarrier (no multicast).
+// 2-D tiled TMA load global -> shared, completion reported on an mbarrier.
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"

@@ -427,6 +427,39 @@ def test_bit_stability(ac, dtype, d):
     assert runs[0][2].tobytes() == runs[1][2].tobytes()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d", [100_000, 3_000_008, 1_000_003])
+def test_power_of_two_scaling_is_exact(ac, dtype, d):
+    """Scaling every gradient by 2^k scales p and q by 4^k, a and m by 2^k and leaves u, Z and gamma
+    alone; with a power of two each of these holds without any rounding, so the coefficients must be
+    bit-identical and the result must be the scaled result, bit for bit, as long as the squares stay
+    in the normal fp32 range.  Covers the single-pass, the TMA and the generic kernels."""
+    w = wl.Workload("pow2", 12, d, dtype, 3, "gauss", seed=77)
+    dev = "cuda:0"
+    Gs = [wl.generate(w, t, dev) for t in range(3)]
+    ref = None
+    for k in (0, -40, 40):
+        h = ac.AdaCons(w.N, w.d, dtype)
+        out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
+        outs = []
+        for G in Gs:
+            Gk = (G.float() * 2.0 ** k).to(w.torch_dtype)       # exact: only the exponent changes
+            assert torch.equal((Gk.float() * 2.0 ** -k).to(w.torch_dtype), G)
+            h.aggregate(Gk, out)
+            outs.append((out.float() * 2.0 ** -k).to(w.torch_dtype))
+        torch.cuda.synchronize()
+        assert h.status() == 0
+        got = (outs, h.coeffs(ac.COEFF_GAMMA).copy(), h.coeffs(ac.COEFF_A).copy() * 2.0 ** -k,
+               h.state()[0].copy() * 2.0 ** -k, h.coeffs(ac.COEFF_Q).copy() * 4.0 ** -k)
+        if ref is None:
+            ref = got
+            continue
+        for a, b in zip(ref[0], got[0]):
+            assert torch.equal(a.view(torch.uint8), b.view(torch.uint8)), k
+        for a, b in zip(ref[1:], got[1:]):
+            assert a.tobytes() == b.tobytes(), k
+
+
 def test_state_roundtrip_and_reset(ac):
     w = wl.Workload("state", 12, 30_000, "f32", 4, "gauss", seed=31)
     dev = "cuda:0"
