@@ -27,6 +27,21 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // each with its own tensor map and its own slice of the partial records.
 constexpr long long kChunkCols = 1ll << 30;
 
+// The opt-in limit on dynamic shared memory is a property of a kernel (per device), not of a
+// context, and contexts of different shapes share kernel instantiations.  Every kernel therefore
+// gets one fixed limit that covers all plans; a plan's own size only goes into its launches.
+constexpr size_t kPass1SmemBudget = 110 * 1024;                    // two blocks per SM
+constexpr size_t kPass1SmemCap = 112 * 1024;                       // budget + barriers
+constexpr size_t kFusedSmemCap = 160 * 1024;
+constexpr size_t kGenericSmemCap = static_cast<size_t>(kWarps) * kMaxN * 2 * sizeof(float);
+
+bool set_smem_cap(const void* kernel, size_t cap) {
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cap)) == cudaSuccess)
+    return true;
+  cudaGetLastError();
+  return false;
+}
+
 struct Pass1Plan {            // TMA-staged pass 1 for this (N, dtype)
   bool available = false;
   int NR = 0, WR = 0;
@@ -201,18 +216,14 @@ int plan_fast(adacons_ctx* c) {
   const size_t xch = WR > 1 ? static_cast<size_t>(2) * WR * WC * 32 * vec * sizeof(float) : 0;
   const size_t fixed = xch + static_cast<size_t>(kWarps) * NR * 2 * sizeof(float) +
                        static_cast<size_t>(2) * NR * kThreads * sizeof(float);   // exchange, block reduce, second-level sums
-  const size_t budget = 110 * 1024;   // two blocks per SM
+  const size_t budget = kPass1SmemBudget;
   int stages = static_cast<int>((budget - fixed - 64) / f.stage_bytes);
   if (stages > 8) stages = 8;
   if (stages < 2) stages = 2;
   f.stages = stages;
   f.smem_bytes = static_cast<size_t>(stages) * f.stage_bytes + fixed + static_cast<size_t>(stages) * 8;
   f.kernel = select_pass1(c->dtype, NR, WR);
-  if (cudaFuncSetAttribute(f.kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(f.smem_bytes)) !=
-      cudaSuccess) {
-    cudaGetLastError();
-    return ADACONS_ECUDA;
-  }
+  if (f.smem_bytes > kPass1SmemCap || !set_smem_cap(f.kernel, kPass1SmemCap)) return ADACONS_ECUDA;
   int per_sm = 0;
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, f.kernel, kThreads, f.smem_bytes) != cudaSuccess ||
       per_sm < 1) {
@@ -241,7 +252,7 @@ int plan_big(adacons_ctx* c) {
   const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_dot_kernel<0>)
                                           : reinterpret_cast<const void*>(&pass1_dot_kernel<1>);
   int per_sm = 0;
-  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->big_smem)) != cudaSuccess ||
+  if (c->big_smem > kPass1SmemCap || !set_smem_cap(k, kPass1SmemCap) ||
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, c->big_smem) != cudaSuccess || per_sm < 1) {
     cudaGetLastError();
     return ADACONS_OK;
@@ -291,11 +302,11 @@ int plan_fused(adacons_ctx* c) {
   if (grid < 1) grid = 1;
   const long long vpb = (num_vec + grid - 1) / grid;
   const size_t smem = static_cast<size_t>(c->N) * vpb * 16 + static_cast<size_t>(kFusedThreads / 32) * c->N * 2 * sizeof(float);
-  if (smem > 160 * 1024) return ADACONS_OK;
+  if (smem > kFusedSmemCap) return ADACONS_OK;
   const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&fused_small_kernel<0>)
                                           : reinterpret_cast<const void*>(&fused_small_kernel<1>);
   int per_sm = 0;
-  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess ||
+  if (!set_smem_cap(k, kFusedSmemCap) ||
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kFusedThreads, smem) != cudaSuccess) {
     cudaGetLastError();
     return ADACONS_OK;
@@ -451,11 +462,7 @@ int build_seg_plan(adacons_ctx* c) {
   c->seg_records = R;
   c->seg_bytes = bytes;
   c->seg_kernel = select_pass1_seg(c->dtype, c->fast.NR, c->fast.WR);
-  if (cudaFuncSetAttribute(c->seg_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           static_cast<int>(c->fast.smem_bytes)) != cudaSuccess) {
-    cudaGetLastError();
-    return ADACONS_ECUDA;
-  }
+  if (!set_smem_cap(c->seg_kernel, kPass1SmemCap)) return ADACONS_ECUDA;
   return ADACONS_OK;
 }
 
@@ -527,11 +534,11 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   // generic path: always available
   c->generic_tiles = static_cast<int>((d + kThreads * 4 - 1) / (kThreads * 4));
   c->generic_smem = static_cast<size_t>(kWarps) * N * 2 * sizeof(float);
-  cudaFuncSetAttribute(reinterpret_cast<const void*>(&pass1_generic_kernel<0>),
-                       cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->generic_smem));
-  cudaFuncSetAttribute(reinterpret_cast<const void*>(&pass1_generic_kernel<1>),
-                       cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->generic_smem));
-  if (!launch_ok()) { delete c; return ADACONS_ECUDA; }
+  if (!set_smem_cap(reinterpret_cast<const void*>(&pass1_generic_kernel<0>), kGenericSmemCap) ||
+      !set_smem_cap(reinterpret_cast<const void*>(&pass1_generic_kernel<1>), kGenericSmemCap)) {
+    delete c;
+    return ADACONS_ECUDA;
+  }
   c->generic_grid = sms * 4;
   if (c->generic_grid > c->generic_tiles) c->generic_grid = c->generic_tiles;
   c->max_partials = c->generic_grid;

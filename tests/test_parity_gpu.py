@@ -877,6 +877,52 @@ def test_two_contexts_on_two_streams_are_independent(ac):
     assert ha.coeffs(stream=sa).tobytes() == ca.tobytes() and hb.coeffs(stream=sb).tobytes() == cb.tobytes()
 
 
+def test_contexts_of_other_shapes_do_not_disturb_an_existing_one(ac):
+    """Contexts whose worker counts fall into the same kernel instantiation (N = 64 and N = 40 share
+    the 8 x 8 pass-1 kernel; all N share the generic and the single-pass kernels) need different
+    amounts of shared memory.  Creating the smaller plan after the larger one must leave the larger
+    one launchable, on every path."""
+    dev = torch.device("cuda:0")
+
+    def check(h, w, G):
+        out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
+        h.aggregate(G, out)
+        torch.cuda.synchronize()
+        res = oc.AdaConsOracle(w.N, w.d).step(to_f64(G)[:, :w.d], storage=w.dtype)
+        assert_coeffs(h.coeffs(ac.COEFF_GAMMA), res["gamma"], f"{w.name} gamma")
+        assert h.status() == 0
+
+    # TMA-staged pass 1: N = 64 needs more shared memory per stage than N = 40
+    big = wl.Workload("shape64", 64, 300_008, "bf16", 1, "gauss", seed=3)
+    small = wl.Workload("shape40", 40, 200_000, "bf16", 1, "gauss", seed=4)
+    hb = ac.AdaCons(big.N, big.d, "bf16"); hb.set_option(ac.OPT_FUSED_SMALL, 0)
+    hs = ac.AdaCons(small.N, small.d, "bf16"); hs.set_option(ac.OPT_FUSED_SMALL, 0)
+    Gb, Gs = wl.generate(big, 0, dev), wl.generate(small, 0, dev)
+    check(hs, small, Gs)
+    check(hb, big, Gb)
+    assert hb.info(ac.INFO_LAST_PATH) == 1 and hs.info(ac.INFO_LAST_PATH) == 1
+    # the allocation-free entry plans a third shape on the same kernel
+    pq = torch.empty(2 * 33, dtype=torch.float64, device=dev)
+    ac.stats_noalloc(wl.generate(wl.Workload("shape33", 33, 100_000, "bf16", 1, "gauss", seed=5), 0, dev), pq)
+    check(hb, big, Gb)
+    # generic path (odd length): N = 700 needs 44 KB, N = 3 a few bytes
+    gbig = wl.Workload("gen700", 700, 20_001, "f32", 1, "gauss", seed=6)
+    gsmall = wl.Workload("gen3", 3, 10_001, "f32", 1, "gauss", seed=7)
+    hgb, hgs = ac.AdaCons(gbig.N, gbig.d, "f32"), ac.AdaCons(gsmall.N, gsmall.d, "f32")
+    check(hgs, gsmall, wl.generate(gsmall, 0, dev))
+    check(hgb, gbig, wl.generate(gbig, 0, dev))
+    assert hgb.info(ac.INFO_LAST_PATH) == 2
+    # single-pass kernel: a matrix that nearly fills the grid's shared memory, then a tiny one
+    fbig = wl.Workload("fused_big", 16, 300_000, "f32", 1, "gauss", seed=8)
+    fsmall = wl.Workload("fused_small", 2, 64, "f32", 1, "gauss", seed=9)
+    hfb, hfs = ac.AdaCons(fbig.N, fbig.d, "f32"), ac.AdaCons(fsmall.N, fsmall.d, "f32")
+    check(hfs, fsmall, wl.generate(fsmall, 0, dev))
+    check(hfb, fbig, wl.generate(fbig, 0, dev))
+    assert hfb.info(ac.INFO_LAST_PATH) == 3
+    for h in (hb, hs, hgb, hgs, hfb, hfs):
+        h.close()
+
+
 def test_profile_and_info_getters(ac):
     w = wl.Workload("prof", 8, 2_000_000, "f32", 1, "gauss", seed=5)
     G = wl.generate(w, 0, "cuda:0")
