@@ -23,7 +23,7 @@ F32, BF16 = 0, 1
 COEFF_A, COEFF_A_TILDE, COEFF_GAMMA, COEFF_P, COEFF_Q = range(5)
 # enum adacons_info
 (INFO_NUM_SEGMENTS, INFO_COEFF_SETS, INFO_PASS1_BLOCKS, INFO_SCRATCH_BYTES, INFO_LAUNCHES_PER_CALL,
- INFO_LAST_PATH, INFO_TOTAL_LAUNCHES) = range(7)
+ INFO_LAST_PATH, INFO_TOTAL_LAUNCHES, INFO_LAST_PASS2) = range(8)
 # enum adacons_flag
 FLAG_ZERO_ROW, FLAG_DEGENERATE_Z, FLAG_NONFINITE, FLAG_NEG_Z, FLAG_TIMEOUT = 1, 2, 4, 8, 0x100
 # enum adacons_error

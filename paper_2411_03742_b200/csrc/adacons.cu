@@ -126,6 +126,7 @@ struct adacons_ctx {
   const void* tmap_for = nullptr;
 
   int last_path = 0;
+  int last_pass2 = 0;                   // 0 none, 1 generic, 2 16-byte vectors, 3 32-byte vectors
   long long total_launches = 0;
 
   // optional per-kernel timing (ADACONS_OPT_PROFILE)
@@ -431,16 +432,18 @@ int build_seg_plan(adacons_ctx* c) {
   }
   int R = 0;
   for (int sgm = 0; sgm < S; ++sgm) { rec_begin[sgm] = R; R += rec_count[sgm]; }
-  // pass 2: block bid covers vectors [num_vec - (bid+1)*span, num_vec - bid*span), clipped at 0
+  // pass 2: block bid owns the pairs of 16-byte groups [num_pairs - (bid+1)*P, num_pairs - bid*P), P = 256,
+  // i.e. groups [2*(num_pairs - (bid+1)*P), 2*(num_pairs - bid*P)) clipped to [0, num_vec) -- both vectorised kernels
   const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
   const long long num_vec = (c->d + vec - 1) / vec;
-  const long long span = static_cast<long long>(kThreads) * kPass2Groups;
-  const long long blocks2 = (num_vec + span - 1) / span;
+  const long long num_pairs = (num_vec + 1) / 2;
+  const long long blocks2 = (num_pairs + kPass2BlockPairs - 1) / kPass2BlockPairs;
   std::vector<int> blk(static_cast<size_t>(blocks2));
   for (long long bid = 0; bid < blocks2; ++bid) {
-    long long vlo = num_vec - (bid + 1) * span;
+    long long vlo = 2 * (num_pairs - (bid + 1) * kPass2BlockPairs);
     if (vlo < 0) vlo = 0;
-    const long long vhi = num_vec - 1 - bid * span;
+    long long vhi = 2 * (num_pairs - bid * kPass2BlockPairs) - 1;
+    if (vhi > num_vec - 1) vhi = num_vec - 1;
     const long long chi = vhi * vec + vec - 1 < c->d - 1 ? vhi * vec + vec - 1 : c->d - 1;
     const int slo = seg_of(vlo * vec), shi = seg_of(chi);
     blk[static_cast<size_t>(bid)] = slo == shi ? slo : -(slo + 1);
@@ -629,6 +632,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); cudaEventRecord(ev[3], st); c->prof_calls += 1; }
     c->last_path = 3;
+    c->last_pass2 = 0;
     c->last_launches = 1;
     c->total_launches += 1;
     return ADACONS_OK;
@@ -723,24 +727,32 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   // ---- pass 2 (Eq. 12) ----
   cudaError_t e2;
   if (aligned) {
-    const long long span = static_cast<long long>(kThreads) * kPass2Groups;
-    const unsigned blocks = static_cast<unsigned>((num_vec + span - 1) / span);
+    const long long num_pairs = (num_vec + 1) / 2;
+    const unsigned blocks = static_cast<unsigned>((num_pairs + kPass2BlockPairs - 1) / kPass2BlockPairs);
     const unsigned char* g8 = static_cast<const unsigned char*>(grads);
     unsigned char* o8 = static_cast<unsigned char*>(out);
     const int* bs = c->d_pass2_blk_seg;
     const long long* so = c->d_seg_off;
-    if (c->dtype == ADACONS_F32)
-      e2 = seg ? launch_kernel(pass2_vec_kernel<0, true>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
-               : launch_kernel(pass2_vec_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
-    else
-      e2 = seg ? launch_kernel(pass2_vec_kernel<1, true>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
-               : launch_kernel(pass2_vec_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems);
+    // 32-byte aligned buffers and pitch: one 256-bit load and store per thread and row
+    const bool wide = (g0 % 32 == 0) && (o0 % 32 == 0) && (row_bytes % 32 == 0);
+#define ADACONS_LAUNCH_PASS2(KERNEL) \
+    launch_kernel(KERNEL, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
+    if (c->dtype == ADACONS_F32) {
+      if (wide) e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_wide_kernel<0, true>)) : ADACONS_LAUNCH_PASS2((pass2_wide_kernel<0, false>));
+      else e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_vec_kernel<0, true>)) : ADACONS_LAUNCH_PASS2((pass2_vec_kernel<0, false>));
+    } else {
+      if (wide) e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_wide_kernel<1, true>)) : ADACONS_LAUNCH_PASS2((pass2_wide_kernel<1, false>));
+      else e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_vec_kernel<1, true>)) : ADACONS_LAUNCH_PASS2((pass2_vec_kernel<1, false>));
+    }
+#undef ADACONS_LAUNCH_PASS2
+    c->last_pass2 = wide ? 3 : 2;
   } else {
     const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);
     if (c->dtype == ADACONS_F32)
       e2 = launch_kernel(pass2_generic_kernel<0>, dim3(blocks), dim3(kThreads), 0, st, false, grads, out, c->gamma_f32, N, c->d, c->pitch);
     else
       e2 = launch_kernel(pass2_generic_kernel<1>, dim3(blocks), dim3(kThreads), 0, st, false, grads, out, c->gamma_f32, N, c->d, c->pitch);
+    c->last_pass2 = 1;
   }
   if (e2 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
   if (ev) { cudaEventRecord(ev[3], st); c->prof_calls += 1; }
@@ -984,6 +996,7 @@ int adacons_get_info(adacons_ctx* c, int key, int64_t* value) {
     case ADACONS_INFO_LAUNCHES_PER_CALL: *value = c->last_launches; return ADACONS_OK;
     case ADACONS_INFO_LAST_PATH: *value = c->last_path; return ADACONS_OK;
     case ADACONS_INFO_TOTAL_LAUNCHES: *value = c->total_launches; return ADACONS_OK;
+    case ADACONS_INFO_LAST_PASS2: *value = c->last_pass2; return ADACONS_OK;
     default: return ADACONS_EINVAL;
   }
 }

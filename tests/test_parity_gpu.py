@@ -737,15 +737,16 @@ def test_replay_from_a_cuda_graph_advances_the_state(ac):
 
 
 # ---- padded rows: any gradient length on the fast paths ------------------------------------------
-def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=None, per_segment=False, expect_path=None):
+def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=None, per_segment=False, expect_path=None,
+                 expect_pass2=None, out_shift=0):
     """Rows live in an N x pitch buffer whose padding is NaN; the result buffer is followed by a
     sentinel.  Neither may influence, or be touched by, the aggregation."""
     dev = torch.device("cuda:0")
     tdt = torch.float32 if dtype == "f32" else torch.bfloat16
     w = wl.Workload(f"pad{N}x{d}", N, d, dtype, steps, "gauss", seed=d % 1000 + N)
     buf = torch.full((N, pitch), float("nan"), dtype=tdt, device=dev)
-    obuf = torch.full((d + 32,), 7.0, dtype=tdt, device=dev)
-    out = obuf[:d]
+    obuf = torch.full((out_shift + d + 32,), 7.0, dtype=tdt, device=dev)
+    out = obuf[out_shift:out_shift + d]
     h = ac.AdaCons(N, d, dtype, seg_offsets=offsets)
     h.set_option(ac.OPT_ROW_PITCH, pitch)
     h.set_option(ac.OPT_FUSED_SMALL, 1 if fused else 0)
@@ -757,6 +758,7 @@ def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=
         h.set_option(k, v)
     h.set_option(ac.OPT_BETA, 0.8)
     orc = oc.AdaConsOracle(N, d, beta=0.8, **oracle_kw)
+    expected_flags = 0                                 # the status word accumulates until a reset
     for t in range(steps):
         G = wl.generate(w, t, dev)
         buf[:, :d] = G
@@ -764,13 +766,16 @@ def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=
         torch.cuda.synchronize()
         if expect_path is not None:
             assert h.info(ac.INFO_LAST_PATH) == expect_path
+        if expect_pass2 is not None:
+            assert h.info(ac.INFO_LAST_PASS2) == expect_pass2
         G64 = to_f64(G)
         res = oracle_step_with_kernel_ranks(orc, G64, dtype, h.coeffs(ac.COEFF_A))
-        assert h.status() == int(np.bitwise_or.reduce(res["flags"]))      # an empty segment raises flags
+        expected_flags |= int(np.bitwise_or.reduce(res["flags"]))          # an empty segment raises flags
+        assert h.status() == expected_flags
         assert_coeffs_by_set(h.coeffs(ac.COEFF_GAMMA), res["gamma"], f"pad gamma {t}")
         assert_coeffs_by_set(h.state()[0], res["m"], f"pad m {t}")
         assert_output(out, res, G64, dtype, f"pad out {t}", offsets)
-        assert bool((obuf[d:] == 7.0).all()), "wrote past the end of out"
+        assert bool((obuf[out_shift + d:] == 7.0).all()) and bool((obuf[:out_shift] == 7.0).all()), "wrote outside out"
         assert bool(torch.isnan(buf[:, d:]).all())
 
 
@@ -780,6 +785,53 @@ def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=
 def test_padded_rows_odd_length(ac, N, d, dtype, pitch, fused):
     big = N * pitch * (4 if dtype == "f32" else 2) > 20e6
     _padded_case(ac, N, d, dtype, pitch, 2, fused=fused, expect_path=1 if (not fused or big) else 3)
+
+
+# (dtype, d, pitch, shift of `out` in elements, pass-2 kernel: 2 = 16-byte vectors, 3 = 32-byte vectors)
+PASS2_WIDTH_CASES = [
+    ("bf16", 200_000, 200_000, 0, 3),    # even number of 16-byte groups, no tail
+    ("bf16", 200_003, 200_016, 0, 3),    # odd number of groups, the single last one partial
+    ("bf16", 200_011, 200_016, 0, 3),    # even number, the second of the last pair partial
+    ("bf16", 200_008, 200_016, 0, 3),    # odd number, full
+    ("bf16", 200_008, 200_008, 0, 2),    # pitch is 16 mod 32
+    ("bf16", 200_003, 200_008, 0, 2),
+    ("bf16", 200_000, 200_000, 8, 2),    # out is 16 mod 32
+    ("bf16", 1_000, 1_008, 0, 3),        # less than one block
+    ("bf16", 9, 16, 0, 3),               # one pair, second group partial
+    ("f32", 100_000, 100_000, 0, 3),
+    ("f32", 100_001, 100_008, 0, 3),
+    ("f32", 100_006, 100_008, 0, 3),
+    ("f32", 100_004, 100_008, 0, 3),
+    ("f32", 100_004, 100_004, 0, 2),
+    ("f32", 100_002, 100_004, 0, 2),
+    ("f32", 100_000, 100_000, 4, 2),
+    ("f32", 5, 8, 0, 3),
+]
+
+
+@pytest.mark.parametrize("dtype,d,pitch,shift,kernel", PASS2_WIDTH_CASES)
+@pytest.mark.parametrize("N", [3, 8, 13])
+def test_pass2_vector_widths(ac, N, dtype, d, pitch, shift, kernel):
+    """Pass 2 moves 32 bytes per instruction when grads, out and the pitch are 32-byte aligned and 16
+    bytes otherwise; both kernels share one block-to-column mapping.  Every combination of an odd or
+    even number of 16-byte groups with a full or partial last group, on both kernels."""
+    _padded_case(ac, N, d, dtype, pitch, 2, fused=False, expect_path=1, expect_pass2=kernel, out_shift=shift)
+
+
+@pytest.mark.parametrize("dtype,d,pitch,shift,kernel", [c for c in PASS2_WIDTH_CASES if c[1] >= 100_000])
+def test_pass2_vector_widths_per_segment(ac, dtype, d, pitch, shift, kernel):
+    """The same with one weight set per segment: boundaries inside a 32-byte pair, inside a 16-byte
+    group, at block edges, empty and one-column segments."""
+    vec = 8 if dtype == "bf16" else 4
+    blockc = 512 * vec                                   # columns of one pass-2 block
+    top = (d + vec - 1) // vec                           # blocks are counted from the end of the row
+    edge = max(0, ((top + 1) // 2 * 2 - 512 * 3)) * vec  # a block edge
+    off = sorted({0, 1, 1, vec + 1, 2 * vec, 3 * vec - 1, edge, edge + blockc // 2 + 3, edge + blockc, edge + blockc,
+                  d // 2, d // 2 + 1, d - vec - 1, d - 1, d})
+    off = [0, 1, 1] + [o for o in off if o > 1 and o < d] + [d - 1, d - 1, d] if d > 4 else [0, d]
+    off = sorted(off)
+    _padded_case(ac, 11, d, dtype, pitch, 2, fused=False, offsets=off, per_segment=True, expect_path=1,
+                 expect_pass2=kernel, out_shift=shift)
 
 
 def test_padded_rows_per_segment(ac):
