@@ -64,6 +64,7 @@ struct adacons_ctx {
   long long pitch = 0;                  // elements between the starts of two rows (>= d)
   int device = 0;
   int num_sms = 0;
+  long long l2_bytes = 0;
   std::vector<long long> seg_offsets;   // S + 1 entries
   int num_segments = 1;
 
@@ -509,11 +510,13 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
     return ADACONS_ECUDA;
   }
   if (major != 10) return ADACONS_EARCH;
+  int l2 = 0;
+  if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) != cudaSuccess) { cudaGetLastError(); l2 = 0; }
 
   adacons_ctx* c = new (std::nothrow) adacons_ctx();
   if (c == nullptr) return ADACONS_ENOMEM;
   c->N = N; c->d = d; c->pitch = d; c->dtype = dtype; c->elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
-  c->device = dev; c->num_sms = sms;
+  c->device = dev; c->num_sms = sms; c->l2_bytes = l2;
   if (num_segments > 0) {
     c->num_segments = num_segments;
     c->seg_offsets.assign(seg_offsets, seg_offsets + num_segments + 1);
@@ -735,16 +738,21 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     const long long* so = c->d_seg_off;
     // 32-byte aligned buffers and pitch: one 256-bit load and store per thread and row
     const bool wide = (g0 % 32 == 0) && (o0 % 32 == 0) && (row_bytes % 32 == 0);
+    // a result that fits in L2 is kept there (evict_last stores); a larger one is written plainly
+    const int keep = static_cast<long long>(obytes) <= c->l2_bytes ? 1 : 0;
 #define ADACONS_LAUNCH_PASS2(KERNEL) \
     launch_kernel(KERNEL, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems)
+#define ADACONS_LAUNCH_PASS2W(KERNEL) \
+    launch_kernel(KERNEL, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, num_vec, bs, so, tail_elems, keep)
     if (c->dtype == ADACONS_F32) {
-      if (wide) e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_wide_kernel<0, true>)) : ADACONS_LAUNCH_PASS2((pass2_wide_kernel<0, false>));
+      if (wide) e2 = seg ? ADACONS_LAUNCH_PASS2W((pass2_wide_kernel<0, true>)) : ADACONS_LAUNCH_PASS2W((pass2_wide_kernel<0, false>));
       else e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_vec_kernel<0, true>)) : ADACONS_LAUNCH_PASS2((pass2_vec_kernel<0, false>));
     } else {
-      if (wide) e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_wide_kernel<1, true>)) : ADACONS_LAUNCH_PASS2((pass2_wide_kernel<1, false>));
+      if (wide) e2 = seg ? ADACONS_LAUNCH_PASS2W((pass2_wide_kernel<1, true>)) : ADACONS_LAUNCH_PASS2W((pass2_wide_kernel<1, false>));
       else e2 = seg ? ADACONS_LAUNCH_PASS2((pass2_vec_kernel<1, true>)) : ADACONS_LAUNCH_PASS2((pass2_vec_kernel<1, false>));
     }
 #undef ADACONS_LAUNCH_PASS2
+#undef ADACONS_LAUNCH_PASS2W
     c->last_pass2 = wide ? 3 : 2;
   } else {
     const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);

@@ -1107,15 +1107,19 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
 // than 16-byte ones (a read-only sweep runs at the same 7.5-7.7 TB/s either way), but the result
 // costs less: a warp stores 1 KB contiguous per instruction and the whole pass takes 2.3 % less
 // (6.19 -> 6.05 ms on 43.5 GB, same GPU, same run).  With the wide store the L2 evict_last hint no
-// longer pays (6.07 with, 6.05 without), so the result is written with plain stores.
+// longer pays for a result larger than L2 (6.07 with, 6.05 without, and the next pass 1 is slower
+// with it), so such a result is written with plain stores.  A result that fits in L2
+// (keep_in_l2 != 0) is still written evict_last: it then stays in L2, where the next call
+// overwrites it and its consumer finds it, and never costs DRAM bandwidth at all.
 template <int DT, bool SEG, int U = kPass2WideRows>
 __global__ void __launch_bounds__(kThreads)
 pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
                   const float* __restrict__ gamma, int N, long long row_bytes, long long num_vec,
-                  const int* __restrict__ blk_seg, const long long* __restrict__ seg_off, int tail_elems) {
+                  const int* __restrict__ blk_seg, const long long* __restrict__ seg_off, int tail_elems, int keep_in_l2) {
   constexpr int VEC = Elem<DT>::kVec;
   constexpr int NP = VEC / 2;
   __shared__ float g_s[kMaxN];
+  const unsigned long long keep = keep_in_l2 ? l2_policy_evict_last() : 0ull;
   pdl_wait();                                        // the coefficient step has finished
   int code = 0;
   if (SEG) code = blk_seg[blockIdx.x];
@@ -1160,19 +1164,19 @@ pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __rest
           for (int h = 0; h < NP; ++h) acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[g], h), g2, acc[g][h]);
       }
       if (tail_elems != 0 && v0 + 1 == num_vec - 1) {          // the row's last group is partial
-        pass2_store<DT, NP>(out, v0, acc[0]);
+        pass2_store<DT, NP>(out, v0, acc[0], keep);
         pass2_store_tail<DT, NP>(out, v0 + 1, acc[1], tail_elems);
       } else {
-        st_global_v8(out + w * 32, pass2_pack<DT, NP>(acc[0]), pass2_pack<DT, NP>(acc[1]), 0ull);
+        st_global_v8(out + w * 32, pass2_pack<DT, NP>(acc[0]), pass2_pack<DT, NP>(acc[1]), keep);
       }
     } else {
-      pass2_single_vector<DT>(grads, out, g_s, N, row_bytes, v0, num_vec, tail_elems, 0ull);
+      pass2_single_vector<DT>(grads, out, g_s, N, row_bytes, v0, num_vec, tail_elems, keep);
     }
   } else {
     if (w < 0) return;
     for (int g = 0; g < 2; ++g)
       if (v0 + g < num_vec)
-        pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v0 + g, num_vec, tail_elems, seg_off, -code - 1, 0ull);
+        pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v0 + g, num_vec, tail_elems, seg_off, -code - 1, keep);
   }
 }
 
