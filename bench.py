@@ -36,7 +36,7 @@ CPU_BASELINE_COLUMNS = 4_000_000       # cpu_baseline leg of the CUDA arm: 3 ste
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/, as a multiple of the algorithmic bytes of that kernel (None = no capture for the
 # current kernel).
-NCU_TRAFFIC_RATIO = {"pass1": 1.0015, "pass2": 0.9876}
+NCU_TRAFFIC_RATIO = {"pass1": 1.0014, "pass2": 0.9988}
 
 
 def parse_args(argv=None):
@@ -96,7 +96,7 @@ def barrier():
 # clocks during the timed region (read-only NVML queries)
 # ------------------------------------------------------------------------------------------------
 class ClockSampler(threading.Thread):
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.005):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None

@@ -1173,10 +1173,14 @@ pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __rest
       pass2_single_vector<DT>(grads, out, g_s, N, row_bytes, v0, num_vec, tail_elems, keep);
     }
   } else {
-    if (w < 0) return;
-    for (int g = 0; g < 2; ++g)
-      if (v0 + g < num_vec)
-        pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v0 + g, num_vec, tail_elems, seg_off, -code - 1, keep);
+    // a block that spans a segment boundary works on single 16-byte groups; thread t takes groups
+    // lo + t and lo + 256 + t of the block's range so that a warp's loads stay contiguous
+    const long long lo = 2 * (num_pairs - (static_cast<long long>(blockIdx.x) + 1) * kPass2BlockPairs);
+    for (int g = 0; g < 2; ++g) {
+      const long long v = lo + threadIdx.x + g * kThreads;
+      if (v >= 0 && v < num_vec)
+        pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v, num_vec, tail_elems, seg_off, -code - 1, keep);
+    }
   }
 }
 
