@@ -88,34 +88,53 @@ def first_order_coefficients(p: np.ndarray, q: np.ndarray) -> np.ndarray:
 
 
 def subspace_momentum(a: np.ndarray, m_prev: np.ndarray, beta: float,
-                      sort: bool = True, assign=None) -> tuple[np.ndarray, np.ndarray, np.ndarray]:
+                      sort: bool = True) -> tuple[np.ndarray, np.ndarray, np.ndarray]:
     """Sorted subspace momentum (Eq. 11):
         m_t      = beta m_{t-1} + (1-beta) S(a)
         a_tilde  = S^{-1}(m_t)
     S sorts ascending and is stable (ties keep worker order).  With sort=False this is
     the index-coupled EMA of Eq. 10.  Returns (m_t, a_tilde, pi) where pi[k] is the
-    worker whose coefficient occupies sorted slot k.
-
-    The sorted values S(a), hence m_t, depend continuously on a, but which worker gets which
-    slot does not: two workers whose coefficients agree to within rounding may swap slots.
-    `assign` (optional, assign[i] = slot handed back to worker i) lets a caller that compares
-    against an implementation working in lower precision prescribe that implementation's
-    S^{-1}; the caller is responsible for checking that it sorts `a` to within its tolerance.
-    m_t is always computed from this function's own sort."""
+    worker whose coefficient occupies sorted slot k."""
     a = np.asarray(a, dtype=np.float64)
     n = a.shape[0]
     pi = np.argsort(a, kind="stable") if sort else np.arange(n)
     m = beta * np.asarray(m_prev, dtype=np.float64) + (1.0 - beta) * a[pi]
     a_tilde = np.empty(n, dtype=np.float64)
-    if assign is None:
-        a_tilde[pi] = m
-    else:
-        a_tilde[:] = m[np.asarray(assign, dtype=np.int64)]
+    a_tilde[pi] = m
     return m, a_tilde, pi
 
 
+def normalised_weights(a_tilde, q, *, normalize: bool = True):
+    """From the (smoothed) subspace coefficients to the weights on the raw gradients
+    (Eq. 8 and the text before Eq. 12, Eq. 13): returns (u, Z, gamma, flags).
+
+    normalize=False keeps lambda = 1 and the 1/N of Eq. 8: gamma_i = u_i / N."""
+    a_tilde = np.asarray(a_tilde, dtype=np.float64)
+    q = np.asarray(q, dtype=np.float64)
+    n = a_tilde.shape[0]
+    flags = 0
+    uniform = np.full(n, 1.0 / n)
+    # P has unit columns, psi = P alpha  =>  weight on g_i is alpha_i / ||g_i||  (Eq. 8)
+    u = np.zeros(n, dtype=np.float64)
+    nz = q > 0
+    u[nz] = a_tilde[nz] / np.sqrt(q[nz])
+    Z = float(np.sum(u))
+    if normalize:
+        # the weights are rescaled so that they add up to one  (text before Eq. 12, Eq. 13)
+        if (not np.isfinite(Z)) or abs(Z) <= DEGENERATE_REL * float(np.sum(np.abs(u))):
+            gamma = uniform
+            flags |= FLAG_DEGENERATE_Z
+        else:
+            gamma = u / Z
+            if Z < 0:
+                flags |= FLAG_NEG_Z
+    else:
+        gamma = u / n
+    return u, Z, gamma, flags
+
+
 def coefficients(p, q, m_prev, beta: float = DEFAULT_BETA, *, momentum: bool = True,
-                 sort: bool = True, normalize: bool = True, assign=None) -> dict:
+                 sort: bool = True, normalize: bool = True) -> dict:
     """Algorithm 1 steps 2-3: from the 2N statistics to the N weights gamma.
 
     momentum=False skips Eq. 11 (a_tilde = a, state untouched); sort=False uses Eq. 10;
@@ -138,27 +157,12 @@ def coefficients(p, q, m_prev, beta: float = DEFAULT_BETA, *, momentum: bool = T
                     flags=flags | FLAG_NONFINITE)
     a = first_order_coefficients(p, q)
     if momentum:
-        m, a_tilde, pi = subspace_momentum(a, m_prev, beta, sort=sort, assign=assign)
+        m, a_tilde, pi = subspace_momentum(a, m_prev, beta, sort=sort)
     else:
         m, a_tilde, pi = m_prev.copy(), a.copy(), np.arange(n)
-    # P has unit columns, psi = P alpha  =>  weight on g_i is alpha_i / ||g_i||  (Eq. 8)
-    u = np.zeros(n, dtype=np.float64)
-    nz = q > 0
-    u[nz] = a_tilde[nz] / np.sqrt(q[nz])
-    Z = float(np.sum(u))
-    if normalize:
-        # the weights are rescaled so that they add up to one  (text before Eq. 12, Eq. 13)
-        if (not np.isfinite(Z)) or abs(Z) <= DEGENERATE_REL * float(np.sum(np.abs(u))):
-            gamma = uniform
-            flags |= FLAG_DEGENERATE_Z
-        else:
-            gamma = u / Z
-            if Z < 0:
-                flags |= FLAG_NEG_Z
-    else:
-        gamma = u / n
+    u, Z, gamma, wflags = normalised_weights(a_tilde, q, normalize=normalize)
     return dict(p=p, q=q, a=a, a_tilde=a_tilde, u=u, Z=Z, gamma=gamma, m=m, pi=pi,
-                flags=flags)
+                flags=flags | wflags)
 
 
 def combine(G: np.ndarray, gamma: np.ndarray) -> np.ndarray:
@@ -219,10 +223,10 @@ class AdaConsOracle:
         self.m = np.zeros((self.S, self.N), dtype=np.float64)
         self.t = 0
 
-    def step(self, G: np.ndarray, storage: str | None = None, assign=None) -> dict:
+    def step(self, G: np.ndarray, storage: str | None = None) -> dict:
         """One aggregation.  Returns per-segment arrays (S x N) of p, q, a, a_tilde,
         gamma, the new state m, flags (S,), psi (d,) and, if `storage` is given, `out`
-        = psi rounded to that format.  `assign` (S x N, optional): see subspace_momentum."""
+        = psi rounded to that format."""
         G = np.asarray(G, dtype=np.float64)
         assert G.shape == (self.N, self.d)
         keys = ("p", "q", "a", "a_tilde", "u", "gamma")
@@ -235,13 +239,14 @@ class AdaConsOracle:
             Gs = G[:, lo:hi]
             p, q = consensus_statistics(Gs)
             c = coefficients(p, q, self.m[s], self.beta, momentum=self.momentum,
-                             sort=self.sort, normalize=self.normalize,
-                             assign=None if assign is None else assign[s])
+                             sort=self.sort, normalize=self.normalize)
             self.m[s] = c["m"]
             for k in keys:
                 res[k][s] = c[k]
             res["Z"][s] = c["Z"]
-            res["flags"][s] = c["flags"]
+            # a segment without columns is no layer (Section 4, layer-wise aggregation): its
+            # all-zero statistics are not a degenerate gradient and raise no flag
+            res["flags"][s] = c["flags"] if hi > lo else 0
             psi[lo:hi] = combine(Gs, c["gamma"])
         self.t += 1
         res["m"] = self.m.copy()

@@ -7,6 +7,7 @@ import pytest
 import torch
 
 from oracle import adacons_oracle as oc
+from parity_util import assert_coeffs, assert_output, oracle_step, to_f64
 
 pytestmark = pytest.mark.gpu
 
@@ -37,11 +38,12 @@ def test_regression_converges_and_tracks_the_oracle(N):
         G = lr.worker_gradients(w, N, 16, gen)
         h.aggregate(G, psi)
         torch.cuda.synchronize()
-        G64 = G.cpu().double().numpy()
-        res = orc.step(G64)
-        # sum(gamma) = 1 and the aggregated direction agree with the oracle
+        G64 = to_f64(G)
+        res = oracle_step(orc, G64, "f32", h.coeffs(ac.COEFF_A), what=f"regression N={N}")
+        # sum(gamma) = 1; state, weights and the aggregated direction agree with the oracle to the
+        # tolerances of the other parity tests (1e-5 relative, 1e-5 max|g| scaled by the weights' mass)
         assert abs(h.coeffs().sum() - 1.0) < 1e-12
-        np.testing.assert_allclose(np.sort(h.state()[0][0]), np.sort(res["m"][0]), rtol=1e-5, atol=1e-9)
-        err = np.abs(psi.cpu().double().numpy() - res["psi"]).max()
-        assert err <= 3e-5 * np.abs(G64).max(), (t, err)
+        assert_coeffs(h.state()[0][0], res["m"][0], f"m step {t}")
+        assert_coeffs(h.coeffs(ac.COEFF_GAMMA)[0], res["gamma"][0], f"gamma step {t}")
+        assert_output(psi, res, G64, "f32", f"regression N={N} step {t}")
         w = w - step * psi

@@ -268,20 +268,59 @@ def test_momentum_state_is_the_ema_of_order_statistics():
         np.testing.assert_allclose(r["a_tilde"][0], np.array(want)[ranks], rtol=1e-12)
 
 
-def test_prescribed_slot_assignment_only_changes_who_gets_which_slot():
-    """`assign` replaces S^{-1} and nothing else: the state is unchanged, the identity assignment
-    of the function's own ranks reproduces the default, and swapping two workers' slots swaps
-    exactly their smoothed coefficients."""
-    a = np.array([0.3, -1.0, 0.7, 0.1])
-    m0 = np.array([0.5, 0.6, 0.7, 0.8])
-    m, at, pi = oc.subspace_momentum(a, m0, 0.9)
-    ranks = np.empty(4, dtype=int); ranks[pi] = np.arange(4)
-    m2, at2, _ = oc.subspace_momentum(a, m0, 0.9, assign=ranks)
-    np.testing.assert_array_equal(m2, m); np.testing.assert_array_equal(at2, at)
-    swapped = ranks.copy(); swapped[[0, 3]] = swapped[[3, 0]]
-    m3, at3, _ = oc.subspace_momentum(a, m0, 0.9, assign=swapped)
-    np.testing.assert_array_equal(m3, m)
-    assert at3[0] == at[3] and at3[3] == at[0] and at3[1] == at[1] and at3[2] == at[2]
+def test_second_worked_example_three_betas():
+    """An independently computed example with irrational norms (tests/golden/): both steps for
+    beta = 0, 0.5 and 0.99, to the digits the example was given with."""
+    g = {}
+    with open(os.path.join(os.path.dirname(GOLD), "second_worked_example.txt")) as fh:
+        for line in fh:
+            line = line.split("#")[0].strip()
+            if line:
+                k, *v = line.split()
+                g[k] = np.array([float(t) for t in v])
+    tol = dict(rtol=5e-6, atol=0)          # half a unit of the sixth significant digit
+    for beta, tag in ((0.0, "beta0"), (0.5, "beta0.5"), (0.99, "beta0.99")):
+        o = oc.AdaConsOracle(3, 2, beta=beta)
+        r1 = o.step(g["step1.G"].reshape(3, 2))
+        r2 = o.step(g["step2.G"].reshape(3, 2))
+        for r, s in ((r1, "step1"), (r2, "step2")):
+            for key in ("p", "q", "a"):
+                np.testing.assert_allclose(r[key][0], g[f"{s}.{key}"], err_msg=f"{tag} {s}.{key}", **tol)
+            order = np.argsort(r["a"][0], kind="stable")
+            np.testing.assert_array_equal(order, g[f"{s}.pi"].astype(int))
+        np.testing.assert_allclose(r1["gamma"][0], g["step1.gamma"], **tol)
+        np.testing.assert_allclose(r1["psi"], g["step1.psi"], **tol)
+        np.testing.assert_allclose(r2["gamma"][0], g[f"{tag}.step2.gamma"], **tol)
+        np.testing.assert_allclose(r2["psi"], g[f"{tag}.step2.psi"], **tol)
+        if f"{tag}.step2.m" in g:
+            np.testing.assert_allclose(r2["m"][0], g[f"{tag}.step2.m"], **tol)
+
+
+def test_normalised_weights_closed_forms():
+    """normalised_weights alone (Eq. 8, Eq. 12-13): with a~_i = c ||g_i|| every u_i is c and the
+    weights are 1/N; in general gamma_i = (a~_i/||g_i||)/sum_j(a~_j/||g_j||), checked in exact
+    rationals with integer norms; lambda = 1 keeps Eq. 8's 1/N; the flags of the degenerate cases."""
+    q = np.array([4.0, 9.0, 25.0, 1.0])
+    u, Z, gamma, flags = oc.normalised_weights(0.7 * np.sqrt(q), q)
+    np.testing.assert_allclose(u, 0.7, rtol=1e-15)
+    np.testing.assert_allclose(gamma, 0.25, rtol=1e-15)
+    assert flags == 0 and abs(Z - 2.8) < 1e-14
+    at = [Fraction(3), Fraction(-1, 2), Fraction(5, 4), Fraction(2)]
+    norms = [2, 3, 5, 1]
+    uf = [x / n for x, n in zip(at, norms)]
+    want = [float(x / sum(uf)) for x in uf]
+    u, Z, gamma, flags = oc.normalised_weights(np.array([float(x) for x in at]), q)
+    np.testing.assert_allclose(gamma, want, rtol=1e-15)
+    assert abs(gamma.sum() - 1.0) < 1e-15 and flags == 0
+    _, _, g_un, _ = oc.normalised_weights(np.array([float(x) for x in at]), q, normalize=False)
+    np.testing.assert_allclose(g_un, [float(x) / 4 for x in uf], rtol=1e-15)
+    _, Z, gamma, flags = oc.normalised_weights(np.array([1.0, -1.0]), np.array([1.0, 1.0]))
+    assert flags == oc.FLAG_DEGENERATE_Z and np.all(gamma == 0.5) and Z == 0.0
+    _, Z, gamma, flags = oc.normalised_weights(np.array([1.0, -3.0]), np.array([1.0, 1.0]))
+    assert flags == oc.FLAG_NEG_Z and Z == -2.0
+    np.testing.assert_allclose(gamma, [-0.5, 1.5], rtol=1e-15)
+    u, _, gamma, _ = oc.normalised_weights(np.array([1.0, 5.0]), np.array([4.0, 0.0]))
+    assert u[1] == 0.0 and gamma[1] == 0.0 and gamma[0] == 1.0          # a zero gradient gets no weight
 
 
 # ---- variants (Table 2) ------------------------------------------------------------------
@@ -314,8 +353,8 @@ def test_per_segment_mode_is_the_global_rule_on_each_slice():
         G = rand_G(N, d, seed=400 + t, noise=1.0)
         r = o.step(G)
         for s in range(4):
-            if off[s + 1] == off[s]:
-                assert r["flags"][s] & oc.FLAG_DEGENERATE_Z
+            if off[s + 1] == off[s]:                 # no columns: no layer, no flag, state untouched
+                assert r["flags"][s] == 0 and not r["m"][s].any()
                 continue
             rs = subs[s].step(G[:, off[s]:off[s + 1]])
             np.testing.assert_allclose(r["psi"][off[s]:off[s + 1]], rs["psi"], rtol=1e-13)
