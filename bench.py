@@ -33,10 +33,14 @@ FALLBACK_HBM_GBS = 6650.0
 ORACLE_SAMPLE_COLUMNS = 2_000_000      # --impl reference: columns per step
 CPU_BASELINE_COLUMNS = 4_000_000       # cpu_baseline leg of the CUDA arm: 3 steps of this many columns
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
-# profiles/, as a multiple of the algorithmic bytes of that kernel (None = no capture for the
-# current kernel).
-NCU_TRAFFIC_RATIO = {"pass1": 1.0014, "pass2": 0.9988}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# captures summarised under profiles/ (a scaled-down case of the same recipe, traffic proportional
+# to the columns processed), as a multiple of that kernel's algorithmic bytes.  Keyed by
+# (workload, coefficient mode, kernel); anything else reports no traffic figure.
+NCU_TRAFFIC_RATIO = {
+    ("bert64", "model-wise", "pass1"): (1.0014, "profiles/pass1_pass2_bert64_d20M_full_set.md (d = 20 M, scaled by d)"),
+    ("bert64", "model-wise", "pass2"): (0.9988, "profiles/pass2_wide_mixed16_full_set.md (result larger than L2)"),
+}
 
 
 def parse_args(argv=None):
@@ -51,8 +55,12 @@ def parse_args(argv=None):
     ap.add_argument("--no-overlap-launch", action="store_true", help="plain stream order for the coefficient kernel too")
     ap.add_argument("--per-segment", action="store_true", help="layer-wise coefficients (workloads with segments)")
     ap.add_argument("--no-profile", action="store_true",
-                    help="keep the per-kernel CUDA events out of the timed region (they are taken in a second loop)")
+                    help="keep the per-kernel CUDA events out of the headline timed region (they are taken in a second loop)")
+    ap.add_argument("--no-extra-loops", action="store_true",
+                    help="skip the two additional loops (per-step events for the median; the launch sequence without events)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--one-launch", type=int, default=-1, choices=[-1, 0, 1, 2],
+                    help="ADACONS_OPT_ONE_LAUNCH (default: the library's own choice by size)")
     return ap.parse_args(argv)
 
 
@@ -250,6 +258,8 @@ def run_ours(args):
         h.set_option(ac.OPT_PER_SEGMENT, 1)
     if args.no_overlap_launch:
         h.set_option(ac.OPT_OVERLAP_LAUNCH, 0)
+    if args.one_launch >= 0:
+        h.set_option(ac.OPT_ONE_LAUNCH, args.one_launch)
     stream = torch.cuda.current_stream()
 
     for t in range(max(args.warmup, 3)):
@@ -285,10 +295,32 @@ def run_ours(args):
             h.aggregate(Gs[t % nbuf], out)
         torch.cuda.synchronize()
     kernel_ms, kcalls = h.profile()
+    extra = {}
+    if not args.no_extra_loops:
+        # (a) the launch sequence a user gets: no events between the kernels, so the coefficient
+        # kernel's launch overlaps pass 1; (b) one event per step, for the median step time
+        h.set_option(ac.OPT_PROFILE, 0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for t in range(args.steps):
+            h.aggregate(Gs[t % nbuf], out)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        extra["ms_per_step_no_kernel_events"] = e0.elapsed_time(e1) / args.steps
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        evs[0].record(stream)
+        for t in range(args.steps):
+            h.aggregate(Gs[t % nbuf], out)
+            evs[t + 1].record(stream)
+        torch.cuda.synchronize()
+        per = sorted(evs[t].elapsed_time(evs[t + 1]) for t in range(args.steps))
+        extra["ms_per_step_median"] = per[len(per) // 2] if len(per) % 2 else 0.5 * (per[len(per) // 2 - 1] + per[len(per) // 2])
+        extra["ms_per_step_min_max"] = [per[0], per[-1]]
     status = h.status()
     assert status == 0, f"library raised status flags {status:#x}"
     path = h.info(ac.INFO_LAST_PATH)
-    assert path in (1, 3), "benchmark must run the aligned fast path"
+    assert path in (1, 3, 5), "benchmark must run the aligned fast path"
 
     units_local = float(w.N) * w.d * args.steps
     ms, units = reduce_over_ranks(ms_local, units_local, device=dev)
@@ -305,15 +337,20 @@ def run_ours(args):
         dom = "fused"
         step_bytes = alg["fused"]
         hbm_gbs = step_bytes * args.steps / (ms_local * 1e-3) / 1e9
+    elif path == 5:   # one launch, two reads: only the whole kernel can be timed
+        alg = {"one_launch": step_bytes}
+        kms = {"one_launch": kernel_ms[0]}
+        dom = "one_launch"
     else:
         alg = {"pass1": float(w.N) * w.d * b, "pass2": float(w.N) * w.d * b + w.d * b}
         kms = {"pass1": kernel_ms[0], "coeff": kernel_ms[1], "pass2": kernel_ms[2]}
         dom = "pass1" if kms["pass1"] >= kms["pass2"] else "pass2"
     achieved = alg[dom] / (kms[dom] * 1e-3) / 1e9
-    ratio = NCU_TRAFFIC_RATIO.get(dom)
+    ratio, ratio_src = NCU_TRAFFIC_RATIO.get((w.name, "per segment" if args.per_segment else "model-wise", dom), (None, None))
     roofline = {
         "bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_source": peak_src, "traffic": (ratio * alg[dom] if ratio else None),
+        "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+        "peak_source": peak_src, "traffic": (ratio * alg[dom] if ratio else None), "traffic_source": ratio_src,
         "algorithmic_bytes_per_launch": alg[dom], "kernel_ms": kms, "timed_calls": kcalls,
         "events_in_timed_region": not args.no_profile,
         "other_kernel_gbs": {k: alg[k] / (kms[k] * 1e-3) / 1e9 for k in alg if k != dom},
@@ -322,11 +359,12 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32", "storage_dtype": w.dtype, "data": "synthetic",
         "config": {"workload": describe(w), "N": w.N, "d": w.d, "storage_dtype": w.dtype,
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "coefficients": "per segment" if args.per_segment else "model-wise",
-                   "path": {1: "three kernels (TMA-staged pass 1)", 3: "single-pass kernel (matrix in shared memory)"}[path],
+                   "path": {1: "three kernels (TMA-staged pass 1)", 3: "single-pass kernel (matrix in shared memory)",
+                            5: "one launch, two reads (pass 1, coefficient step, pass 2 in one cooperative kernel)"}[path],
                    "l2": (f"inputs ({gbytes / 1e9:.2f} GB) larger than the 126 MB L2; no flush between steps" if nbuf == 1 else
                           f"{nbuf} distinct input matrices of {gbytes / 1e9:.3f} GB used in turn ({nbuf * gbytes / 1e9:.2f} GB "
                           "between two uses of one matrix, larger than the 126 MB L2); no flush")},
@@ -334,6 +372,7 @@ def run_ours(args):
         "minimal_bytes_per_step": step_bytes,
         "roofline": roofline, "clocks": clocks, "gpu_launches": int(launches),
     }
+    line.update(extra)
 
     # ---- end to end through the host-buffer entry point -----------------------------------------
     if not args.no_e2e:

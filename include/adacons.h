@@ -56,18 +56,24 @@ enum adacons_error {
   ADACONS_ENOMEM = 3, /* device or host allocation failed                                       */
   ADACONS_ECUDA = 4,  /* a CUDA runtime/driver call failed, or no CUDA device                   */
   ADACONS_EARCH = 5,  /* the current device is not compute capability 10.x                      */
-  ADACONS_ETIMEOUT = 6, /* a bounded on-device wait gave up (reported by adacons_get_status)    */
+  ADACONS_ETIMEOUT = 6, /* reserved; an expired on-device wait is reported through the flag
+                           ADACONS_FLAG_TIMEOUT of adacons_get_status, not as a return code    */
   ADACONS_ELIMIT = 7   /* problem larger than the fixed scratch of adacons_stats_noalloc         */
 };
 
 /* Flags returned by adacons_get_status (OR over all segments since the last reset). */
 enum adacons_flag {
-  ADACONS_FLAG_ZERO_ROW = 1u,     /* some ||g_i|| = 0: that worker got weight 0                  */
+  ADACONS_FLAG_ZERO_ROW = 1u,     /* some ||g_i|| = 0: that worker got weight 0.  (A segment with
+                                     no columns at all is not data and raises neither this flag
+                                     nor the next; its weights read 1/N.)                        */
   ADACONS_FLAG_DEGENERATE_Z = 2u, /* sum_i u_i = 0 (|Z| <= 1e-12 sum|u_i|) or not finite:
                                      gamma_i = 1/N (plain mean) was used                         */
   ADACONS_FLAG_NONFINITE = 4u,    /* Inf/NaN statistic: gamma_i = 1/N, momentum state unchanged  */
   ADACONS_FLAG_NEG_Z = 8u,        /* sum_i u_i < 0: computed as defined                          */
-  ADACONS_FLAG_TIMEOUT = 0x100u   /* a bounded wait inside a kernel expired; result is invalid   */
+  ADACONS_FLAG_TIMEOUT = 0x100u   /* a bounded wait inside a kernel expired; the result of that
+                                     call is invalid.  Call adacons_reset before the next
+                                     aggregation: it also re-arms the single-pass kernel's grid
+                                     barrier, which a call that gave up leaves out of step.       */
 };
 
 /* Options (adacons_set_option / adacons_get_option).  Variants follow the ablation in Table 2. */
@@ -96,13 +102,31 @@ enum adacons_option {
                                   the grid (about 148 x 160 KB) and the buffers are 16-byte
                                   aligned, one cooperative kernel reads it from HBM once and does
                                   all three steps; 0: always the three-kernel path.              */
-  ADACONS_OPT_ROW_PITCH = 8    /* elements between the starts of two consecutive rows of the
+  ADACONS_OPT_ROW_PITCH = 8,   /* elements between the starts of two consecutive rows of the
                                   gradient matrix, >= d; default d (contiguous rows).  Applies to
                                   adacons_aggregate and adacons_aggregate_host.  A gradient length
                                   that is not a multiple of 16 bytes runs on the fast path when the
                                   rows are padded to a pitch that is; the padding is never read
-                                  as data and nothing is written past out[d-1].  Setting it
-                                  synchronises the device and may re-allocate scratch.           */
+                                  as data and nothing is written past out[d-1], but the vector
+                                  loads may touch it: with a pitch > d the whole N * pitch
+                                  elements must be readable (and out must not overlap them).
+                                  Setting it synchronises the device and may re-allocate scratch. */
+  ADACONS_OPT_ONE_LAUNCH = 9,  /* 1 (default): a matrix of up to 1 GiB that does not fit in shared
+                                  memory, on 32-byte aligned buffers and pitch with N <= 64, is
+                                  aggregated by ONE cooperative kernel (pass 1, the coefficient
+                                  step of Algorithm 1 steps 2-3 by the block that finishes pass 1
+                                  last, pass 2) instead of three launches: two reads of the
+                                  matrix as before, no kernel boundaries.  2: whenever the
+                                  buffers allow it, whatever the size.  0: never.  Same
+                                  coefficients, state and output bytes as the three-kernel path
+                                  (the block partials are added in the same fixed order).         */
+  ADACONS_OPT_CLUSTER_PASS1 = 10 /* 1 (default): with 64 < N <= 512 on aligned buffers pass 1 reads
+                                  the matrix ONCE: a thread-block cluster of 2, 4 or 8 blocks
+                                  shares each column tile, 64 rows per block, and exchanges the
+                                  partial column sums through distributed shared memory.  0: the
+                                  two-read form (column sums first, then dot products per 64
+                                  rows), which N > 512 always takes.  Results agree to fp32
+                                  rounding of the column sums.                                   */
 };
 
 /* Which N-vector adacons_get_coeffs returns (values of the most recent aggregate call). */
@@ -123,7 +147,10 @@ enum adacons_info {
   ADACONS_INFO_LAUNCHES_PER_CALL = 4,/* kernels launched by the most recent adacons_aggregate    */
   ADACONS_INFO_LAST_PATH = 5,        /* 0 = none yet, 1 = TMA-staged fast path, 2 = generic path,
                                         3 = single-pass kernel (matrix held in shared memory),
-                                        4 = N > 64: column sums, then dot products per 64 rows  */
+                                        4 = N > 64: column sums, then dot products per 64 rows,
+                                        5 = one launch, two reads (see ADACONS_OPT_ONE_LAUNCH),
+                                        6 = 64 < N <= 512: clusters, one read in pass 1
+                                            (see ADACONS_OPT_CLUSTER_PASS1)                      */
   ADACONS_INFO_TOTAL_LAUNCHES = 6,   /* kernels launched by this context so far                  */
   ADACONS_INFO_LAST_PASS2 = 7        /* pass-2 kernel of the most recent aggregate call: 0 = none
                                         (no call yet, or the single-pass kernel), 1 = generic,
@@ -156,8 +183,9 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  *   Fast path: grads and out 16-byte aligned, the row pitch in bytes (d*sizeof(element) unless
  *   ADACONS_OPT_ROW_PITCH says otherwise) a multiple of 16; with all three multiples of 32 pass 2
  *   moves 32 bytes per instruction and is about 2 % faster still.  With N <= 64 the matrix is read
- *   twice; with N > 64 three times (column sums first, then dot products per 64 rows; needs d
- *   floats of scratch, allocated in adacons_create).  Misaligned buffers or pitch are served by a
+ *   twice, and so it is with 64 < N <= 512 (thread-block clusters share a column tile); with
+ *   N > 512 three times (column sums first, then dot products per 64 rows; needs d floats of
+ *   scratch, allocated in adacons_create).  Misaligned buffers or pitch are served by a
  *   slower generic path with the same results.
  * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
  * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.
@@ -178,7 +206,9 @@ int adacons_aggregate(adacons_ctx *ctx, const void *grads, void *out, void *cuda
 int adacons_aggregate_host(adacons_ctx *ctx, const void *host_grads, void *host_out,
                            void *cuda_stream);
 
-/* alpha^m := 0, t := 0, status flags cleared (asynchronous on the stream). */
+/* Forget the history of Eq. 11: the momentum state alpha^m := 0 (so that the next call is the
+ * momentum-free rule of Eq. 7 and Eq. 12-13), t := 0, status flags cleared, the single-pass
+ * kernel's grid barrier re-armed.  Asynchronous on the stream.  Errors: EINVAL, ENOMEM, ECUDA. */
 int adacons_reset(adacons_ctx *ctx, void *cuda_stream);
 
 /* Free the context and everything it owns.  The caller must make sure no work of this context
@@ -262,10 +292,12 @@ int adacons_stats_noalloc(const void *grads, int N, int64_t d, int dtype, double
 
 /*
  * Self-test of the hang protection (no paper counterpart).  Every wait inside the library's
- * kernels -- on a TMA completion barrier, on the grid barrier of the single-pass kernel -- gives
+ * kernels -- on a TMA completion barrier, on the grid barrier of the single-pass kernel, on the
+ * published weights in the one-launch kernel -- gives
  * up after 2 s, raises ADACONS_FLAG_TIMEOUT and lets the kernel return.  This call launches a tiny
  * kernel whose wait can never be satisfied (which = 0: an mbarrier nobody arrives on; which = 1: a
- * grid barrier that expects one more block than was launched) so that the give-up path can be
+ * grid barrier that expects one more block than was launched; which = 2: the one-launch kernel's
+ * wait for weights that nobody publishes) so that the give-up path can be
  * exercised without faulting or hanging the device: about 2 s later adacons_get_status reports
  * ADACONS_FLAG_TIMEOUT.  Call adacons_reset afterwards (it clears the flag and the barrier
  * counter that which = 1 leaves odd).  Errors: EINVAL, ECUDA.

@@ -18,7 +18,7 @@ LIB_NAME = "libadacons_b200.so"
 F32, BF16 = 0, 1
 # enum adacons_option
 (OPT_BETA, OPT_MOMENTUM, OPT_SORTED, OPT_NORMALIZE, OPT_PER_SEGMENT, OPT_PROFILE, OPT_OVERLAP_LAUNCH,
- OPT_FUSED_SMALL, OPT_ROW_PITCH) = range(9)
+ OPT_FUSED_SMALL, OPT_ROW_PITCH, OPT_ONE_LAUNCH, OPT_CLUSTER_PASS1) = range(11)
 # enum adacons_coeff
 COEFF_A, COEFF_A_TILDE, COEFF_GAMMA, COEFF_P, COEFF_Q = range(5)
 # enum adacons_info
@@ -105,9 +105,18 @@ def stats_noalloc(grads, pq_out, stream=None) -> None:
     For callers that cannot allocate: e.g. a gradient hook inside a framework whose caching
     allocator already owns the device's memory."""
     import torch
+    if grads.dim() != 2 or grads.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("grads must be an N x d matrix of float32 or bfloat16")
     N, d = grads.shape
-    dt = {torch.float32: F32, torch.bfloat16: BF16}[grads.dtype]
-    assert pq_out.dtype == torch.float64 and pq_out.numel() >= 2 * N and pq_out.is_cuda and grads.is_cuda
+    if (N > 1 and grads.stride(0) != d) or (d > 1 and grads.stride(1) != 1):
+        raise ValueError("grads must be contiguous (rows d elements apart, unit column stride)")
+    if pq_out.dtype != torch.float64 or pq_out.dim() != 1 or pq_out.numel() < 2 * N or not pq_out.is_contiguous():
+        raise ValueError("pq_out must be a contiguous float64 vector of at least 2N elements")
+    if not (grads.is_cuda and pq_out.is_cuda) or grads.device != pq_out.device:
+        raise ValueError("grads and pq_out must live on the same CUDA device")
+    if grads.device.index != torch.cuda.current_device():
+        raise ValueError("grads must live on the current CUDA device")
+    dt = F32 if grads.dtype == torch.float32 else BF16
     _check(load_library().adacons_stats_noalloc(grads.data_ptr(), N, d, dt, pq_out.data_ptr(), _stream_handle(stream)),
            "adacons_stats_noalloc")
 

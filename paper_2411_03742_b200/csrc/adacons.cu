@@ -34,6 +34,9 @@ constexpr size_t kPass1SmemBudget = 110 * 1024;                    // two blocks
 constexpr size_t kPass1SmemCap = 112 * 1024;                       // budget + barriers
 constexpr size_t kFusedSmemCap = 160 * 1024;
 constexpr size_t kGenericSmemCap = static_cast<size_t>(kWarps) * kMaxN * 2 * sizeof(float);
+// Largest matrix (bytes) that takes the one-launch kernel by default: beyond it two kernel
+// boundaries are a negligible share of the step and the separate kernels are at least as fast.
+constexpr long long kOneLaunchMaxBytes = 1ll << 30;
 
 bool set_smem_cap(const void* kernel, size_t cap) {
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cap)) == cudaSuccess)
@@ -99,6 +102,11 @@ struct adacons_ctx {
   size_t colsum_bytes = 0;
   CUtensorMap tmap_big;
   const void* tmap_big_for = nullptr;
+  // 64 < N <= 512: one read of the matrix by clusters of 2, 4 or 8 blocks (64 rows each)
+  bool cl_available = false;
+  int cl_size = 0, cl_grid = 0, cl_tiles = 0;
+  size_t cl_smem = 0;
+  int cluster_pass1 = 1;                // ADACONS_OPT_CLUSTER_PASS1
   int last_launches = 3;
 
   // single-pass path for problems that fit in the grid's shared memory
@@ -106,6 +114,12 @@ struct adacons_ctx {
   int fused_grid = 0, fused_vpb = 0;
   size_t fused_smem = 0;
   unsigned long long* d_barrier = nullptr;
+
+  // one launch for mid-size matrices: pass 1, coefficient step and pass 2 in one cooperative kernel
+  bool mid_available = false;
+  int mid_grid = 0;
+  const void* mid_kernel = nullptr;
+  int one_launch = 1;                   // ADACONS_OPT_ONE_LAUNCH: 0 never, 1 by size, 2 whenever possible
 
   // per-segment ("layer-wise") plan, built when ADACONS_OPT_PER_SEGMENT is switched on
   int seg_grid = 0;               // blocks of pass1_seg_kernel
@@ -118,7 +132,7 @@ struct adacons_ctx {
   int* d_rec_count = nullptr;           // [S]
   int* d_set_first_block = nullptr;     // [S]
   float* d_records = nullptr;           // [seg_records][2N]
-  int* d_pass2_blk_seg = nullptr;       // [pass-2 blocks]
+  int* d_pass2_blk_seg = nullptr;       // [pass-2 blocks][2]: segment code, last segment
   size_t seg_bytes = 0;
 
   EncodeTiledFn encode = nullptr;
@@ -175,6 +189,25 @@ const void* select_pass1_seg(int dtype, int NR, int WR) {
   if (WR == 2) return pass1_seg_fn<DT, 8, 2>();              \
   if (WR == 4) return pass1_seg_fn<DT, 8, 4>();              \
   return pass1_seg_fn<DT, 8, 8>();
+  if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
+  ADACONS_PICK(1)
+#undef ADACONS_PICK
+}
+
+template <int DT, int NR, int WR>
+const void* mid_fn() { return reinterpret_cast<const void*>(&mid_fused_kernel<DT, NR, WR>); }
+
+const void* select_mid(int dtype, int NR, int WR) {
+#define ADACONS_PICK(DT)                                     \
+  if (WR == 1) {                                             \
+    if (NR == 1) return mid_fn<DT, 1, 1>();                  \
+    if (NR == 2) return mid_fn<DT, 2, 1>();                  \
+    if (NR == 4) return mid_fn<DT, 4, 1>();                  \
+    return mid_fn<DT, 8, 1>();                               \
+  }                                                          \
+  if (WR == 2) return mid_fn<DT, 8, 2>();                    \
+  if (WR == 4) return mid_fn<DT, 8, 4>();                    \
+  return mid_fn<DT, 8, 8>();
   if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
   ADACONS_PICK(1)
 #undef ADACONS_PICK
@@ -274,6 +307,38 @@ int plan_big(adacons_ctx* c) {
   return ADACONS_OK;
 }
 
+// 64 < N <= 512 on the aligned path: clusters of ceil(N / 64) blocks rounded up to 2, 4 or 8.
+// Shares the tensor map (boxes of 64 rows) and the shared-memory carve-up of the N > 64 path.
+int plan_cluster(adacons_ctx* c) {
+  c->cl_available = false;
+  if (c->N <= kMaxFastN || c->N > 512) return ADACONS_OK;
+  if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > kChunkCols) return ADACONS_OK;
+  const int tile_cols = kBoxRowBytes / c->elem_bytes;
+  c->cl_tiles = static_cast<int>((c->d + tile_cols - 1) / tile_cols);
+  c->cl_size = c->N <= 128 ? 2 : c->N <= 256 ? 4 : 8;
+  const uint32_t stage_bytes = 64u * kBoxRowBytes;
+  const int vec = c->dtype == ADACONS_F32 ? 4 : 8;
+  const size_t fixed = static_cast<size_t>(2) * 8 * 32 * vec * sizeof(float) + static_cast<size_t>(kWarps) * 8 * 2 * sizeof(float) +
+                       static_cast<size_t>(2) * 8 * kThreads * sizeof(float);
+  const size_t smem = 2 * static_cast<size_t>(stage_bytes) + fixed + 2 * 8;
+  const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_cluster_kernel<0>)
+                                          : reinterpret_cast<const void*>(&pass1_cluster_kernel<1>);
+  if (smem > kPass1SmemCap || !set_smem_cap(k, kPass1SmemCap)) return ADACONS_OK;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(c->cl_size) * 8); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(c->cl_size); attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  int clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&clusters, k, &cfg) != cudaSuccess || clusters < 1) { cudaGetLastError(); return ADACONS_OK; }
+  if (clusters > c->cl_tiles) clusters = c->cl_tiles;
+  c->cl_grid = clusters * c->cl_size;
+  c->cl_smem = smem;
+  c->cl_available = true;
+  return ADACONS_OK;
+}
+
 int encode_map_big(adacons_ctx* c, const void* grads) {
   if (c->tmap_big_for == grads) return ADACONS_OK;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
@@ -318,6 +383,31 @@ int plan_fused(adacons_ctx* c) {
   c->fused_vpb = static_cast<int>(vpb);
   c->fused_smem = smem;
   c->fused_available = true;
+  return ADACONS_OK;
+}
+
+// The one-launch kernel shares pass 1's plan (tiles, ring, shared memory); it needs a cooperative
+// launch of pass 1's grid and one column chunk.
+int plan_mid(adacons_ctx* c) {
+  c->mid_available = false;
+  if (!c->fast.available || c->num_chunks != 1) return ADACONS_OK;
+  int coop = 0;
+  if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) != cudaSuccess || !coop) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  const void* k = select_mid(c->dtype, c->fast.NR, c->fast.WR);
+  int per_sm = 0;
+  if (!set_smem_cap(k, kPass1SmemCap) ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, c->fast.smem_bytes) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  int grid = per_sm * c->num_sms;
+  if (grid > c->fast.grid) grid = c->fast.grid;       // never more blocks than pass 1 would use (or than tiles)
+  c->mid_grid = grid;
+  c->mid_kernel = k;
+  c->mid_available = true;
   return ADACONS_OK;
 }
 
@@ -439,7 +529,7 @@ int build_seg_plan(adacons_ctx* c) {
   const long long num_vec = (c->d + vec - 1) / vec;
   const long long num_pairs = (num_vec + 1) / 2;
   const long long blocks2 = (num_pairs + kPass2BlockPairs - 1) / kPass2BlockPairs;
-  std::vector<int> blk(static_cast<size_t>(blocks2));
+  std::vector<int> blk(static_cast<size_t>(2 * blocks2));   // per block: code, last segment
   for (long long bid = 0; bid < blocks2; ++bid) {
     long long vlo = 2 * (num_pairs - (bid + 1) * kPass2BlockPairs);
     if (vlo < 0) vlo = 0;
@@ -447,7 +537,8 @@ int build_seg_plan(adacons_ctx* c) {
     if (vhi > num_vec - 1) vhi = num_vec - 1;
     const long long chi = vhi * vec + vec - 1 < c->d - 1 ? vhi * vec + vec - 1 : c->d - 1;
     const int slo = seg_of(vlo * vec), shi = seg_of(chi);
-    blk[static_cast<size_t>(bid)] = slo == shi ? slo : -(slo + 1);
+    blk[static_cast<size_t>(2 * bid)] = slo == shi ? slo : -(slo + 1);
+    blk[static_cast<size_t>(2 * bid + 1)] = shi;
   }
   size_t bytes = 0;
   int rc;
@@ -551,16 +642,19 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   if (c->fast.available && c->fast.grid * c->num_chunks > c->max_partials) c->max_partials = c->fast.grid * c->num_chunks;
   plan_fused(c);
   if (c->fused_available && c->fused_grid > c->max_partials) c->max_partials = c->fused_grid;
+  plan_mid(c);
   rc = plan_big(c);
   if (rc != ADACONS_OK) { adacons_destroy(c); return rc; }
   if (c->big_available && c->big_grid > c->max_partials) c->max_partials = c->big_grid;
+  plan_cluster(c);
+  if (c->cl_available && c->cl_grid / c->cl_size > c->max_partials) c->max_partials = c->cl_grid / c->cl_size;
 
   if (cudaMalloc(&c->flags, sizeof(uint32_t)) != cudaSuccess || cudaMalloc(&c->step, sizeof(long long)) != cudaSuccess ||
-      cudaMalloc(&c->d_barrier, sizeof(unsigned long long)) != cudaSuccess) {
+      cudaMalloc(&c->d_barrier, 4 * sizeof(unsigned long long)) != cudaSuccess) {
     cudaGetLastError(); adacons_destroy(c); return ADACONS_ENOMEM;
   }
   if (cudaMemset(c->flags, 0, sizeof(uint32_t)) != cudaSuccess || cudaMemset(c->step, 0, sizeof(long long)) != cudaSuccess ||
-      cudaMemset(c->d_barrier, 0, sizeof(unsigned long long)) != cudaSuccess) {
+      cudaMemset(c->d_barrier, 0, 4 * sizeof(unsigned long long)) != cudaSuccess) {
     adacons_destroy(c); return ADACONS_ECUDA;
   }
   const size_t b_part = static_cast<size_t>(c->max_partials) * 2 * N * sizeof(float);
@@ -592,7 +686,8 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   // an option change that ran out of memory half-way leaves the context without its buffers
   if (c->partials == nullptr || c->coef == nullptr || c->gamma_f32 == nullptr || c->m == nullptr || c->z == nullptr)
     return ADACONS_ENOMEM;
-  const size_t gbytes = (static_cast<size_t>(c->N - 1) * c->pitch + c->d) * c->elem_bytes;
+  // with padded rows the vector loads may touch the last row's padding too: the matrix is N * pitch elements
+  const size_t gbytes = static_cast<size_t>(c->N) * c->pitch * c->elem_bytes;
   const size_t obytes = static_cast<size_t>(c->d) * c->elem_bytes;
   const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads), o0 = reinterpret_cast<uintptr_t>(out);
   if (o0 < g0 + gbytes && g0 < o0 + obytes) return ADACONS_EINVAL;   // out overlaps grads
@@ -624,7 +719,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     CoeffParams& q = f.coeff;
     q.N = N; q.num_partials = c->fused_grid; q.sets = 1; q.beta = c->beta;
     q.momentum = c->momentum; q.sorted = c->sorted; q.normalize = c->normalize;
-    q.partials = c->partials; q.rec_begin = nullptr; q.rec_count = nullptr;
+    q.partials = c->partials; q.rec_begin = nullptr; q.rec_count = nullptr; q.seg_off = nullptr;
     q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.z = c->z; q.flags = c->flags; q.step = c->step;
     const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&fused_small_kernel<0>)
                                             : reinterpret_cast<const void*>(&fused_small_kernel<1>);
@@ -636,6 +731,37 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); cudaEventRecord(ev[3], st); c->prof_calls += 1; }
     c->last_path = 3;
     c->last_pass2 = 0;
+    c->last_launches = 1;
+    c->total_launches += 1;
+    return ADACONS_OK;
+  }
+
+  // ---- one launch, two reads: mid-size matrices on 32-byte aligned buffers ----
+  if (!seg && aligned && c->mid_available && (g0 % 32 == 0) && (o0 % 32 == 0) && (row_bytes % 32 == 0) &&
+      (c->one_launch == 2 ||
+       (c->one_launch == 1 && static_cast<long long>(c->N) * row_bytes <= kOneLaunchMaxBytes))) {
+    int rc = encode_map(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    MidParams mp;
+    mp.p1.N = N; mp.p1.num_tiles = c->fast.num_tiles; mp.p1.stages = c->fast.stages; mp.p1.stage_bytes = c->fast.stage_bytes;
+    mp.p1.partials = c->partials; mp.p1.flags = c->flags;
+    CoeffParams& q = mp.coeff;
+    q.N = N; q.num_partials = c->mid_grid; q.sets = 1; q.beta = c->beta;
+    q.momentum = c->momentum; q.sorted = c->sorted; q.normalize = c->normalize;
+    q.partials = c->partials; q.rec_begin = nullptr; q.rec_count = nullptr; q.seg_off = nullptr;
+    q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.z = c->z; q.flags = c->flags; q.step = c->step;
+    mp.grads = static_cast<const unsigned char*>(grads); mp.out = static_cast<unsigned char*>(out);
+    mp.row_bytes = row_bytes; mp.num_vec = num_vec; mp.tail_elems = tail_elems;
+    mp.keep_in_l2 = static_cast<long long>(obytes) <= c->l2_bytes ? 1 : 0;
+    mp.sync = c->d_barrier + 1;
+    void* args[2] = {&c->tmaps[0], &mp};
+    if (cudaLaunchCooperativeKernel(c->mid_kernel, dim3(c->mid_grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); cudaEventRecord(ev[3], st); c->prof_calls += 1; }
+    c->last_path = 5;
+    c->last_pass2 = 3;
     c->last_launches = 1;
     c->total_launches += 1;
     return ADACONS_OK;
@@ -676,6 +802,24 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     num_partials = c->fast.grid * c->num_chunks;
     c->last_path = 1;
+  } else if (aligned && c->cl_available && c->cluster_pass1) {
+    int rc = encode_map_big(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    Pass1ClusterParams p;
+    p.N = N; p.num_tiles = c->cl_tiles; p.stages = 2; p.stage_bytes = 64u * kBoxRowBytes;
+    p.partials = c->partials; p.flags = c->flags;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(c->cl_grid)); cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = c->cl_smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(c->cl_size); attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e1 = c->dtype == ADACONS_F32 ? cudaLaunchKernelEx(&cfg, pass1_cluster_kernel<0>, c->tmap_big, p)
+                                                   : cudaLaunchKernelEx(&cfg, pass1_cluster_kernel<1>, c->tmap_big, p);
+    if (e1 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
+    num_partials = c->cl_grid / c->cl_size;
+    c->last_path = 6;
   } else if (aligned && c->big_available) {
     int rc = encode_map_big(c, grads);
     if (rc != ADACONS_OK) return rc;
@@ -717,6 +861,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   q.partials = seg ? c->d_records : c->partials;
   q.rec_begin = seg ? c->d_rec_begin : nullptr;
   q.rec_count = seg ? c->d_rec_count : nullptr;
+  q.seg_off = seg ? c->d_seg_off : nullptr;
   q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.z = c->z;
   q.flags = c->flags; q.step = c->step;
   int cthreads = 1024;
@@ -840,6 +985,10 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
     }
     case ADACONS_OPT_OVERLAP_LAUNCH: c->overlap_launch = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: c->fused_small = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_CLUSTER_PASS1: c->cluster_pass1 = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_ONE_LAUNCH:
+      if (value != 0.0 && value != 1.0 && value != 2.0) return ADACONS_EINVAL;
+      c->one_launch = static_cast<int>(value); return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: {
       const long long pitch = static_cast<long long>(value);
       if (static_cast<double>(pitch) != value || pitch < c->d || pitch >= (1ll << 40)) return ADACONS_EINVAL;
@@ -853,13 +1002,18 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       if (rc != ADACONS_OK) return rc;
       c->tmaps.resize(static_cast<size_t>(c->num_chunks));
       plan_fused(c);
+      plan_mid(c);
+      // the grid barrier and the ticket counter count in units of a plan's grid: start them afresh
+      if (cudaMemset(c->d_barrier, 0, 4 * sizeof(unsigned long long)) != cudaSuccess) return ADACONS_ECUDA;
       c->tmap_big_for = nullptr;
       rc = plan_big(c);
       if (rc != ADACONS_OK) return rc;
+      plan_cluster(c);
       int need = c->generic_grid;
       if (c->fast.available && c->fast.grid * c->num_chunks > need) need = c->fast.grid * c->num_chunks;
       if (c->fused_available && c->fused_grid > need) need = c->fused_grid;
       if (c->big_available && c->big_grid > need) need = c->big_grid;
+      if (c->cl_available && c->cl_grid / c->cl_size > need) need = c->cl_grid / c->cl_size;
       if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
         cudaFree(c->partials);
         c->partials = nullptr;
@@ -902,6 +1056,8 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_PROFILE: *value = c->profile; return ADACONS_OK;
     case ADACONS_OPT_OVERLAP_LAUNCH: *value = c->overlap_launch; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: *value = c->fused_small; return ADACONS_OK;
+    case ADACONS_OPT_ONE_LAUNCH: *value = c->one_launch; return ADACONS_OK;
+    case ADACONS_OPT_CLUSTER_PASS1: *value = c->cluster_pass1; return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: *value = static_cast<double>(c->pitch); return ADACONS_OK;
     default: return ADACONS_EINVAL;
   }
@@ -985,7 +1141,7 @@ int adacons_get_profile(adacons_ctx* c, double ms[3], int64_t* calls, void* cuda
 }
 
 int adacons_selftest_bounded_wait(adacons_ctx* c, int which, void* cuda_stream) {
-  if (c == nullptr || (which != 0 && which != 1)) return ADACONS_EINVAL;
+  if (c == nullptr || which < 0 || which > 2) return ADACONS_EINVAL;
   DeviceGuard guard(c->device);
   if (!guard.ok) return ADACONS_ECUDA;
   selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(which, c->d_barrier, c->flags);
@@ -1032,6 +1188,11 @@ struct NoAllocDevice {
   unsigned char* scratch = nullptr;   // device address of g_noalloc_scratch on this device
   EncodeTiledFn encode = nullptr;
   int sms = 0;
+  // launch plan of the most recent shape (a hook calls with the same shape every step)
+  bool plan_valid = false;
+  int plan_N = 0, plan_dtype = 0, plan_chunks = 1;
+  long long plan_d = 0;
+  Pass1Plan plan;
 };
 NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
 pthread_mutex_t g_noalloc_mutex = PTHREAD_MUTEX_INITIALIZER;
@@ -1095,10 +1256,23 @@ extern "C" int adacons_stats_noalloc(const void* grads, int N, int64_t d, int dt
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
   // A context object on the host stack only carries the launch plan; it owns no device memory.
+  // The plan (kernel attributes, occupancy query) is made once per shape and kept.
   adacons_ctx plan;
   plan.N = N; plan.d = d; plan.pitch = d; plan.dtype = dtype; plan.elem_bytes = dtype == ADACONS_F32 ? 4 : 2;
   plan.device = dev; plan.num_sms = nd->sms; plan.encode = nd->encode;
-  rc = plan_fast(&plan);
+  pthread_mutex_lock(&g_noalloc_mutex);
+  if (nd->plan_valid && nd->plan_N == N && nd->plan_d == d && nd->plan_dtype == dtype) {
+    plan.fast = nd->plan;
+    plan.num_chunks = nd->plan_chunks;
+    rc = ADACONS_OK;
+  } else {
+    rc = plan_fast(&plan);
+    if (rc == ADACONS_OK) {
+      nd->plan = plan.fast; nd->plan_chunks = plan.num_chunks;
+      nd->plan_N = N; nd->plan_d = d; nd->plan_dtype = dtype; nd->plan_valid = true;
+    }
+  }
+  pthread_mutex_unlock(&g_noalloc_mutex);
   if (rc != ADACONS_OK) return rc;
 
   float* partials = reinterpret_cast<float*>(nd->scratch);

@@ -561,6 +561,132 @@ pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams 
   p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst + prm.r0, dst + prm.N + prm.r0, prm.rows);
 }
 
+// ---- pass 1 for 64 < N <= 512 in ONE read of the matrix: a thread-block cluster per column tile ----
+// A cluster of C = 2, 4 or 8 blocks owns column tiles c, c + clusters, ...; block r of the cluster
+// stages rows [64 r, 64 r + 64) of a tile (one TMA box; rows past N are zero-filled, a block with
+// no rows at all stages nothing), adds them up as pass1_tma_kernel<DT, 8, 8> does, and leaves its
+// 64-row column sums in its own shared memory.  After a cluster barrier every block reads the C
+// partial column sums through distributed shared memory and adds them in rank order -- all blocks
+// get the same bits -- and accumulates x*s and x*x for its own rows.  The partial sums are
+// double-buffered, so one cluster barrier per tile suffices: a block overwrites buffer k & 1 only
+// after the barrier of tile k + 1, which its peers reach after they have read tile k's sums.
+// A cluster writes ONE partial record, each block its rows' slice.  A block whose wait on a copy
+// expired keeps meeting its peers at every barrier (with zeros) so that nobody is left waiting.
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_nctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_id_x() { uint32_t r; asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_count_x() { uint32_t r; asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// 16 bytes from the shared memory of block `rank` of this cluster, at the address `local` has here
+__device__ __forceinline__ float4 ld_cluster_v4(const float* local, uint32_t rank) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_addr(local)), "r"(rank));
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+  return v;
+}
+
+struct Pass1ClusterParams {
+  int N;
+  int num_tiles;
+  int stages;
+  uint32_t stage_bytes; // 64 * 512
+  float* partials;      // [clusters][2N]
+  uint32_t* flags;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 2)
+pass1_cluster_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1ClusterParams prm) {
+  using C = P1<DT, 8, 8>;
+  constexpr int VEC = C::VEC;
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int s_abort;
+  __shared__ __align__(16) float s_col[2][C::TILEC];    // this block's column sums of its 64 rows, in the exchange layout
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rw = warp;                                  // WR = 8, WC = 1
+  const uint32_t rank = cluster_ctarank(), csize = cluster_nctarank();
+  const int cid = static_cast<int>(cluster_id_x()), ncl = static_cast<int>(cluster_count_x());
+  const int r0 = static_cast<int>(rank) * 64;
+  const int rows = prm.N - r0 < 0 ? 0 : (prm.N - r0 < 64 ? prm.N - r0 : 64);
+  const bool idle = rows == 0;                          // a block beyond the last row only meets the barriers
+  const P1Smem sm = p1_carve<C>(smem_raw, prm.stages, prm.stage_bytes);
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < prm.stages; ++s) mbar_init(&sm.full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+  const int my_tiles = cid < prm.num_tiles ? (prm.num_tiles - cid + ncl - 1) / ncl : 0;   // the same in every block of the cluster
+  auto issue = [&](int k, int s) {
+    mbar_expect_tx(&sm.full[s], prm.stage_bytes);
+    tma_load_2d(sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes, &tmap, &sm.full[s], (cid + k * ncl) * C::TILEC, r0);
+  };
+  int issued = 0;
+  if (tid == 0 && !idle) {
+    const int pre = my_tiles < prm.stages ? my_tiles : prm.stages;
+    for (int k = 0; k < pre; ++k) issue(k, k);
+    issued = pre;
+  }
+  float2 pacc[8], qacc[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  p1_outer_clear<C>(sm.outer);
+  int s = 0;
+  uint32_t parity = 0;
+  bool dead = false;                                    // block-uniform: a wait expired earlier
+  for (int k = 0; k < my_tiles; ++k) {
+    uint4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
+    if (!idle && !dead) {
+      if (mbar_wait_bounded(&sm.full[s], parity)) p1_load_rows<C>(v, sm.stage_base + static_cast<size_t>(s) * prm.stage_bytes + lane * 16, rw, 64);
+      else atomicOr(&s_abort, 1);
+    }
+    float2 sp[C::NP];
+    p1_colsum<DT, C>(v, sp);
+    p1_xch_write<C>(sm.xch, sp, rw, 0, lane);
+    __syncthreads();                                    // the stage is in registers, the partials are written
+    if (s_abort) dead = true;
+    if (tid == 0 && !idle && !dead && k + prm.stages < my_tiles) {
+      fence_proxy_async_smem();
+      issue(k + prm.stages, s);
+      issued = k + prm.stages + 1;
+    }
+    float* mine = s_col[k & 1];
+    for (int idx = tid; idx < C::TILEC; idx += kThreads) {   // this block's 64-row sum of one column, row warps in order
+      float a = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) a += sm.xch[r * C::TILEC + idx];
+      mine[idx] = a;
+    }
+    cluster_sync_all();
+#pragma unroll
+    for (int h = 0; h < C::NP; ++h) sp[h] = make_float2(0.f, 0.f);
+    for (uint32_t r = 0; r < csize; ++r)                // blocks in rank order: the same sum everywhere
+#pragma unroll
+      for (int h2 = 0; h2 < VEC / 4; ++h2) {
+        const float4 w4 = ld_cluster_v4(mine + h2 * 128 + lane * 4, r);
+        sp[2 * h2] = __fadd2_rn(sp[2 * h2], make_float2(w4.x, w4.y));
+        sp[2 * h2 + 1] = __fadd2_rn(sp[2 * h2 + 1], make_float2(w4.z, w4.w));
+      }
+    p1_accumulate<DT, C>(v, sp, pacc, qacc);
+    if ((k & (kFoldTiles - 1)) == kFoldTiles - 1) p1_fold<C>(pacc, qacc, sm.outer);
+    if (++s == prm.stages) { s = 0; parity ^= 1u; }
+  }
+  cluster_sync_all();                                   // nobody leaves while a peer may still read its column sums
+  float* dst = prm.partials + static_cast<size_t>(cid) * 2 * prm.N;
+  if (dead) {
+    if (tid == 0) p1_drain_after_timeout(sm.full, prm.stages, issued, prm.flags);
+    if (tid < rows) { dst[r0 + tid] = 0.f; dst[prm.N + r0 + tid] = 0.f; }
+    return;
+  }
+  if (!idle) p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst + r0, dst + prm.N + r0, rows);
+}
+
 // ---- per-segment ("layer-wise") pass 1 ----------------------------------------------------------
 // Block b owns the contiguous tile range [b*T/G, (b+1)*T/G).  The column sums of a tile do not
 // depend on the segments; only the destination of x*s and x*x does.  The block keeps accumulators
@@ -775,6 +901,7 @@ struct CoeffParams {
   const float* partials; // [records][2N]
   const int* rec_begin;  // per set (nullptr in global mode)
   const int* rec_count;
+  const long long* seg_off; // per-segment mode: [sets + 1] column offsets (nullptr in global mode)
   double* coef;          // [5][sets][N]: a, a~, gamma, p, q   (enum adacons_coeff order)
   float* gamma_f32;      // [sets][N]   weights as pass 2 reads them
   double* m;             // [sets][N]   momentum state, in place
@@ -783,10 +910,12 @@ struct CoeffParams {
   long long* step;       // aggregation counter
 };
 
-__device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set) {
-  __shared__ double sh_part[2 * kMaxN];
-  __shared__ double sh_a[kMaxN];
-  __shared__ double sh_u[kMaxN];
+// Work arrays in shared memory: sh_part holds part_cap doubles (at least 2N), sh_a and sh_u N each.
+// The records are split into `groups` interleaved subsequences, which fixes the order of the fp64
+// sum; groups follows from N, part_cap and group_threads alone (not from the block size), so two
+// kernels that pass the same values add the same records in the same order.
+__device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set, double* sh_part, const int part_cap,
+                                           const int group_threads, double* sh_a, double* sh_u) {
   __shared__ int sh_bad, sh_zero;
   __shared__ double sh_Z;
   __shared__ int sh_uniform;
@@ -798,12 +927,12 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
   const int count = prm.rec_count ? prm.rec_count[set] : prm.num_partials;
   const float* base = prm.partials + static_cast<size_t>(begin) * V;
   // A record is V = 2N floats, read as 16-byte (N even) or 8-byte vectors; `groups` interleaved
-  // subsequences of the records are summed in parallel (at most 32, and groups * V <= 2048).
+  // subsequences of the records are summed in parallel (at most 32, and groups * V <= part_cap).
   const int w = (V % 4 == 0) ? 4 : 2;
   const int units = V / w;
-  int groups = T / units;
+  int groups = group_threads / units;
   if (groups > 32) groups = 32;
-  if (groups > 2 * kMaxN / V) groups = 2 * kMaxN / V;
+  if (groups > part_cap / V) groups = part_cap / V;
   if (groups < 1) groups = 1;
   for (int slot = i; slot < units * groups; slot += T) {
     const int g = slot / units, u = slot - g * units;
@@ -838,7 +967,10 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
     prm.coef[4 * per + set * N + i] = q;
   }
   __syncthreads();
-  uint32_t flags = sh_zero ? kFlagZeroRow : 0u;
+  // A segment without columns is no layer: its all-zero statistics take the usual fallbacks
+  // (weights 1/N, state unchanged at zero) but are no degeneracy of the data and raise no flag.
+  const bool empty_set = prm.seg_off != nullptr && prm.seg_off[set + 1] == prm.seg_off[set];
+  uint32_t flags = (sh_zero && !empty_set) ? kFlagZeroRow : 0u;
   const double uniform = 1.0 / static_cast<double>(N);
   if (sh_bad) {   // non-finite statistic: plain mean, momentum state left as it was
     if (i < N) {
@@ -870,7 +1002,8 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
       }
     }
     double* slot = prm.m + static_cast<size_t>(set) * N + rank;
-    at = prm.beta * (*slot) + (1.0 - prm.beta) * a;              // exactly one writer per slot
+    // spelled out so that every kernel this is inlined into rounds the same way (one product, one fused step)
+    at = __fma_rn(prm.beta, *slot, __dmul_rn(1.0 - prm.beta, a));   // exactly one writer per slot
     *slot = at;
   }
   const double u = q > 0.0 ? at / rq : 0.0;                      // unit-column P: weight on raw g_i
@@ -883,7 +1016,7 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
     prm.z[set] = Z;
     sh_uniform = 0;
     if (prm.normalize) {
-      if (!isfinite(Z) || fabs(Z) <= 1e-12 * A) { sh_uniform = 1; flags |= kFlagDegenerateZ; }
+      if (!isfinite(Z) || fabs(Z) <= 1e-12 * A) { sh_uniform = 1; if (!empty_set) flags |= kFlagDegenerateZ; }
       else if (Z < 0.0) flags |= kFlagNegZ;
     }
     if (flags) atomicOr(prm.flags, flags);
@@ -901,6 +1034,13 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
   }
 }
 
+__device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set) {
+  __shared__ double sh_part[2 * kMaxN];
+  __shared__ double sh_a[kMaxN];
+  __shared__ double sh_u[kMaxN];
+  coeff_core(prm, set, sh_part, 2 * kMaxN, static_cast<int>(blockDim.x), sh_a, sh_u);
+}
+
 __global__ void __launch_bounds__(kMaxN)
 coeff_kernel(const CoeffParams prm) {
   pdl_launch_dependents();
@@ -915,9 +1055,9 @@ coeff_kernel(const CoeffParams prm) {
 // 0.119 ms whether the preceding sweep read the same matrix or another one, in either direction,
 // and evict_last hints on the sweep's last 16-128 MB move it by under 3 %.)  Rows are added in
 // index order with fp32 FMA.
-// SEG = true: one weight set per segment.  blk_seg[b] >= 0 names the single segment that holds
-// all columns of block b; otherwise -(s+1), s = segment of the block's lowest column, and every
-// thread finds the segment of each of its columns itself.
+// SEG = true: one weight set per segment.  blk_seg[2b] >= 0 names the single segment that holds
+// all columns of block b; otherwise it is -(s+1), s = segment of the block's lowest column, and
+// blk_seg[2b+1] is the segment of its highest column (see "blocks that span segment boundaries").
 // ----------------------------------------------------------------------------------------------
 // `policy` is an L2 eviction-priority descriptor (0 = none).  The 16-byte kernel writes its
 // result with evict_last: the 680 MB-scale result is only 1/N of the traffic but, left to the
@@ -1032,6 +1172,66 @@ __device__ __forceinline__ void pass2_mixed_vector(const unsigned char* __restri
   pass2_store_any<DT, NP>(out, v, acc, num_vec, tail_elems, policy);
 }
 
+// ---- blocks that span segment boundaries (SEG kernels) -------------------------------------------
+// Such a block keeps the weights of ALL segments it touches in shared memory ([nseg][N], at most
+// kSegSmemFloats floats and kSegSmemSegs segments) next to their column offsets.  A thread whose
+// columns lie in one segment -- all but the few that straddle a boundary -- runs the ordinary
+// vector loop with that segment's row of weights; a straddling thread looks the weight of each of
+// its columns up in shared memory.  Blocks that touch more segments than fit fall back to
+// pass2_mixed_vector (weights from global memory).
+constexpr int kSegSmemFloats = 4096;
+constexpr int kSegSmemSegs = 128;
+
+// index (relative to the block's first segment) of the segment that holds column c
+__device__ __forceinline__ int seg_find(const long long* off_s, int nseg, long long c) {
+  int lo = 0, hi = nseg - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (off_s[mid + 1] > c) hi = mid; else lo = mid + 1;
+  }
+  return lo;
+}
+
+template <int DT>
+__device__ __forceinline__ void pass2_mixed_vector_smem(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
+                                                        const float* g_seg, const long long* off_s, int nseg, int N,
+                                                        long long row_bytes, long long v, long long num_vec, int tail_elems,
+                                                        unsigned long long policy) {
+  constexpr int VEC = Elem<DT>::kVec;
+  constexpr int NP = VEC / 2;
+  const long long d_cols = (num_vec - 1) * VEC + (tail_elems ? tail_elems : VEC);
+  int sg = seg_find(off_s, nseg, v * VEC);
+  int seg_of[VEC];
+#pragma unroll
+  for (int e = 0; e < VEC; ++e) {
+    const long long c = v * VEC + e;
+    if (c < d_cols)
+      while (c >= off_s[sg + 1]) ++sg;
+    seg_of[e] = sg * N;                          // padding columns: any set, never stored
+  }
+  const unsigned char* col = grads + v * 16;
+  float2 acc[NP];
+#pragma unroll
+  for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+  for (int i = 0; i < N; ++i) {
+    const uint4 x = ld_stream_v4(col + static_cast<long long>(i) * row_bytes);
+#pragma unroll
+    for (int h = 0; h < NP; ++h)
+      acc[h] = __ffma2_rn(unpack_pair<DT>(x, h), make_float2(g_seg[seg_of[2 * h] + i], g_seg[seg_of[2 * h + 1] + i]), acc[h]);
+  }
+  pass2_store_any<DT, NP>(out, v, acc, num_vec, tail_elems, policy);
+}
+
+// Loads the weights and offsets of segments sg0..sg1 into shared memory; false if they do not fit.
+__device__ __forceinline__ bool seg_block_setup(float* g_seg, long long* off_s, const float* __restrict__ gamma,
+                                                const long long* __restrict__ seg_off, int sg0, int sg1, int N) {
+  const int nseg = sg1 - sg0 + 1;
+  if (nseg > kSegSmemSegs || nseg * N > kSegSmemFloats) return false;
+  for (int idx = threadIdx.x; idx < nseg * N; idx += kThreads) g_seg[idx] = gamma[static_cast<size_t>(sg0) * N + idx];
+  for (int j = threadIdx.x; j <= nseg; j += kThreads) off_s[j] = seg_off[sg0 + j];
+  return true;
+}
+
 // Narrow kernel (buffers 16-byte but not 32-byte aligned): thread t of block b owns the groups
 // lo + t and lo + 256 + t of the block's range, one 16-byte load each.
 template <int DT, bool SEG, int U = kPass2Rows>
@@ -1042,11 +1242,12 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
   constexpr int VEC = Elem<DT>::kVec;
   constexpr int NP = VEC / 2;
   constexpr int CG = 2;
-  __shared__ float g_s[kMaxN];
+  __shared__ float g_s[SEG ? kSegSmemFloats : kMaxN];
+  __shared__ long long off_s[SEG ? kSegSmemSegs + 1 : 1];
   const unsigned long long keep = l2_policy_evict_last();
   pdl_wait();                                        // the coefficient step has finished
   int code = 0;
-  if (SEG) code = blk_seg[blockIdx.x];
+  if (SEG) code = blk_seg[2 * blockIdx.x];
   const long long num_pairs = (num_vec + 1) / 2;
   const long long base = 2 * (num_pairs - (static_cast<long long>(blockIdx.x) + 1) * kPass2BlockPairs) + threadIdx.x;
   if (!SEG || code >= 0) {
@@ -1096,12 +1297,64 @@ pass2_vec_kernel(const unsigned char* __restrict__ grads, unsigned char* __restr
         if (v >= 0 && v < num_vec) pass2_single_vector<DT>(grads, out, g_s, N, row_bytes, v, num_vec, tail_elems, keep);
       }
     }
-  } else {
+  } else if (SEG) {
+    // the block spans segment boundaries: weights of all its segments in shared memory if they fit
+    const int sg0 = -code - 1, sg1 = blk_seg[2 * blockIdx.x + 1];
+    const bool fits = seg_block_setup(g_s, off_s, gamma, seg_off, sg0, sg1, N);   // block-uniform
+    __syncthreads();
+    const long long d_cols = (num_vec - 1) * VEC + (tail_elems ? tail_elems : VEC);
     for (int g = 0; g < CG; ++g) {
       const long long v = base + g * kThreads;
-      if (v >= 0 && v < num_vec)
-        pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v, num_vec, tail_elems, seg_off, -code - 1, keep);
+      if (v < 0 || v >= num_vec) continue;
+      if (!fits) {
+        pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v, num_vec, tail_elems, seg_off, sg0, keep);
+        continue;
+      }
+      const int nseg = sg1 - sg0 + 1;
+      const int sl = seg_find(off_s, nseg, v * VEC);
+      const long long c_last = (v * VEC + VEC < d_cols ? v * VEC + VEC : d_cols) - 1;
+      if (c_last < off_s[sl + 1])                      // the whole group lies in one segment
+        pass2_single_vector<DT>(grads, out, g_s + sl * N, N, row_bytes, v, num_vec, tail_elems, keep);
+      else
+        pass2_mixed_vector_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, v, num_vec, tail_elems, keep);
     }
+  }
+}
+
+// 32 contiguous bytes (two 16-byte column groups) of every row, weights from shared memory: one
+// 256-bit streaming load per row, U rows in flight, rows added in index order.
+template <int DT, int U>
+__device__ __forceinline__ void pass2_wide_pair(const unsigned char* __restrict__ col, const float* g_s, int N,
+                                                long long row_bytes, float2 (&acc)[2][Elem<DT>::kVec / 2]) {
+  constexpr int NP = Elem<DT>::kVec / 2;
+#pragma unroll
+  for (int g = 0; g < 2; ++g)
+#pragma unroll
+    for (int h = 0; h < NP; ++h) acc[g][h] = make_float2(0.f, 0.f);
+  int i0 = 0;
+  for (; i0 + U <= N; i0 += U) {
+    uint4 x[U][2];
+#pragma unroll
+    for (int u = 0; u < U; ++u) ld_stream_v8(col + static_cast<long long>(i0 + u) * row_bytes, x[u][0], x[u][1]);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const float gm = g_s[i0 + u];
+      const float2 g2 = make_float2(gm, gm);
+#pragma unroll
+      for (int g = 0; g < 2; ++g)
+#pragma unroll
+        for (int h = 0; h < NP; ++h) acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[u][g], h), g2, acc[g][h]);
+    }
+  }
+  for (; i0 < N; ++i0) {
+    uint4 x[2];
+    ld_stream_v8(col + static_cast<long long>(i0) * row_bytes, x[0], x[1]);
+    const float gm = g_s[i0];
+    const float2 g2 = make_float2(gm, gm);
+#pragma unroll
+    for (int g = 0; g < 2; ++g)
+#pragma unroll
+      for (int h = 0; h < NP; ++h) acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[g], h), g2, acc[g][h]);
   }
 }
 
@@ -1122,69 +1375,64 @@ pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __rest
                   const int* __restrict__ blk_seg, const long long* __restrict__ seg_off, int tail_elems, int keep_in_l2) {
   constexpr int VEC = Elem<DT>::kVec;
   constexpr int NP = VEC / 2;
-  __shared__ float g_s[kMaxN];
+  __shared__ float g_s[SEG ? kSegSmemFloats : kMaxN];
+  __shared__ long long off_s[SEG ? kSegSmemSegs + 1 : 1];
   const unsigned long long keep = keep_in_l2 ? l2_policy_evict_last() : 0ull;
   pdl_wait();                                        // the coefficient step has finished
   int code = 0;
-  if (SEG) code = blk_seg[blockIdx.x];
+  if (SEG) code = blk_seg[2 * blockIdx.x];
   const long long num_pairs = (num_vec + 1) / 2;
   const long long w = num_pairs - (static_cast<long long>(blockIdx.x) + 1) * kPass2BlockPairs + threadIdx.x;
   const long long v0 = 2 * w;
+  const float* gw = g_s;                             // this thread's row of weights
+  bool straddles = false;                            // its 32 bytes hold a segment boundary
+  int nseg = 1;
   if (!SEG || code >= 0) {
     const float* gsrc = gamma + static_cast<size_t>(SEG ? code : 0) * N;
     for (int i = threadIdx.x; i < N; i += kThreads) g_s[i] = gsrc[i];
     __syncthreads();
     if (w < 0) return;
-    if (v0 + 1 < num_vec) {                          // the pair is complete (all but an odd row's last group)
-      float2 acc[2][NP];
-#pragma unroll
-      for (int g = 0; g < 2; ++g)
-#pragma unroll
-        for (int h = 0; h < NP; ++h) acc[g][h] = make_float2(0.f, 0.f);
-      const unsigned char* col = grads + w * 32;
-      int i0 = 0;
-      for (; i0 + U <= N; i0 += U) {
-        uint4 x[U][2];
-#pragma unroll
-        for (int u = 0; u < U; ++u) ld_stream_v8(col + static_cast<long long>(i0 + u) * row_bytes, x[u][0], x[u][1]);
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const float gm = g_s[i0 + u];
-          const float2 g2 = make_float2(gm, gm);
-#pragma unroll
-          for (int g = 0; g < 2; ++g)
-#pragma unroll
-            for (int h = 0; h < NP; ++h) acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[u][g], h), g2, acc[g][h]);
-        }
+  } else {
+    // the block spans segment boundaries: weights of all its segments in shared memory if they fit
+    const int sg0 = -code - 1, sg1 = blk_seg[2 * blockIdx.x + 1];
+    const bool fits = seg_block_setup(g_s, off_s, gamma, seg_off, sg0, sg1, N);   // block-uniform
+    __syncthreads();
+    if (!fits) {
+      // too many tiny segments for shared memory: single 16-byte groups, weights from global memory;
+      // thread t takes groups lo + t and lo + 256 + t so that a warp's loads stay contiguous
+      const long long lo = 2 * (num_pairs - (static_cast<long long>(blockIdx.x) + 1) * kPass2BlockPairs);
+      for (int g = 0; g < 2; ++g) {
+        const long long v = lo + threadIdx.x + g * kThreads;
+        if (v >= 0 && v < num_vec)
+          pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v, num_vec, tail_elems, seg_off, sg0, keep);
       }
-      for (; i0 < N; ++i0) {
-        uint4 x[2];
-        ld_stream_v8(col + static_cast<long long>(i0) * row_bytes, x[0], x[1]);
-        const float gm = g_s[i0];
-        const float2 g2 = make_float2(gm, gm);
-#pragma unroll
-        for (int g = 0; g < 2; ++g)
-#pragma unroll
-          for (int h = 0; h < NP; ++h) acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[g], h), g2, acc[g][h]);
-      }
-      if (tail_elems != 0 && v0 + 1 == num_vec - 1) {          // the row's last group is partial
-        pass2_store<DT, NP>(out, v0, acc[0], keep);
-        pass2_store_tail<DT, NP>(out, v0 + 1, acc[1], tail_elems);
-      } else {
-        st_global_v8(out + w * 32, pass2_pack<DT, NP>(acc[0]), pass2_pack<DT, NP>(acc[1]), keep);
-      }
+      return;
+    }
+    if (w < 0) return;
+    nseg = sg1 - sg0 + 1;
+    const long long d_cols = (num_vec - 1) * VEC + (tail_elems ? tail_elems : VEC);
+    const int sl = seg_find(off_s, nseg, v0 * VEC);
+    const long long c_last = (v0 * VEC + 2 * VEC < d_cols ? v0 * VEC + 2 * VEC : d_cols) - 1;
+    straddles = c_last >= off_s[sl + 1];
+    gw = g_s + sl * N;
+  }
+  if (SEG && straddles) {
+    for (int g = 0; g < 2; ++g)
+      if (v0 + g < num_vec)
+        pass2_mixed_vector_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, v0 + g, num_vec, tail_elems, keep);
+    return;
+  }
+  if (v0 + 1 < num_vec) {                            // the pair is complete (all but an odd row's last group)
+    float2 acc[2][NP];
+    pass2_wide_pair<DT, U>(grads + w * 32, gw, N, row_bytes, acc);
+    if (tail_elems != 0 && v0 + 1 == num_vec - 1) {            // the row's last group is partial
+      pass2_store<DT, NP>(out, v0, acc[0], keep);
+      pass2_store_tail<DT, NP>(out, v0 + 1, acc[1], tail_elems);
     } else {
-      pass2_single_vector<DT>(grads, out, g_s, N, row_bytes, v0, num_vec, tail_elems, keep);
+      st_global_v8(out + w * 32, pass2_pack<DT, NP>(acc[0]), pass2_pack<DT, NP>(acc[1]), keep);
     }
   } else {
-    // a block that spans a segment boundary works on single 16-byte groups; thread t takes groups
-    // lo + t and lo + 256 + t of the block's range so that a warp's loads stay contiguous
-    const long long lo = 2 * (num_pairs - (static_cast<long long>(blockIdx.x) + 1) * kPass2BlockPairs);
-    for (int g = 0; g < 2; ++g) {
-      const long long v = lo + threadIdx.x + g * kThreads;
-      if (v >= 0 && v < num_vec)
-        pass2_mixed_vector<DT>(grads, out, gamma, N, row_bytes, v, num_vec, tail_elems, seg_off, -code - 1, keep);
-    }
+    pass2_single_vector<DT>(grads, out, gw, N, row_bytes, v0, num_vec, tail_elems, keep);
   }
 }
 
@@ -1351,8 +1599,193 @@ fused_small_kernel(const FusedParams prm) {
   }
 }
 
+// ----------------------------------------------------------------------------------------------
+// One launch, two reads: pass 1, the coefficient step and pass 2 in ONE cooperative kernel, for
+// matrices too large for shared memory but small enough that two kernel boundaries and a third
+// launch are a visible share of the step (hundreds of MB to a few GB).
+//   phase 1  exactly pass1_tma_kernel's loop; the block's partial goes to global memory.
+//   ticket   every block takes a ticket (integer atomic).  Nobody waits here: the block that draws
+//            the last ticket of the launch adds up all partials in index order (so the result does
+//            not depend on who came last), runs Eq. 7 / 11 / 12-13 and publishes the weights with
+//            a release store of the launch's generation number.
+//   phase 2  the other blocks poll that word (bounded, 2 s), then all blocks form
+//            sum_i gamma_i g_i for the 8 KB-per-row column ranges b, b + grid, ... counted from the
+//            END of the vector -- the columns phase 1 read last come first -- with the loop, the
+//            row order and the rounding of pass2_wide_kernel, so the output bytes are the same.
+// The launch is cooperative (all blocks resident), the grid is phase 1's.  sync[0] is the ticket
+// counter, sync[1] the published generation; both only grow, a launch owns tickets
+// [gen * grid, (gen + 1) * grid), so the kernel can be replayed from a CUDA graph.
+// ----------------------------------------------------------------------------------------------
+// One thread waits until a monotonically growing word in global memory reaches `want` (written
+// with a release store by another block of the same launch), for at most kWaitLimitNs.
+__device__ __forceinline__ bool wait_generation_bounded(const unsigned long long* word, unsigned long long want, uint32_t* flags) {
+  const unsigned long long t0 = global_timer_ns();
+  bool ok = true;
+  for (;;) {
+    unsigned long long cur;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(cur) : "l"(word) : "memory");
+    if (cur >= want) break;
+    if (global_timer_ns() - t0 > kWaitLimitNs) { ok = false; atomicOr(flags, kFlagTimeout); break; }
+  }
+  __threadfence();
+  return ok;
+}
+
+struct MidParams {
+  Pass1Params p1;
+  CoeffParams coeff;               // sets = 1, partials = p1.partials, num_partials = gridDim.x
+  const unsigned char* grads;
+  unsigned char* out;
+  long long row_bytes;
+  long long num_vec;               // 16-byte column groups per row (the last may be partial)
+  int tail_elems;
+  int keep_in_l2;                  // the result fits in L2: store it evict_last
+  unsigned long long* sync;        // [0] tickets drawn, [1] generations published
+};
+
+constexpr int kMidPartCap = 2 * kMaxN;   // as coeff_kernel (1024 threads): the same summation order, the same bits
+constexpr int kMidRows = 8;        // rows in flight per thread in phase 2
+
+template <int DT, int NR, int WR>
+__global__ void __launch_bounds__(kThreads, 2)
+mid_fused_kernel(const __grid_constant__ CUtensorMap tmap, const MidParams prm) {
+  using C = P1<DT, NR, WR>;
+  constexpr int NP = Elem<DT>::kVec / 2;
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int s_abort;
+  __shared__ int s_role;                       // 0 = waits for the weights, 1 = computes them, -1 = gave up
+  __shared__ unsigned long long s_gen;
+  __shared__ float g_s[kMaxFastN];
+  const Pass1Params& p1 = prm.p1;
+  const int N = p1.N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int cw = warp / WR, rw = warp % WR;
+  const P1Smem sm = p1_carve<C>(smem_raw, p1.stages, p1.stage_bytes);
+
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < p1.stages; ++s) mbar_init(&sm.full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+
+  // ---- phase 1 (Eq. 7): as pass1_tma_kernel
+  const int first = blockIdx.x;
+  const int stride = gridDim.x;
+  const int my_tiles = first < p1.num_tiles ? (p1.num_tiles - first + stride - 1) / stride : 0;
+  auto issue = [&](int k, int s) {
+    const int col0 = (first + k * stride) * C::TILEC;
+    mbar_expect_tx(&sm.full[s], p1.stage_bytes);
+#pragma unroll
+    for (int c = 0; c < C::WC; ++c)
+      tma_load_2d(sm.stage_base + static_cast<size_t>(s) * p1.stage_bytes + static_cast<size_t>(c) * N * kBoxRowBytes,
+                  &tmap, &sm.full[s], col0 + c * C::BOXC, 0);
+  };
+  int issued = 0;
+  if (tid == 0) {
+    const int pre = my_tiles < p1.stages ? my_tiles : p1.stages;
+    for (int k = 0; k < pre; ++k) issue(k, k);
+    issued = pre;
+  }
+  float2 pacc[NR], qacc[NR];
+#pragma unroll
+  for (int j = 0; j < NR; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  p1_outer_clear<C>(sm.outer);
+  {
+    int s = 0;
+    uint32_t parity = 0;
+    for (int k = 0; k < my_tiles; ++k) {
+      uint4 v[NR];
+      if (mbar_wait_bounded(&sm.full[s], parity)) {
+        p1_load_rows<C>(v, sm.stage_base + static_cast<size_t>(s) * p1.stage_bytes +
+                               static_cast<size_t>(cw) * N * kBoxRowBytes + lane * 16, rw, N);
+      } else {
+#pragma unroll
+        for (int j = 0; j < NR; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
+        atomicOr(&s_abort, 1);
+      }
+      float2 sp[C::NP];
+      p1_colsum<DT, C>(v, sp);
+      float* xbuf = p1_xch_buffer<C>(sm.xch, k);
+      if (WR > 1) p1_xch_write<C>(xbuf, sp, rw, cw, lane);
+      __syncthreads();
+      if (s_abort) break;
+      if (tid == 0 && k + p1.stages < my_tiles) {
+        fence_proxy_async_smem();
+        issue(k + p1.stages, s);
+        issued = k + p1.stages + 1;
+      }
+      p1_xch_finish<C>(sm.xch, k, sp, cw, lane);
+      p1_accumulate<DT, C>(v, sp, pacc, qacc);
+      if ((k & (kFoldTiles - 1)) == kFoldTiles - 1) p1_fold<C>(pacc, qacc, sm.outer);
+      if (++s == p1.stages) { s = 0; parity ^= 1u; }
+    }
+  }
+  float* dst = p1.partials + static_cast<size_t>(blockIdx.x) * 2 * N;
+  const bool aborted = s_abort != 0;           // block-uniform (read after the loop's barrier)
+  if (aborted) {
+    if (tid == 0) p1_drain_after_timeout(sm.full, p1.stages, issued, p1.flags);
+    if (tid < 2 * N) dst[tid] = 0.f;
+    __syncthreads();
+  } else {
+    p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst, dst + N, N);   // ends with a barrier
+  }
+
+  // ---- ticket; the last block of the launch computes the weights (Eq. 7, 11, 12-13)
+  if (tid == 0) {
+    __threadfence();                                            // this block's partial is visible ...
+    const unsigned long long t = atomicAdd(&prm.sync[0], 1ull); // ... before its ticket is
+    s_gen = t / gridDim.x;
+    s_role = ((t + 1ull) % gridDim.x == 0ull) ? 1 : 0;
+    __threadfence();
+  }
+  __syncthreads();
+  if (s_role == 1) {
+    // every copy into this block's ring has landed, so the ring is free to hold the work arrays
+    double* work = reinterpret_cast<double*>(smem_raw);
+    coeff_core(prm.coeff, 0, work, kMidPartCap, kMaxN, work + kMidPartCap, work + kMidPartCap + kMaxFastN);
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      const unsigned long long g = s_gen + 1ull;
+      asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(prm.sync + 1), "l"(g) : "memory");
+    }
+  } else if (tid == 0) {
+    if (!wait_generation_bounded(prm.sync + 1, s_gen + 1ull, p1.flags)) s_role = -1;
+  }
+  __syncthreads();
+  if (s_role < 0 || aborted) return;
+  if (tid < N) g_s[tid] = __ldcg(prm.coeff.gamma_f32 + tid);
+  __syncthreads();
+
+  // ---- phase 2 (Eq. 12): pass2_wide_kernel's block b for b = blockIdx.x, blockIdx.x + grid, ...
+  const unsigned long long keep = prm.keep_in_l2 ? l2_policy_evict_last() : 0ull;
+  const long long num_vec = prm.num_vec;
+  const long long num_pairs = (num_vec + 1) / 2;
+  const long long blocks2 = (num_pairs + kPass2BlockPairs - 1) / kPass2BlockPairs;
+  for (long long b = blockIdx.x; b < blocks2; b += gridDim.x) {
+    const long long w = num_pairs - (b + 1) * kPass2BlockPairs + tid;
+    if (w < 0) continue;
+    const long long v0 = 2 * w;
+    if (v0 + 1 < num_vec) {
+      float2 acc[2][NP];
+      pass2_wide_pair<DT, kMidRows>(prm.grads + w * 32, g_s, N, prm.row_bytes, acc);
+      if (prm.tail_elems != 0 && v0 + 1 == num_vec - 1) {
+        pass2_store<DT, NP>(prm.out, v0, acc[0], keep);
+        pass2_store_tail<DT, NP>(prm.out, v0 + 1, acc[1], prm.tail_elems);
+      } else {
+        st_global_v8(prm.out + w * 32, pass2_pack<DT, NP>(acc[0]), pass2_pack<DT, NP>(acc[1]), keep);
+      }
+    } else {
+      pass2_single_vector<DT>(prm.grads, prm.out, g_s, N, prm.row_bytes, v0, num_vec, prm.tail_elems, keep);
+    }
+  }
+}
+
 // Self-test of the bounded waits (no data path): which = 0 waits on an mbarrier that nobody arrives
-// on, which = 1 on a grid barrier that expects one more block than exists.  Both give up after
+// on, which = 1 on a grid barrier that expects one more block than exists, which = 2 on a
+// generation word that nobody advances.  All give up after
 // kWaitLimitNs, raise the time-out flag and return; the context stays usable.
 __global__ void selftest_wait_kernel(int which, unsigned long long* barrier, uint32_t* flags) {
   __shared__ __align__(8) uint64_t bar;
@@ -1363,8 +1796,11 @@ __global__ void selftest_wait_kernel(int which, unsigned long long* barrier, uin
     }
     __syncthreads();
     if (threadIdx.x == 0 && !mbar_wait_bounded(&bar, 0u)) atomicOr(flags, kFlagTimeout);
-  } else {
+  } else if (which == 1) {
     (void)grid_barrier_bounded(barrier, gridDim.x + 1u, flags);
+  } else {
+    // the one-launch kernel's wait for the weights: a generation that nobody publishes
+    if (threadIdx.x == 0) (void)wait_generation_bounded(barrier + 2, barrier[2] + 1ull, flags);
   }
 }
 
@@ -1372,7 +1808,10 @@ __global__ void reset_kernel(double* m, long long n, uint32_t* flags, long long*
   for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < n;
        i += static_cast<long long>(gridDim.x) * blockDim.x)
     m[i] = 0.0;
-  if (blockIdx.x == 0 && threadIdx.x == 0) { *flags = 0u; *step = 0; *barrier = 0ull; }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    *flags = 0u; *step = 0;
+    barrier[0] = 0ull; barrier[1] = 0ull; barrier[2] = 0ull;    // grid barrier; ticket counter and generation of the one-launch kernel
+  }
 }
 
 }  // namespace adacons

@@ -14,7 +14,7 @@ from paper_2411_03742_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("which", [0, 1], ids=["mbarrier", "grid-barrier"])
+@pytest.mark.parametrize("which", [0, 1, 2], ids=["mbarrier", "grid-barrier", "published-weights"])
 def test_unsatisfiable_wait_times_out_and_context_survives(which):
     from paper_2411_03742_b200 import binding as ac
     w = wl.Workload("bw", 6, 40_000, "f32", 1, "gauss", seed=8)
@@ -33,11 +33,13 @@ def test_unsatisfiable_wait_times_out_and_context_survives(which):
     assert h.status() & ac.FLAG_TIMEOUT
     h.reset()
     assert h.status() == 0
-    for fused in (1, 0):                                    # both paths still work, incl. the grid barrier
+    for fused, one_launch, path in ((1, 0, 3), (0, 2, 5), (0, 0, 1)):   # every path still works, incl. its waits
         h.set_option(ac.OPT_FUSED_SMALL, fused)
+        h.set_option(ac.OPT_ONE_LAUNCH, one_launch)
         h.reset()
         h.aggregate(G, out)
         torch.cuda.synchronize()
+        assert h.info(ac.INFO_LAST_PATH) == path
         res = oc.AdaConsOracle(w.N, w.d).step(G.cpu().double().numpy())
         np.testing.assert_allclose(h.coeffs()[0], res["gamma"][0], rtol=1e-5)
         assert h.status() == 0

@@ -23,9 +23,10 @@ def ac():
 
 
 def run_case(ac, w, steps, *, beta=0.99, options=None, oracle_kw=None, offsets=None, per_segment=False,
-             fused=False, expect_path=None, allow_swaps=True, what=None):
+             fused=False, one_launch=0, expect_path=None, allow_swaps=True, what=None):
     """fused=False keeps small cases on the three-kernel path (the one the large workloads take);
     fused=True lets the library pick the single-pass kernel when the matrix fits in shared memory.
+    one_launch: ADACONS_OPT_ONE_LAUNCH (0 = three kernels, 2 = the one-launch kernel whenever possible).
     allow_swaps=False: the recipe's coefficients are well separated, so the kernel's slot order
     must be the oracle's on every step (no near-tie rule)."""
     what = what or w.name
@@ -33,6 +34,7 @@ def run_case(ac, w, steps, *, beta=0.99, options=None, oracle_kw=None, offsets=N
     oracle_kw = dict(oracle_kw or {})
     h = ac.AdaCons(w.N, w.d, w.dtype, seg_offsets=offsets)
     h.set_option(ac.OPT_FUSED_SMALL, 1 if fused else 0)
+    h.set_option(ac.OPT_ONE_LAUNCH, one_launch)
     if per_segment:
         h.set_option(ac.OPT_PER_SEGMENT, 1)
         oracle_kw.update(seg_offsets=offsets, per_segment=True)
@@ -106,9 +108,81 @@ def test_full_step_recipe(ac, name, d, per_segment):
              allow_swaps=(name != "mixed16"), what=f"{w.name} recipe" + (" per segment" if per_segment else ""))
 
 
-def test_config2_full_size_three_steps(ac):
+@pytest.mark.parametrize("one_launch", [0, 2], ids=["three-kernels", "one-launch"])
+def test_config2_full_size_three_steps(ac, one_launch):
     w = wl.WORKLOADS["resnet8"]
-    run_case(ac, w, 3)
+    run_case(ac, w, 3, one_launch=one_launch, expect_path=5 if one_launch else 1)
+
+
+# ---- the one-launch kernel (pass 1, coefficient step by the last block, pass 2) ------------------
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N", [1, 2, 3, 4, 5, 7, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64])
+def test_one_launch_all_worker_counts(ac, N, dtype):
+    w = wl.Workload(f"ol{N}", N, 200_016, dtype, 3, "gauss", seed=250 + N)
+    run_case(ac, w, 3, beta=0.7, one_launch=2, expect_path=5)
+
+
+@pytest.mark.parametrize("name,d,steps", [("resnet8", 1_000_016, 6), ("mixed16", 1_200_016, 5), ("bert64", 400_016, 4),
+                                          ("ragged32", 1_000_008, 4)])
+def test_one_launch_scaled_configs(ac, name, d, steps):
+    w = wl.WORKLOADS[name].scaled(d)
+    run_case(ac, w, steps, one_launch=2, expect_path=5, allow_swaps=(name != "mixed16"), what=f"{w.name} one launch")
+
+
+def test_one_launch_default_by_size_and_alignment(ac):
+    """By default the one-launch kernel serves what does not fit in shared memory, up to 1 GiB, on
+    32-byte aligned buffers; per-segment mode and 16-byte-only alignment keep the three kernels."""
+    dev = torch.device("cuda:0")
+    w = wl.Workload("olsel", 8, 2_000_000, "f32", 1, "gauss", seed=2)
+    G = wl.generate(w, 0, dev)
+    out = torch.empty(w.d + 8, device=dev)
+    h = ac.AdaCons(w.N, w.d, "f32")
+    assert h.get_option(ac.OPT_ONE_LAUNCH) == 1
+    h.aggregate(G, out[:w.d])
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 5 and h.info(ac.INFO_LAUNCHES_PER_CALL) == 1 and h.info(ac.INFO_LAST_PASS2) == 3
+    h.aggregate(G, out[4:w.d + 4])                     # out is 16 but not 32 bytes aligned
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 1 and h.info(ac.INFO_LAUNCHES_PER_CALL) == 3 and h.info(ac.INFO_LAST_PASS2) == 2
+    h.set_option(ac.OPT_ONE_LAUNCH, 0)
+    h.aggregate(G, out[:w.d])
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 1
+    with pytest.raises(ac.AdaConsError):
+        h.set_option(ac.OPT_ONE_LAUNCH, 3)
+    h2 = ac.AdaCons(w.N, w.d, "f32", seg_offsets=[0, 1000, w.d])
+    h2.set_option(ac.OPT_PER_SEGMENT, 1)
+    h2.aggregate(G, out[:w.d])
+    torch.cuda.synchronize()
+    assert h2.info(ac.INFO_LAST_PATH) == 1
+
+
+@pytest.mark.parametrize("N,d,dtype", [(8, 3_000_000, "f32"), (64, 500_000, "bf16"), (16, 1_500_016, "bf16"), (32, 700_000, "f32")])
+def test_one_launch_gives_the_bytes_of_the_three_kernel_path(ac, N, d, dtype):
+    """Both paths add the same block partials in the same order and share pass 2's arithmetic: the
+    coefficients, the state and the output are bit-identical over several steps with momentum."""
+    dev = torch.device("cuda:0")
+    w = wl.Workload("olbits", N, d, dtype, 3, "gauss_outlier", seed=N)
+    Gs = [wl.generate(w, t, dev) for t in range(3)]
+    runs = []
+    for mode in (0, 2, 2):
+        h = ac.AdaCons(N, d, dtype)
+        h.set_option(ac.OPT_FUSED_SMALL, 0)
+        h.set_option(ac.OPT_ONE_LAUNCH, mode)
+        out = torch.empty(d, dtype=w.torch_dtype, device=dev)
+        outs = []
+        for G in Gs:
+            h.aggregate(G, out)
+            outs.append(out.clone())
+        torch.cuda.synchronize()
+        assert h.info(ac.INFO_LAST_PATH) == (5 if mode else 1) and h.status() == 0
+        runs.append((outs, [h.coeffs(k).copy() for k in range(5)], h.state()[0].copy()))
+    for other in runs[1:]:
+        for a, b in zip(runs[0][0], other[0]):
+            assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+        for a, b in zip(runs[0][1], other[1]):
+            assert a.tobytes() == b.tobytes()
+        assert runs[0][2].tobytes() == other[2].tobytes()
 
 
 # ---- every pass-1 instantiation, masked rows, both types ---------------------------------------
@@ -141,18 +215,19 @@ def test_single_pass_kernel_is_not_used_when_the_matrix_does_not_fit(ac):
 
 
 def test_single_pass_and_three_kernel_paths_share_state(ac):
-    """Switching between the two paths mid-run continues the same momentum state."""
-    w = wl.Workload("mix", 12, 50_000, "f32", 4, "gauss", seed=33)
+    """Switching between the three paths mid-run continues the same momentum state."""
+    w = wl.Workload("mix", 12, 50_000, "f32", 6, "gauss", seed=33)
     dev = "cuda:0"
     h = ac.AdaCons(w.N, w.d, "f32")
     orc = oc.AdaConsOracle(w.N, w.d)
     out = torch.empty(w.d, device=dev)
-    for t in range(4):
-        h.set_option(ac.OPT_FUSED_SMALL, t % 2)
+    for t in range(6):
+        h.set_option(ac.OPT_FUSED_SMALL, 1 if t % 3 == 1 else 0)
+        h.set_option(ac.OPT_ONE_LAUNCH, 2 if t % 3 == 2 else 0)
         G = wl.generate(w, t, dev)
         h.aggregate(G, out)
         torch.cuda.synchronize()
-        assert h.info(ac.INFO_LAST_PATH) == (3 if t % 2 else 1)
+        assert h.info(ac.INFO_LAST_PATH) == (1, 3, 5)[t % 3]
         res = oracle_step(orc, to_f64(G), "f32", h.coeffs(ac.COEFF_A), what="paths share state")
         assert_coeffs(h.coeffs(), res["gamma"], f"gamma step {t}")
         assert_coeffs(h.state()[0], res["m"], f"m step {t}")
@@ -170,8 +245,13 @@ def test_path_selection_and_launch_counts(ac):
     h.set_option(ac.OPT_FUSED_SMALL, 0)
     h.aggregate(G, out)
     torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 5                      # too large for shared memory by decree: one launch, two reads
+    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 1 and h.info(ac.INFO_TOTAL_LAUNCHES) == 2
+    h.set_option(ac.OPT_ONE_LAUNCH, 0)
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
     assert h.info(ac.INFO_LAST_PATH) == 1
-    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 3 and h.info(ac.INFO_TOTAL_LAUNCHES) == 4
+    assert h.info(ac.INFO_LAUNCHES_PER_CALL) == 3 and h.info(ac.INFO_TOTAL_LAUNCHES) == 5
 
 
 # ---- generic path: odd lengths, misaligned pointers, many workers ------------------------------
@@ -223,6 +303,7 @@ def test_generic_and_fast_paths_agree(ac):
     o0, o1 = torch.empty(d, device="cuda:0", dtype=torch.bfloat16), torch.empty(d, device="cuda:0", dtype=torch.bfloat16)
     h0, h1 = ac.AdaCons(N, d, "bf16"), ac.AdaCons(N, d, "bf16")
     h0.set_option(ac.OPT_FUSED_SMALL, 0)
+    h0.set_option(ac.OPT_ONE_LAUNCH, 0)
     h0.aggregate(G0, o0); h1.aggregate(G1, o1)
     torch.cuda.synchronize()
     assert (h0.info(ac.INFO_LAST_PATH), h1.info(ac.INFO_LAST_PATH)) == (1, 2)
@@ -492,7 +573,7 @@ def full_size_case(ac, name, steps, *, per_segment=False, need_gb=60, allow_swap
         G = wl.generate(w, t, dev, out=G)
         h.aggregate(G, out)
         torch.cuda.synchronize()
-        assert h.info(ac.INFO_LAST_PATH) == 1 and h.status() == 0
+        assert h.info(ac.INFO_LAST_PATH) == (1 if per_segment or w.N * w.d * w.elem_bytes > 1 << 30 else 5) and h.status() == 0
         if per_segment:
             with ThreadPoolExecutor(max_workers=8) as ex:
                 stats = list(ex.map(lambda s_: oc.consensus_statistics(to_f64(G[:, bounds[s_]:bounds[s_ + 1]])), range(S)))
@@ -563,26 +644,41 @@ def test_config3_full_size(ac):
 @pytest.mark.parametrize("N", [512, 600, 1024])
 def test_many_workers(ac, N):
     w = wl.Workload(f"many{N}", N, 3_000, "f32", 2, "gauss", seed=N)
-    run_case(ac, w, 2, beta=0.9, expect_path=4)
+    run_case(ac, w, 2, beta=0.9, expect_path=6 if N <= 512 else 4)
     w = wl.Workload(f"manyodd{N}", N, 3_001, "f32", 2, "gauss", seed=N)      # unaligned: generic path
     run_case(ac, w, 2, beta=0.9, expect_path=2)
 
 
 @pytest.mark.parametrize("N,d,dtype", [(65, 400_008, "bf16"), (100, 300_004, "f32"), (128, 500_000, "bf16"),
-                                       (200, 150_000, "f32"), (257, 100_008, "bf16")])
-def test_more_than_64_workers_column_sum_then_dot_path(ac, N, d, dtype):
-    """N > 64 on aligned buffers: column sums to scratch, then one dot-product launch per 64 rows
-    (the last chunk is ragged)."""
-    w = wl.Workload(f"big{N}", N, d, dtype, 2, "gauss", seed=N)
-    h = run_case(ac, w, 2, beta=0.8, expect_path=4)
+                                       (129, 200_000, "bf16"), (200, 150_000, "f32"), (257, 100_008, "bf16"),
+                                       (448, 60_000, "bf16"), (512, 50_000, "f32")])
+@pytest.mark.parametrize("cluster", [1, 0], ids=["clusters-one-read", "column-sums-then-dots"])
+def test_more_than_64_workers(ac, N, d, dtype, cluster):
+    """N > 64 on aligned buffers.  Default for N <= 512: a thread-block cluster of 2, 4 or 8 blocks
+    shares each column tile (64 rows per block, the last block's rows ragged or absent) and pass 1
+    reads the matrix once.  Otherwise: column sums to scratch, then one dot-product launch per 64
+    rows."""
+    w = wl.Workload(f"big{N}", N, d, dtype, 3, "gauss", seed=N)
+    run_case(ac, w, 3, beta=0.8, options={ac.OPT_CLUSTER_PASS1: cluster}, expect_path=6 if cluster else 4)
 
 
-def test_more_than_64_workers_with_padded_rows(ac):
-    _padded_case(ac, 96, 123_457, "bf16", 123_464, 2, fused=False, expect_path=4)
+@pytest.mark.parametrize("N,dtype", [(128, "f32"), (128, "bf16"), (96, "bf16"), (300, "f32")])
+def test_cluster_pass1_many_tiles_per_cluster(ac, N, dtype):
+    """Long enough that every cluster walks many tiles (the double-buffered exchange of the partial
+    column sums wraps around many times) and the last tile is ragged."""
+    w = wl.Workload(f"cl{N}", N, 2_000_008, dtype, 2, "student_flip", seed=N)
+    run_case(ac, w, 2, beta=0.9, expect_path=6)
+
+
+@pytest.mark.parametrize("cluster", [1, 0])
+def test_more_than_64_workers_with_padded_rows(ac, cluster):
+    _padded_case(ac, 96, 123_457, "bf16", 123_464, 2, fused=False, options={ac.OPT_CLUSTER_PASS1: cluster},
+                 expect_path=6 if cluster else 4)
 
 
 # ---- the call neither allocates nor synchronises: it can be recorded once and replayed -----------
-def test_replay_from_a_cuda_graph_advances_the_state(ac):
+@pytest.mark.parametrize("one_launch", [0, 2], ids=["three-kernels", "one-launch"])
+def test_replay_from_a_cuda_graph_advances_the_state(ac, one_launch):
     w = wl.Workload("graph", 16, 600_000, "bf16", 3, "gauss", seed=123)
     dev = torch.device("cuda:0")
     G = wl.generate(w, 0, dev)
@@ -590,6 +686,7 @@ def test_replay_from_a_cuda_graph_advances_the_state(ac):
     out = torch.empty(w.d, dtype=torch.bfloat16, device=dev)
     h = ac.AdaCons(w.N, w.d, "bf16")
     h.set_option(ac.OPT_FUSED_SMALL, 0)
+    h.set_option(ac.OPT_ONE_LAUNCH, one_launch)
     static_G.copy_(G)
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -611,12 +708,12 @@ def test_replay_from_a_cuda_graph_advances_the_state(ac):
         assert_coeffs(h.coeffs(), res["gamma"], f"gamma replay {t}")
         assert_coeffs(h.state()[0], res["m"], f"m replay {t}")
         assert_output(out, res, to_f64(static_G), "bf16", f"replay {t}")
-    assert h.state()[1] == 3
+    assert h.state()[1] == 3 and h.info(ac.INFO_LAST_PATH) == (5 if one_launch else 1) and h.status() == 0
 
 
 # ---- padded rows: any gradient length on the fast paths ------------------------------------------
 def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=None, per_segment=False, expect_path=None,
-                 expect_pass2=None, out_shift=0):
+                 expect_pass2=None, out_shift=0, one_launch=0):
     """Rows live in an N x pitch buffer whose padding is NaN; the result buffer is followed by a
     sentinel.  Neither may influence, or be touched by, the aggregation."""
     dev = torch.device("cuda:0")
@@ -628,6 +725,7 @@ def _padded_case(ac, N, d, dtype, pitch, steps, *, fused, options=None, offsets=
     h = ac.AdaCons(N, d, dtype, seg_offsets=offsets)
     h.set_option(ac.OPT_ROW_PITCH, pitch)
     h.set_option(ac.OPT_FUSED_SMALL, 1 if fused else 0)
+    h.set_option(ac.OPT_ONE_LAUNCH, one_launch)
     oracle_kw = {}
     if per_segment:
         h.set_option(ac.OPT_PER_SEGMENT, 1)
@@ -694,6 +792,14 @@ def test_pass2_vector_widths(ac, N, dtype, d, pitch, shift, kernel):
     bytes otherwise; both kernels share one block-to-column mapping.  Every combination of an odd or
     even number of 16-byte groups with a full or partial last group, on both kernels."""
     _padded_case(ac, N, d, dtype, pitch, 2, fused=False, expect_path=1, expect_pass2=kernel, out_shift=shift)
+
+
+@pytest.mark.parametrize("dtype,d,pitch,shift,kernel", [c for c in PASS2_WIDTH_CASES if c[4] == 3])
+@pytest.mark.parametrize("N", [3, 13, 40])
+def test_one_launch_padded_rows_and_tails(ac, N, dtype, d, pitch, shift, kernel):
+    """The one-launch kernel on every tail shape of the 32-byte pass 2 (odd or even number of 16-byte
+    groups, full or partial last group, less than one block), NaN padding and a guarded result."""
+    _padded_case(ac, N, d, dtype, pitch, 2, fused=False, one_launch=2, expect_path=5, expect_pass2=3, out_shift=shift)
 
 
 @pytest.mark.parametrize("dtype,d,pitch,shift,kernel", [c for c in PASS2_WIDTH_CASES if c[1] >= 100_000])
@@ -781,6 +887,7 @@ def test_two_contexts_on_two_streams_are_independent(ac):
     def alone(w, Gs, dtype):
         h = ac.AdaCons(w.N, w.d, dtype)
         h.set_option(ac.OPT_FUSED_SMALL, 0)
+        h.set_option(ac.OPT_ONE_LAUNCH, 0)
         out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
         outs = []
         for G in Gs:
@@ -794,6 +901,7 @@ def test_two_contexts_on_two_streams_are_independent(ac):
     sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
     ha, hb = ac.AdaCons(wa.N, wa.d, "bf16"), ac.AdaCons(wb.N, wb.d, "f32")
     ha.set_option(ac.OPT_FUSED_SMALL, 0); hb.set_option(ac.OPT_FUSED_SMALL, 0)
+    ha.set_option(ac.OPT_ONE_LAUNCH, 0); hb.set_option(ac.OPT_ONE_LAUNCH, 0)    # two cooperative kernels cannot share the GPU
     oa = [torch.empty(wa.d, dtype=torch.bfloat16, device=dev) for _ in range(3)]
     ob = [torch.empty(wb.d, device=dev) for _ in range(3)]
     torch.cuda.synchronize()
@@ -825,8 +933,8 @@ def test_contexts_of_other_shapes_do_not_disturb_an_existing_one(ac):
     # TMA-staged pass 1: N = 64 needs more shared memory per stage than N = 40
     big = wl.Workload("shape64", 64, 300_008, "bf16", 1, "gauss", seed=3)
     small = wl.Workload("shape40", 40, 200_000, "bf16", 1, "gauss", seed=4)
-    hb = ac.AdaCons(big.N, big.d, "bf16"); hb.set_option(ac.OPT_FUSED_SMALL, 0)
-    hs = ac.AdaCons(small.N, small.d, "bf16"); hs.set_option(ac.OPT_FUSED_SMALL, 0)
+    hb = ac.AdaCons(big.N, big.d, "bf16"); hb.set_option(ac.OPT_FUSED_SMALL, 0); hb.set_option(ac.OPT_ONE_LAUNCH, 0)
+    hs = ac.AdaCons(small.N, small.d, "bf16"); hs.set_option(ac.OPT_FUSED_SMALL, 0); hs.set_option(ac.OPT_ONE_LAUNCH, 0)
     Gb, Gs = wl.generate(big, 0, dev), wl.generate(small, 0, dev)
     check(hs, small, Gs)
     check(hb, big, Gb)
