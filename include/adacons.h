@@ -112,7 +112,7 @@ enum adacons_option {
                                   elements must be readable (and out must not overlap them).
                                   Setting it synchronises the device and may re-allocate scratch. */
   ADACONS_OPT_ONE_LAUNCH = 9,  /* 1 (default): a matrix of up to 1 GiB that does not fit in shared
-                                  memory, on 32-byte aligned buffers and pitch with N <= 64, is
+                                  memory, on 16-byte aligned buffers and pitch with N <= 64, is
                                   aggregated by ONE cooperative kernel (pass 1, the coefficient
                                   step of Algorithm 1 steps 2-3 by the block that finishes pass 1
                                   last, pass 2) instead of three launches: two reads of the
@@ -155,7 +155,8 @@ enum adacons_info {
   ADACONS_INFO_LAST_PASS2 = 7        /* pass-2 kernel of the most recent aggregate call: 0 = none
                                         (no call yet, or the single-pass kernel), 1 = generic,
                                         2 = 16-byte vectors, 3 = 32-byte vectors (grads, out and
-                                        the row pitch 32-byte aligned)                           */
+                                        the row pitch 32-byte aligned), 4 = the second phase of
+                                        the one-launch kernel (TMA-staged chunks of 8 rows)      */
 };
 
 /*

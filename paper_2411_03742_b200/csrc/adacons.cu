@@ -37,6 +37,10 @@ constexpr size_t kGenericSmemCap = static_cast<size_t>(kWarps) * kMaxN * 2 * siz
 // Largest matrix (bytes) that takes the one-launch kernel by default: beyond it two kernel
 // boundaries are a negligible share of the step and the separate kernels are at least as fast.
 constexpr long long kOneLaunchMaxBytes = 1ll << 30;
+// Ring depth of the one-launch kernel's second phase.  Two stages of 32 KB per block (two blocks per
+// SM) keep enough bytes in flight; a third made the phase 3-5 % slower on both mid-size workloads.
+constexpr int kMidStages2 = 2;
+static_assert(kMidStages2 >= 2 && kMidStages2 <= kMidMaxStages2, "the ring needs two stages: a stage's item fields are rewritten one barrier after they are read");
 
 bool set_smem_cap(const void* kernel, size_t cap) {
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(cap)) == cudaSuccess)
@@ -117,8 +121,11 @@ struct adacons_ctx {
 
   // one launch for mid-size matrices: pass 1, coefficient step and pass 2 in one cooperative kernel
   bool mid_available = false;
-  int mid_grid = 0;
+  int mid_grid = 0, mid_stages2 = 0;
+  size_t mid_smem = 0;
   const void* mid_kernel = nullptr;
+  CUtensorMap tmap_mid2;                // phase 2: boxes of min(N, 8) rows x 512 bytes
+  const void* tmap_mid2_for = nullptr;
   int one_launch = 1;                   // ADACONS_OPT_ONE_LAUNCH: 0 never, 1 by size, 2 whenever possible
 
   // per-segment ("layer-wise") plan, built when ADACONS_OPT_PER_SEGMENT is switched on
@@ -397,12 +404,22 @@ int plan_mid(adacons_ctx* c) {
     return ADACONS_OK;
   }
   const void* k = select_mid(c->dtype, c->fast.NR, c->fast.WR);
+  // phase 2 re-uses the dynamic shared memory as a ring of stages of 8 boxes x min(N, 8) rows x 512 bytes
+  const size_t stage2 = static_cast<size_t>(kWarps) * (c->N < kMidChunkRows ? c->N : kMidChunkRows) * kBoxRowBytes;
+  const int stages2 = kMidStages2;
+  size_t smem = c->fast.smem_bytes;
+  if (smem < stages2 * stage2) smem = stages2 * stage2;
+  const size_t work = (static_cast<size_t>(kMidPartCap) + 3 * kMaxFastN) * sizeof(double);   // the coefficient step's arrays
+  if (smem < work) smem = work;
   int per_sm = 0;
-  if (!set_smem_cap(k, kPass1SmemCap) ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, c->fast.smem_bytes) != cudaSuccess || per_sm < 1) {
+  if (smem > kPass1SmemCap || !set_smem_cap(k, kPass1SmemCap) ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, smem) != cudaSuccess || per_sm < 1) {
     cudaGetLastError();
     return ADACONS_OK;
   }
+  c->mid_stages2 = stages2;
+  c->mid_smem = smem;
+  c->tmap_mid2_for = nullptr;
   int grid = per_sm * c->num_sms;
   if (grid > c->fast.grid) grid = c->fast.grid;       // never more blocks than pass 1 would use (or than tiles)
   c->mid_grid = grid;
@@ -425,6 +442,24 @@ int encode_chunk_map(const adacons_ctx* c, const void* grads, int ch, CUtensorMa
                                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? ADACONS_OK : ADACONS_ECUDA;
+}
+
+// Tensor map of the one-launch kernel's second phase: the same matrix, boxes of min(N, 8) rows.
+int encode_map_mid2(adacons_ctx* c, const void* grads) {
+  if (c->tmap_mid2_for == grads) return ADACONS_OK;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes),
+                             static_cast<cuuint32_t>(c->N < kMidChunkRows ? c->N : kMidChunkRows)};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = c->encode(&c->tmap_mid2,
+                               c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                               2, const_cast<void*>(grads), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  c->tmap_mid2_for = grads;
+  return ADACONS_OK;
 }
 
 // All chunk maps of a context (its vector was sized when the plan was made).
@@ -736,11 +771,12 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     return ADACONS_OK;
   }
 
-  // ---- one launch, two reads: mid-size matrices on 32-byte aligned buffers ----
-  if (!seg && aligned && c->mid_available && (g0 % 32 == 0) && (o0 % 32 == 0) && (row_bytes % 32 == 0) &&
+  // ---- one launch, two reads: mid-size matrices ----
+  if (!seg && aligned && c->mid_available &&
       (c->one_launch == 2 ||
        (c->one_launch == 1 && static_cast<long long>(c->N) * row_bytes <= kOneLaunchMaxBytes))) {
     int rc = encode_map(c, grads);
+    if (rc == ADACONS_OK) rc = encode_map_mid2(c, grads);
     if (rc != ADACONS_OK) return rc;
     MidParams mp;
     mp.p1.N = N; mp.p1.num_tiles = c->fast.num_tiles; mp.p1.stages = c->fast.stages; mp.p1.stage_bytes = c->fast.stage_bytes;
@@ -753,15 +789,16 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     mp.grads = static_cast<const unsigned char*>(grads); mp.out = static_cast<unsigned char*>(out);
     mp.row_bytes = row_bytes; mp.num_vec = num_vec; mp.tail_elems = tail_elems;
     mp.keep_in_l2 = static_cast<long long>(obytes) <= c->l2_bytes ? 1 : 0;
+    mp.stages2 = c->mid_stages2;
     mp.sync = c->d_barrier + 1;
-    void* args[2] = {&c->tmaps[0], &mp};
-    if (cudaLaunchCooperativeKernel(c->mid_kernel, dim3(c->mid_grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
+    void* args[3] = {&c->tmaps[0], &c->tmap_mid2, &mp};
+    if (cudaLaunchCooperativeKernel(c->mid_kernel, dim3(c->mid_grid), dim3(kThreads), args, c->mid_smem, st) != cudaSuccess) {
       cudaGetLastError();
       return ADACONS_ECUDA;
     }
     if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); cudaEventRecord(ev[3], st); c->prof_calls += 1; }
     c->last_path = 5;
-    c->last_pass2 = 3;
+    c->last_pass2 = 4;
     c->last_launches = 1;
     c->total_launches += 1;
     return ADACONS_OK;
@@ -998,6 +1035,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
       c->pitch = pitch;
       c->tmap_for = nullptr;
+      c->tmap_mid2_for = nullptr;
       int rc = plan_fast(c);
       if (rc != ADACONS_OK) return rc;
       c->tmaps.resize(static_cast<size_t>(c->num_chunks));

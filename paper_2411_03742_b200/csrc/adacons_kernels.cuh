@@ -910,12 +910,12 @@ struct CoeffParams {
   long long* step;       // aggregation counter
 };
 
-// Work arrays in shared memory: sh_part holds part_cap doubles (at least 2N), sh_a and sh_u N each.
+// Work arrays in shared memory: sh_part holds part_cap doubles (at least 2N), sh_a, sh_u and sh_m N each.
 // The records are split into `groups` interleaved subsequences, which fixes the order of the fp64
 // sum; groups follows from N, part_cap and group_threads alone (not from the block size), so two
 // kernels that pass the same values add the same records in the same order.
 __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set, double* sh_part, const int part_cap,
-                                           const int group_threads, double* sh_a, double* sh_u) {
+                                           const int group_threads, double* sh_a, double* sh_u, double* sh_m) {
   __shared__ int sh_bad, sh_zero;
   __shared__ double sh_Z;
   __shared__ int sh_uniform;
@@ -923,6 +923,7 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
   const int V = 2 * N;
   const size_t per = static_cast<size_t>(prm.sets) * N;   // stride between coefficient kinds
   if (i == 0) { sh_bad = 0; sh_zero = 0; }
+  if (i < N) sh_m[i] = prm.m[static_cast<size_t>(set) * N + i];   // the old state, fetched while the partials are summed
   const int begin = prm.rec_begin ? prm.rec_begin[set] : 0;
   const int count = prm.rec_count ? prm.rec_count[set] : prm.num_partials;
   const float* base = prm.partials + static_cast<size_t>(begin) * V;
@@ -939,8 +940,19 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
     double acc[4] = {0.0, 0.0, 0.0, 0.0};
     const float* src = base + static_cast<size_t>(u) * w;
     if (w == 4) {
-#pragma unroll 4
-      for (int c = g; c < count; c += groups) {
+      // eight records in flight, added in record order (the latency of a round trip to L2 is what this step costs)
+      int c = g;
+      for (; c + 7 * groups < count; c += 8 * groups) {
+        float4 x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = __ldcg(reinterpret_cast<const float4*>(src + static_cast<size_t>(c + j * groups) * V));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          acc[0] += static_cast<double>(x[j].x); acc[1] += static_cast<double>(x[j].y);
+          acc[2] += static_cast<double>(x[j].z); acc[3] += static_cast<double>(x[j].w);
+        }
+      }
+      for (; c < count; c += groups) {
         const float4 x = __ldcg(reinterpret_cast<const float4*>(src + static_cast<size_t>(c) * V));
         acc[0] += static_cast<double>(x.x); acc[1] += static_cast<double>(x.y);
         acc[2] += static_cast<double>(x.z); acc[3] += static_cast<double>(x.w);
@@ -983,7 +995,7 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
     if (i == 0) {
       atomicOr(prm.flags, flags | kFlagNonfinite);
       prm.z[set] = __longlong_as_double(0x7ff8000000000000ll);
-      if (set == 0) *prm.step += 1;
+      if (set == 0) atomicAdd(reinterpret_cast<unsigned long long*>(prm.step), 1ull);   // no round trip
     }
     return;
   }
@@ -1001,10 +1013,9 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
         rank += (aj < a || (aj == a && j < i)) ? 1 : 0;
       }
     }
-    double* slot = prm.m + static_cast<size_t>(set) * N + rank;
     // spelled out so that every kernel this is inlined into rounds the same way (one product, one fused step)
-    at = __fma_rn(prm.beta, *slot, __dmul_rn(1.0 - prm.beta, a));   // exactly one writer per slot
-    *slot = at;
+    at = __fma_rn(prm.beta, sh_m[rank], __dmul_rn(1.0 - prm.beta, a));
+    prm.m[static_cast<size_t>(set) * N + rank] = at;              // exactly one writer per slot
   }
   const double u = q > 0.0 ? at / rq : 0.0;                      // unit-column P: weight on raw g_i
   if (i < N) sh_u[i] = u;
@@ -1020,7 +1031,7 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
       else if (Z < 0.0) flags |= kFlagNegZ;
     }
     if (flags) atomicOr(prm.flags, flags);
-    if (set == 0) *prm.step += 1;
+    if (set == 0) atomicAdd(reinterpret_cast<unsigned long long*>(prm.step), 1ull);   // no round trip
   }
   __syncthreads();
   if (i < N) {
@@ -1038,7 +1049,8 @@ __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set
   __shared__ double sh_part[2 * kMaxN];
   __shared__ double sh_a[kMaxN];
   __shared__ double sh_u[kMaxN];
-  coeff_core(prm, set, sh_part, 2 * kMaxN, static_cast<int>(blockDim.x), sh_a, sh_u);
+  __shared__ double sh_m[kMaxN];
+  coeff_core(prm, set, sh_part, 2 * kMaxN, static_cast<int>(blockDim.x), sh_a, sh_u, sh_m);
 }
 
 __global__ void __launch_bounds__(kMaxN)
@@ -1608,13 +1620,16 @@ fused_small_kernel(const FusedParams prm) {
 //            the last ticket of the launch adds up all partials in index order (so the result does
 //            not depend on who came last), runs Eq. 7 / 11 / 12-13 and publishes the weights with
 //            a release store of the launch's generation number.
-//   phase 2  the other blocks poll that word (bounded, 2 s), then all blocks form
-//            sum_i gamma_i g_i for the 8 KB-per-row column ranges b, b + grid, ... counted from the
-//            END of the vector -- the columns phase 1 read last come first -- with the loop, the
-//            row order and the rounding of pass2_wide_kernel, so the output bytes are the same.
+//   phase 2  the other blocks poll that word (bounded, 2 s) while their first copies of phase 2
+//            are already in flight (fetching needs no weights), then all blocks form
+//            sum_i gamma_i g_i for the 4 KB-per-row column tiles b, b + grid, ... counted from the
+//            END of the vector -- the columns phase 1 read last come first.  The matrix is staged
+//            by TMA in chunks of 8 rows; a thread owns 16 bytes of every row and adds the rows up
+//            in index order, the order and rounding of the pass-2 kernels: the same output bytes.
 // The launch is cooperative (all blocks resident), the grid is phase 1's.  sync[0] is the ticket
 // counter, sync[1] the published generation; both only grow, a launch owns tickets
-// [gen * grid, (gen + 1) * grid), so the kernel can be replayed from a CUDA graph.
+// [gen * grid, (gen + 1) * grid), so the kernel can be replayed from a CUDA graph; sync[2], the
+// tile counter of phase 2, is set by the block that publishes the weights.
 // ----------------------------------------------------------------------------------------------
 // One thread waits until a monotonically growing word in global memory reaches `want` (written
 // with a release store by another block of the same launch), for at most kWaitLimitNs.
@@ -1640,15 +1655,17 @@ struct MidParams {
   long long num_vec;               // 16-byte column groups per row (the last may be partial)
   int tail_elems;
   int keep_in_l2;                  // the result fits in L2: store it evict_last
-  unsigned long long* sync;        // [0] tickets drawn, [1] generations published
+  int stages2;                     // depth of phase 2's ring (stages of 8 boxes x min(N, 8) rows x 512 bytes)
+  unsigned long long* sync;        // [0] tickets drawn, [1] generations published, [2] phase-2 tile counter
 };
 
 constexpr int kMidPartCap = 2 * kMaxN;   // as coeff_kernel (1024 threads): the same summation order, the same bits
-constexpr int kMidRows = 8;        // rows in flight per thread in phase 2
+constexpr int kMidChunkRows = 8;   // rows of one phase-2 stage
+constexpr int kMidMaxStages2 = 8;
 
 template <int DT, int NR, int WR>
 __global__ void __launch_bounds__(kThreads, 2)
-mid_fused_kernel(const __grid_constant__ CUtensorMap tmap, const MidParams prm) {
+mid_fused_kernel(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap2, const MidParams prm) {
   using C = P1<DT, NR, WR>;
   constexpr int NP = Elem<DT>::kVec / 2;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -1656,6 +1673,9 @@ mid_fused_kernel(const __grid_constant__ CUtensorMap tmap, const MidParams prm) 
   __shared__ int s_role;                       // 0 = waits for the weights, 1 = computes them, -1 = gave up
   __shared__ unsigned long long s_gen;
   __shared__ float g_s[kMaxFastN];
+  __shared__ __align__(8) uint64_t s_full2[kMidMaxStages2];
+  __shared__ long long s_item_tile[kMidMaxStages2];   // per stage: the tile id of the item it holds (-1: the ring ends here)
+  __shared__ int s_item_chunk[kMidMaxStages2];        // ... and which chunk of rows
   const Pass1Params& p1 = prm.p1;
   const int N = p1.N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1732,54 +1752,164 @@ mid_fused_kernel(const __grid_constant__ CUtensorMap tmap, const MidParams prm) 
     p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst, dst + N, N);   // ends with a barrier
   }
 
-  // ---- ticket; the last block of the launch computes the weights (Eq. 7, 11, 12-13)
+  // ---- phase 2 set-up: a ring of row chunks (see below).  Nothing of phase 1 lives in shared
+  // memory any more; its barriers are invalidated before their bytes are reused.
+  // Column tiles of phase 2 are handed out dynamically -- an output element is formed entirely
+  // inside one thread, so who computes which tile cannot change a bit of the result, and blocks
+  // that run slower simply take fewer tiles.  Tile ids count from the END of the vector.  The
+  // first kStatic ids of a block are fixed (b, b + grid, ...), enough to fill its ring before the
+  // weights exist; later ids come from a counter that the block publishing the weights sets to
+  // kStatic * grid first.  The elected thread fetches the next id one tile ahead of its use.
+  const int RB = N < kMidChunkRows ? N : kMidChunkRows;       // rows per chunk = rows of one box
+  const int RC = (N + RB - 1) / RB;                           // chunks per column tile
+  const uint32_t stage2_bytes = static_cast<uint32_t>(kWarps) * RB * kBoxRowBytes;
+  constexpr int T2COLS = kWarps * C::BOXC;                    // columns per phase-2 tile: 4 KB of every row
+  const long long tiles2 = (prm.num_vec * C::VEC + T2COLS - 1) / T2COLS;
+  const int kStatic = (prm.stages2 + RC - 1) / RC;
+  // the ticket first: its round trip to L2 overlaps the set-up of phase 2's barriers
+  unsigned long long ticket = 0ull;
   if (tid == 0) {
     __threadfence();                                            // this block's partial is visible ...
-    const unsigned long long t = atomicAdd(&prm.sync[0], 1ull); // ... before its ticket is
-    s_gen = t / gridDim.x;
-    s_role = ((t + 1ull) % gridDim.x == 0ull) ? 1 : 0;
+    ticket = atomicAdd(&prm.sync[0], 1ull);                     // ... before its ticket is
+    for (int s = 0; s < p1.stages; ++s) asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_addr(&sm.full[s])) : "memory");
+    for (int s = 0; s < prm.stages2; ++s) { mbar_init(&s_full2[s], 1); s_item_tile[s] = -1; }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();                                 // phase 1 wrote these bytes with ordinary stores
+  }
+  // producer state (elected thread only)
+  long long p_tile = -1;          // id of the tile being issued (-1: none left)
+  int p_chunk = 0;                // next chunk of it
+  int p_static = 0;               // static ids taken so far
+  long long p_next_dyn = -1;      // dynamic id fetched ahead (valid once the weights are published)
+  bool p_dyn_ready = false;
+  int issued2 = 0;                // items issued (for the drain after a time-out)
+  auto next_tile = [&]() -> long long {
+    if (p_static < kStatic) {
+      const long long id = first + static_cast<long long>(p_static) * stride;
+      ++p_static;
+      return id < tiles2 ? id : -1;
+    }
+    if (!p_dyn_ready) return -1;                               // not before the weights are published (initial fill only)
+    const long long id = p_next_dyn;
+    if (id >= tiles2) return -1;
+    p_next_dyn = static_cast<long long>(atomicAdd(&prm.sync[2], 1ull));   // for the tile after this one
+    return id;
+  };
+  auto issue_next = [&](int s) -> bool {  // put the next item into stage s; false when there is none
+    if (p_tile < 0 || p_chunk == RC) {
+      p_tile = next_tile();
+      p_chunk = 0;
+      if (p_tile < 0) { s_item_tile[s] = -1; return false; }
+    }
+    s_item_tile[s] = p_tile;
+    s_item_chunk[s] = p_chunk;
+    const int col0 = static_cast<int>((tiles2 - 1 - p_tile) * T2COLS);
+    const int row0 = p_chunk * RB;
+    mbar_expect_tx(&s_full2[s], stage2_bytes);
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w)
+      tma_load_2d(smem_raw + static_cast<size_t>(s) * stage2_bytes + static_cast<size_t>(w) * RB * kBoxRowBytes, &tmap2,
+                  &s_full2[s], col0 + w * C::BOXC, row0);
+    ++p_chunk;
+    ++issued2;
+    return true;
+  };
+
+  // ---- the last block of the launch computes the weights (Eq. 7, 11, 12-13)
+  if (tid == 0) {
+    s_gen = ticket / gridDim.x;
+    s_role = ((ticket + 1ull) % gridDim.x == 0ull) ? 1 : 0;
     __threadfence();
+    if (s_role == 0 && !aborted)                                // fetching needs no weights: fill the ring while waiting
+      for (int s = 0; s < prm.stages2; ++s)
+        if (!issue_next(s)) break;
   }
   __syncthreads();
   if (s_role == 1) {
-    // every copy into this block's ring has landed, so the ring is free to hold the work arrays
+    // this block's ring is idle until it has published the weights: it holds the work arrays
     double* work = reinterpret_cast<double*>(smem_raw);
-    coeff_core(prm.coeff, 0, work, kMidPartCap, kMaxN, work + kMidPartCap, work + kMidPartCap + kMaxFastN);
+    coeff_core(prm.coeff, 0, work, kMidPartCap, kMaxN, work + kMidPartCap, work + kMidPartCap + kMaxFastN,
+               work + kMidPartCap + 2 * kMaxFastN);
     __syncthreads();
     if (tid == 0) {
+      prm.sync[2] = static_cast<unsigned long long>(kStatic) * gridDim.x;   // first dynamic tile id of this launch
       __threadfence();
       const unsigned long long g = s_gen + 1ull;
       asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(prm.sync + 1), "l"(g) : "memory");
+      if (!aborted) {
+        fence_proxy_async_smem();
+        for (int s = 0; s < prm.stages2; ++s)
+          if (!issue_next(s)) break;
+      }
     }
   } else if (tid == 0) {
     if (!wait_generation_bounded(prm.sync + 1, s_gen + 1ull, p1.flags)) s_role = -1;
   }
   __syncthreads();
-  if (s_role < 0 || aborted) return;
-  if (tid < N) g_s[tid] = __ldcg(prm.coeff.gamma_f32 + tid);
+  if (aborted) return;                                          // nothing of phase 2 was issued
+  if (s_role < 0) {                                             // the weights never came: wait for the copies in flight, leave
+    if (tid == 0) p1_drain_after_timeout(s_full2, prm.stages2, issued2, p1.flags);
+    return;
+  }
+  if (tid == 0) {                                               // the counter is valid now: fetch the first dynamic id ahead
+    p_next_dyn = static_cast<long long>(atomicAdd(&prm.sync[2], 1ull));
+    p_dyn_ready = true;
+  }
+  if (tid < kMaxFastN) g_s[tid] = tid < N ? __ldcg(prm.coeff.gamma_f32 + tid) : 0.f;
   __syncthreads();
 
-  // ---- phase 2 (Eq. 12): pass2_wide_kernel's block b for b = blockIdx.x, blockIdx.x + grid, ...
+  // ---- phase 2 (Eq. 12).  A stage holds RB rows of a 4 KB-per-row column tile: one TMA box of
+  // RB x 512 bytes per warp.  Thread (warp, lane) owns the 16-byte column group `lane` of its warp's
+  // box and walks the row chunks of a tile in order, adding gamma_i * g_i row by row into registers
+  // (the order and rounding of the pass-2 kernels); after the last chunk it stores its 16 bytes.
+  // No data crosses threads.
   const unsigned long long keep = prm.keep_in_l2 ? l2_policy_evict_last() : 0ull;
-  const long long num_vec = prm.num_vec;
-  const long long num_pairs = (num_vec + 1) / 2;
-  const long long blocks2 = (num_pairs + kPass2BlockPairs - 1) / kPass2BlockPairs;
-  for (long long b = blockIdx.x; b < blocks2; b += gridDim.x) {
-    const long long w = num_pairs - (b + 1) * kPass2BlockPairs + tid;
-    if (w < 0) continue;
-    const long long v0 = 2 * w;
-    if (v0 + 1 < num_vec) {
-      float2 acc[2][NP];
-      pass2_wide_pair<DT, kMidRows>(prm.grads + w * 32, g_s, N, prm.row_bytes, acc);
-      if (prm.tail_elems != 0 && v0 + 1 == num_vec - 1) {
-        pass2_store<DT, NP>(prm.out, v0, acc[0], keep);
-        pass2_store_tail<DT, NP>(prm.out, v0 + 1, acc[1], prm.tail_elems);
-      } else {
-        st_global_v8(prm.out + w * 32, pass2_pack<DT, NP>(acc[0]), pass2_pack<DT, NP>(acc[1]), keep);
-      }
+  float2 acc[NP];
+#pragma unroll
+  for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+  int s2 = 0;
+  uint32_t parity2 = 0;
+  for (;;) {
+    const long long tile = s_item_tile[s2];                     // written by the elected thread at least one barrier ago
+    if (tile < 0) break;
+    const int rc = s_item_chunk[s2];
+    uint4 xr[kMidChunkRows];
+    const unsigned char* box = smem_raw + static_cast<size_t>(s2) * stage2_bytes + static_cast<size_t>(warp) * RB * kBoxRowBytes + lane * 16;
+    if (mbar_wait_bounded(&s_full2[s2], parity2)) {
+#pragma unroll
+      for (int r = 0; r < kMidChunkRows; ++r) xr[r] = r < RB ? ld_shared_v4(box + r * kBoxRowBytes) : make_uint4(0u, 0u, 0u, 0u);
     } else {
-      pass2_single_vector<DT>(prm.grads, prm.out, g_s, N, prm.row_bytes, v0, num_vec, prm.tail_elems, keep);
+#pragma unroll
+      for (int r = 0; r < kMidChunkRows; ++r) xr[r] = make_uint4(0u, 0u, 0u, 0u);
+      atomicOr(&s_abort, 1);
     }
+    __syncthreads();                                            // the stage is in registers; its item fields are read
+    if (s_abort) break;
+    if (tid == 0) {
+      fence_proxy_async_smem();
+      (void)issue_next(s2);
+    }
+    const int rbase = rc * RB;
+#pragma unroll
+    for (int r = 0; r < kMidChunkRows; ++r) {
+      if (r < RB && rbase + r < N) {
+        const float gm = g_s[rbase + r];
+        const float2 g2 = make_float2(gm, gm);
+#pragma unroll
+        for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(xr[r], h), g2, acc[h]);
+      }
+    }
+    if (rc == RC - 1) {
+      const long long v = (tiles2 - 1 - tile) * (T2COLS / C::VEC) + warp * 32 + lane;
+      if (v < prm.num_vec) pass2_store_any<DT, NP>(prm.out, v, acc, prm.num_vec, prm.tail_elems, keep);
+#pragma unroll
+      for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+    }
+    if (++s2 == prm.stages2) { s2 = 0; parity2 ^= 1u; }
+  }
+  if (s_abort) {
+    if (tid == 0) p1_drain_after_timeout(s_full2, prm.stages2, issued2, p1.flags);
+    return;
   }
 }
 

@@ -131,7 +131,7 @@ def test_one_launch_scaled_configs(ac, name, d, steps):
 
 def test_one_launch_default_by_size_and_alignment(ac):
     """By default the one-launch kernel serves what does not fit in shared memory, up to 1 GiB, on
-    32-byte aligned buffers; per-segment mode and 16-byte-only alignment keep the three kernels."""
+    16-byte aligned buffers; per-segment mode keeps the three kernels."""
     dev = torch.device("cuda:0")
     w = wl.Workload("olsel", 8, 2_000_000, "f32", 1, "gauss", seed=2)
     G = wl.generate(w, 0, dev)
@@ -140,10 +140,13 @@ def test_one_launch_default_by_size_and_alignment(ac):
     assert h.get_option(ac.OPT_ONE_LAUNCH) == 1
     h.aggregate(G, out[:w.d])
     torch.cuda.synchronize()
-    assert h.info(ac.INFO_LAST_PATH) == 5 and h.info(ac.INFO_LAUNCHES_PER_CALL) == 1 and h.info(ac.INFO_LAST_PASS2) == 3
-    h.aggregate(G, out[4:w.d + 4])                     # out is 16 but not 32 bytes aligned
+    assert h.info(ac.INFO_LAST_PATH) == 5 and h.info(ac.INFO_LAUNCHES_PER_CALL) == 1 and h.info(ac.INFO_LAST_PASS2) == 4
+    h.aggregate(G, out[4:w.d + 4])                     # out is 16 but not 32 bytes aligned: still one launch
     torch.cuda.synchronize()
-    assert h.info(ac.INFO_LAST_PATH) == 1 and h.info(ac.INFO_LAUNCHES_PER_CALL) == 3 and h.info(ac.INFO_LAST_PASS2) == 2
+    assert h.info(ac.INFO_LAST_PATH) == 5
+    h.aggregate(G, out[1:w.d + 1])                     # out is not 16 bytes aligned: the generic path
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 2
     h.set_option(ac.OPT_ONE_LAUNCH, 0)
     h.aggregate(G, out[:w.d])
     torch.cuda.synchronize()
@@ -794,12 +797,13 @@ def test_pass2_vector_widths(ac, N, dtype, d, pitch, shift, kernel):
     _padded_case(ac, N, d, dtype, pitch, 2, fused=False, expect_path=1, expect_pass2=kernel, out_shift=shift)
 
 
-@pytest.mark.parametrize("dtype,d,pitch,shift,kernel", [c for c in PASS2_WIDTH_CASES if c[4] == 3])
+@pytest.mark.parametrize("dtype,d,pitch,shift,kernel", PASS2_WIDTH_CASES)
 @pytest.mark.parametrize("N", [3, 13, 40])
 def test_one_launch_padded_rows_and_tails(ac, N, dtype, d, pitch, shift, kernel):
-    """The one-launch kernel on every tail shape of the 32-byte pass 2 (odd or even number of 16-byte
-    groups, full or partial last group, less than one block), NaN padding and a guarded result."""
-    _padded_case(ac, N, d, dtype, pitch, 2, fused=False, one_launch=2, expect_path=5, expect_pass2=3, out_shift=shift)
+    """The one-launch kernel on every tail shape of pass 2 (odd or even number of 16-byte groups,
+    full or partial last group, less than one tile, 16- and 32-byte alignment), NaN padding and a
+    guarded result."""
+    _padded_case(ac, N, d, dtype, pitch, 2, fused=False, one_launch=2, expect_path=5, expect_pass2=4, out_shift=shift)
 
 
 @pytest.mark.parametrize("dtype,d,pitch,shift,kernel", [c for c in PASS2_WIDTH_CASES if c[1] >= 100_000])
