@@ -179,10 +179,15 @@ __device__ __forceinline__ P1Smem p1_carve(unsigned char* raw, int stages, uint3
 // rows of this thread from a landed stage (zeros for rows >= N)
 template <class C>
 __device__ __forceinline__ void p1_load_rows(uint4 (&v)[C::NR], const unsigned char* box_lane, int rw, int N) {
+  if (N == C::NR * C::WR) {                  // every row exists (block-uniform): no per-row test
 #pragma unroll
-  for (int j = 0; j < C::NR; ++j) {
-    const int row = rw + C::WR * j;
-    v[j] = (row < N) ? ld_shared_v4(box_lane + row * kBoxRowBytes) : make_uint4(0u, 0u, 0u, 0u);
+    for (int j = 0; j < C::NR; ++j) v[j] = ld_shared_v4(box_lane + (rw + C::WR * j) * kBoxRowBytes);
+  } else {
+#pragma unroll
+    for (int j = 0; j < C::NR; ++j) {
+      const int row = rw + C::WR * j;
+      v[j] = (row < N) ? ld_shared_v4(box_lane + row * kBoxRowBytes) : make_uint4(0u, 0u, 0u, 0u);
+    }
   }
 }
 template <int DT, class C>
@@ -1205,7 +1210,8 @@ __device__ __forceinline__ int seg_find(const long long* off_s, int nseg, long l
 }
 
 template <int DT>
-__device__ __forceinline__ void pass2_mixed_vector_smem(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
+__device__ __noinline__ void pass2_mixed_vector_smem(   // rare (threads that straddle a boundary): kept out of the vector loop's registers
+    const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
                                                         const float* g_seg, const long long* off_s, int nseg, int N,
                                                         long long row_bytes, long long v, long long num_vec, int tail_elems,
                                                         unsigned long long policy) {
@@ -1225,13 +1231,83 @@ __device__ __forceinline__ void pass2_mixed_vector_smem(const unsigned char* __r
   float2 acc[NP];
 #pragma unroll
   for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
-  for (int i = 0; i < N; ++i) {
-    const uint4 x = ld_stream_v4(col + static_cast<long long>(i) * row_bytes);
+  constexpr int U = 4;                           // rows in flight: this thread's block waits for it
+  int i0 = 0;
+  for (; i0 + U <= N; i0 += U) {
+    uint4 x[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) x[u] = ld_stream_v4(col + static_cast<long long>(i0 + u) * row_bytes);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int h = 0; h < NP; ++h)
+        acc[h] = __ffma2_rn(unpack_pair<DT>(x[u], h),
+                            make_float2(g_seg[seg_of[2 * h] + i0 + u], g_seg[seg_of[2 * h + 1] + i0 + u]), acc[h]);
+  }
+  for (; i0 < N; ++i0) {
+    const uint4 x = ld_stream_v4(col + static_cast<long long>(i0) * row_bytes);
 #pragma unroll
     for (int h = 0; h < NP; ++h)
-      acc[h] = __ffma2_rn(unpack_pair<DT>(x, h), make_float2(g_seg[seg_of[2 * h] + i], g_seg[seg_of[2 * h + 1] + i]), acc[h]);
+      acc[h] = __ffma2_rn(unpack_pair<DT>(x, h), make_float2(g_seg[seg_of[2 * h] + i0], g_seg[seg_of[2 * h + 1] + i0]), acc[h]);
   }
   pass2_store_any<DT, NP>(out, v, acc, num_vec, tail_elems, policy);
+}
+
+// The same for a complete 32-byte pair (groups 2w and 2w + 1): one 256-bit load per row, four rows in
+// flight, so that a straddling thread needs no more round trips to memory than its neighbours and
+// does not keep its block waiting.
+template <int DT>
+__device__ __noinline__ void pass2_mixed_pair_smem(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
+                                                   const float* g_seg, const long long* off_s, int nseg, int N,
+                                                   long long row_bytes, long long w, long long num_vec, int tail_elems,
+                                                   unsigned long long policy) {
+  constexpr int VEC = Elem<DT>::kVec;
+  constexpr int NP = VEC / 2;
+  const long long v0 = 2 * w;
+  const long long d_cols = (num_vec - 1) * VEC + (tail_elems ? tail_elems : VEC);
+  int sg = seg_find(off_s, nseg, v0 * VEC);
+  int seg_of[2 * VEC];
+#pragma unroll
+  for (int e = 0; e < 2 * VEC; ++e) {
+    const long long c = v0 * VEC + e;
+    if (c < d_cols)
+      while (c >= off_s[sg + 1]) ++sg;
+    seg_of[e] = sg * N;
+  }
+  const unsigned char* col = grads + w * 32;
+  float2 acc[2][NP];
+#pragma unroll
+  for (int g = 0; g < 2; ++g)
+#pragma unroll
+    for (int h = 0; h < NP; ++h) acc[g][h] = make_float2(0.f, 0.f);
+  constexpr int U = 4;
+  int i0 = 0;
+  for (; i0 + U <= N; i0 += U) {
+    uint4 x[U][2];
+#pragma unroll
+    for (int u = 0; u < U; ++u) ld_stream_v8(col + static_cast<long long>(i0 + u) * row_bytes, x[u][0], x[u][1]);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int g = 0; g < 2; ++g)
+#pragma unroll
+        for (int h = 0; h < NP; ++h)
+          acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[u][g], h),
+                                 make_float2(g_seg[seg_of[g * VEC + 2 * h] + i0 + u], g_seg[seg_of[g * VEC + 2 * h + 1] + i0 + u]),
+                                 acc[g][h]);
+  }
+  for (; i0 < N; ++i0) {
+    uint4 x[2];
+    ld_stream_v8(col + static_cast<long long>(i0) * row_bytes, x[0], x[1]);
+#pragma unroll
+    for (int g = 0; g < 2; ++g)
+#pragma unroll
+      for (int h = 0; h < NP; ++h)
+        acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[g], h),
+                               make_float2(g_seg[seg_of[g * VEC + 2 * h] + i0], g_seg[seg_of[g * VEC + 2 * h + 1] + i0]), acc[g][h]);
+  }
+  pass2_store_any<DT, NP>(out, v0, acc[0], num_vec, tail_elems, policy);
+  pass2_store_any<DT, NP>(out, v0 + 1, acc[1], num_vec, tail_elems, policy);
 }
 
 // Loads the weights and offsets of segments sg0..sg1 into shared memory; false if they do not fit.
@@ -1381,7 +1457,7 @@ __device__ __forceinline__ void pass2_wide_pair(const unsigned char* __restrict_
 // (keep_in_l2 != 0) is still written evict_last: it then stays in L2, where the next call
 // overwrites it and its consumer finds it, and never costs DRAM bandwidth at all.
 template <int DT, bool SEG, int U = kPass2WideRows>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)     // four blocks per SM: the rare per-column path may spill, the vector loop does not
 pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out,
                   const float* __restrict__ gamma, int N, long long row_bytes, long long num_vec,
                   const int* __restrict__ blk_seg, const long long* __restrict__ seg_off, int tail_elems, int keep_in_l2) {
@@ -1429,9 +1505,8 @@ pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __rest
     gw = g_s + sl * N;
   }
   if (SEG && straddles) {
-    for (int g = 0; g < 2; ++g)
-      if (v0 + g < num_vec)
-        pass2_mixed_vector_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, v0 + g, num_vec, tail_elems, keep);
+    if (v0 + 1 < num_vec) pass2_mixed_pair_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, w, num_vec, tail_elems, keep);
+    else pass2_mixed_vector_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, v0, num_vec, tail_elems, keep);
     return;
   }
   if (v0 + 1 < num_vec) {                            // the pair is complete (all but an odd row's last group)
