@@ -59,6 +59,9 @@ def parse_args(argv=None):
     ap.add_argument("--no-extra-loops", action="store_true",
                     help="skip the two additional loops (per-step events for the median; the launch sequence without events)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shape", default="", help="N,d,dtype of an ad-hoc Gaussian workload instead of a named one, e.g. 128,20000000,bf16")
+    ap.add_argument("--cluster-pass1", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_CLUSTER_PASS1 (64 < N <= 512)")
+    ap.add_argument("--tall-tiles", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_TALL_TILES (64 < N <= 128)")
     ap.add_argument("--one-launch", type=int, default=-1, choices=[-1, 0, 1, 2],
                     help="ADACONS_OPT_ONE_LAUNCH (default: the library's own choice by size)")
     return ap.parse_args(argv)
@@ -204,9 +207,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
-    w = wl.WORKLOADS[args.workload]
-    if args.d:
-        w = w.scaled(args.d)
+    w = pick_workload(args)
     sec, elems, ws = oracle_sample_steps(w, args.steps, min(args.warmup, 1), ORACLE_SAMPLE_COLUMNS)
     value = elems / sec
     line = {
@@ -222,6 +223,15 @@ def run_reference(args):
     }
     print(json.dumps(line), flush=True)
     return 0
+
+
+def pick_workload(args):
+    from paper_2411_03742_b200 import workloads as wl
+    if args.shape:
+        n, d, dt = args.shape.split(",")
+        return wl.Workload(f"custom{n}x{d}", int(n), int(d), dt, 10, "gauss", seed=9000, note="signal N(0,1) + noise N(0,0.5^2)")
+    w = wl.WORKLOADS[args.workload]
+    return w.scaled(args.d) if args.d else w
 
 
 def describe(w) -> str:
@@ -241,9 +251,7 @@ def run_ours(args):
     rank, world, local = dist_setup(args.gpus, use_cuda=True)
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    w = wl.WORKLOADS[args.workload]
-    if args.d:
-        w = w.scaled(args.d)
+    w = pick_workload(args)
     w_rank = __import__("dataclasses").replace(w, seed=w.seed + 100_000 * rank)
 
     # One matrix when it dwarfs the 126 MB L2; otherwise enough distinct matrices, used in turn, that
@@ -260,6 +268,10 @@ def run_ours(args):
         h.set_option(ac.OPT_OVERLAP_LAUNCH, 0)
     if args.one_launch >= 0:
         h.set_option(ac.OPT_ONE_LAUNCH, args.one_launch)
+    if args.cluster_pass1 >= 0:
+        h.set_option(ac.OPT_CLUSTER_PASS1, args.cluster_pass1)
+    if args.tall_tiles >= 0:
+        h.set_option(ac.OPT_TALL_TILES, args.tall_tiles)
     stream = torch.cuda.current_stream()
 
     for t in range(max(args.warmup, 3)):
@@ -320,7 +332,7 @@ def run_ours(args):
     status = h.status()
     assert status == 0, f"library raised status flags {status:#x}"
     path = h.info(ac.INFO_LAST_PATH)
-    assert path in (1, 3, 5), "benchmark must run the aligned fast path"
+    assert path in (1, 3, 4, 5, 6, 7), "benchmark must run an aligned path"
 
     units_local = float(w.N) * w.d * args.steps
     ms, units = reduce_over_ranks(ms_local, units_local, device=dev)
@@ -364,6 +376,9 @@ def run_ours(args):
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "coefficients": "per segment" if args.per_segment else "model-wise",
                    "path": {1: "three kernels (TMA-staged pass 1)", 3: "single-pass kernel (matrix in shared memory)",
+                            4: "N > 64: column sums, dot products per 64 rows, pass 2 (three reads)",
+                            6: "N > 64: cluster pass 1 (one read), coefficient step, pass 2",
+                            7: "64 < N <= 128: pass 1 on 128-row tiles (one read), coefficient step, pass 2",
                             5: "one launch, two reads (pass 1, coefficient step, pass 2 in one cooperative kernel)"}[path],
                    "l2": (f"inputs ({gbytes / 1e9:.2f} GB) larger than the 126 MB L2; no flush between steps" if nbuf == 1 else
                           f"{nbuf} distinct input matrices of {gbytes / 1e9:.3f} GB used in turn ({nbuf * gbytes / 1e9:.2f} GB "

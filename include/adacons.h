@@ -120,13 +120,21 @@ enum adacons_option {
                                   buffers allow it, whatever the size.  0: never.  Same
                                   coefficients, state and output bytes as the three-kernel path
                                   (the block partials are added in the same fixed order).         */
-  ADACONS_OPT_CLUSTER_PASS1 = 10 /* 1 (default): with 64 < N <= 512 on aligned buffers pass 1 reads
-                                  the matrix ONCE: a thread-block cluster of 2, 4 or 8 blocks
-                                  shares each column tile, 64 rows per block, and exchanges the
-                                  partial column sums through distributed shared memory.  0: the
-                                  two-read form (column sums first, then dot products per 64
-                                  rows), which N > 512 always takes.  Results agree to fp32
-                                  rounding of the column sums.                                   */
+  ADACONS_OPT_TALL_TILES = 11, /* 1 (default): with 64 < N <= 128 on aligned buffers pass 1 reads the
+                                  matrix ONCE, as for N <= 64, from tiles of 128 rows x 256 bytes
+                                  (half a warp per row).  0: the two-read form (column sums
+                                  first, then dot products per 64 rows), which N > 128 always
+                                  takes unless ADACONS_OPT_CLUSTER_PASS1 says otherwise.  The
+                                  forms agree to fp32 rounding of the column sums.               */
+  ADACONS_OPT_CLUSTER_PASS1 = 10 /* 0 (default) / 1: with 64 < N <= 512 on aligned buffers pass 1
+                                  reads the matrix ONCE through thread-block clusters of 2, 4 or 8
+                                  blocks that share each column tile (64 rows per block) and
+                                  exchange partial column sums through distributed shared memory,
+                                  one cluster barrier per tile.  Takes precedence over
+                                  ADACONS_OPT_TALL_TILES.  Off by default: the barrier per tile
+                                  makes it slower than the alternatives except for N <= 128,
+                                  where the tall tiles are faster still.  The forms agree to
+                                  fp32 rounding of the column sums.                              */
 };
 
 /* Which N-vector adacons_get_coeffs returns (values of the most recent aggregate call). */
@@ -149,8 +157,10 @@ enum adacons_info {
                                         3 = single-pass kernel (matrix held in shared memory),
                                         4 = N > 64: column sums, then dot products per 64 rows,
                                         5 = one launch, two reads (see ADACONS_OPT_ONE_LAUNCH),
-                                        6 = 64 < N <= 512: clusters, one read in pass 1
-                                            (see ADACONS_OPT_CLUSTER_PASS1)                      */
+                                        6 = N > 64: clusters, one read in pass 1
+                                            (see ADACONS_OPT_CLUSTER_PASS1),
+                                        7 = 64 < N <= 128: tiles of 128 rows, one read in pass 1
+                                            (see ADACONS_OPT_TALL_TILES)                         */
   ADACONS_INFO_TOTAL_LAUNCHES = 6,   /* kernels launched by this context so far                  */
   ADACONS_INFO_LAST_PASS2 = 7        /* pass-2 kernel of the most recent aggregate call: 0 = none
                                         (no call yet, or the single-pass kernel), 1 = generic,
@@ -184,9 +194,9 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  *   Fast path: grads and out 16-byte aligned, the row pitch in bytes (d*sizeof(element) unless
  *   ADACONS_OPT_ROW_PITCH says otherwise) a multiple of 16; with all three multiples of 32 pass 2
  *   moves 32 bytes per instruction and is about 2 % faster still.  With N <= 64 the matrix is read
- *   twice, and so it is with 64 < N <= 512 (thread-block clusters share a column tile); with
- *   N > 512 three times (column sums first, then dot products per 64 rows; needs d floats of
- *   scratch, allocated in adacons_create).  Misaligned buffers or pitch are served by a
+ *   twice, and so it is with 64 < N <= 128 (tiles of 128 rows, see ADACONS_OPT_TALL_TILES); with
+ *   N > 128 three times (column sums first, then dot products per 64 rows; needs d floats of
+ *   scratch, allocated in adacons_create; see ADACONS_OPT_CLUSTER_PASS1).  Misaligned buffers or pitch are served by a
  *   slower generic path with the same results.
  * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
  * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.

@@ -106,11 +106,18 @@ struct adacons_ctx {
   size_t colsum_bytes = 0;
   CUtensorMap tmap_big;
   const void* tmap_big_for = nullptr;
+  // 64 < N <= 128: one read of the matrix, one block per tile of 128 rows x 256 bytes
+  bool tall_available = false;
+  int tall_grid = 0, tall_tiles = 0, tall_stages = 0;
+  size_t tall_smem = 0;
+  int tall_tiles_opt = 1;               // ADACONS_OPT_TALL_TILES
+  CUtensorMap tmap_tall;
+  const void* tmap_tall_for = nullptr;
   // 64 < N <= 512: one read of the matrix by clusters of 2, 4 or 8 blocks (64 rows each)
   bool cl_available = false;
   int cl_size = 0, cl_grid = 0, cl_tiles = 0;
   size_t cl_smem = 0;
-  int cluster_pass1 = 1;                // ADACONS_OPT_CLUSTER_PASS1
+  int cluster_pass1 = 0;                // ADACONS_OPT_CLUSTER_PASS1 (opt-in)
   int last_launches = 3;
 
   // single-pass path for problems that fit in the grid's shared memory
@@ -314,8 +321,59 @@ int plan_big(adacons_ctx* c) {
   return ADACONS_OK;
 }
 
+// 64 < N <= 128 on the aligned path: tiles of 128 rows x 256 bytes, one block per tile (pass1_tall_kernel).
+int plan_tall(adacons_ctx* c) {
+  c->tall_available = false;
+  if (c->N <= kMaxFastN || c->N > 128) return ADACONS_OK;
+  if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > kChunkCols) return ADACONS_OK;
+  const int tile_cols = 256 / c->elem_bytes;
+  c->tall_tiles = static_cast<int>((c->d + tile_cols - 1) / tile_cols);
+  const size_t fixed = c->dtype == ADACONS_F32 ? P1H<0>::kFixedBytes : P1H<1>::kFixedBytes;
+  const size_t stage = P1H<0>::kStageBytes;
+  int stages = static_cast<int>((kPass1SmemBudget - fixed - 64) / stage);
+  if (stages > 8) stages = 8;
+  if (stages < 2) return ADACONS_OK;
+  const size_t smem = stages * stage + fixed + static_cast<size_t>(stages) * 8;
+  const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_tall_kernel<0>)
+                                          : reinterpret_cast<const void*>(&pass1_tall_kernel<1>);
+  int per_sm = 0;
+  if (smem > kPass1SmemCap || !set_smem_cap(k, kPass1SmemCap) ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, smem) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  c->tall_stages = stages;
+  c->tall_smem = smem;
+  c->tall_grid = per_sm * c->num_sms;
+  if (c->tall_grid > c->tall_tiles) c->tall_grid = c->tall_tiles;
+  c->tmap_tall_for = nullptr;
+  c->tall_available = true;
+  return ADACONS_OK;
+}
+
+int encode_map_tall(adacons_ctx* c, const void* grads) {
+  if (c->tmap_tall_for == grads) return ADACONS_OK;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(256 / c->elem_bytes), 128u};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = c->encode(&c->tmap_tall,
+                               c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                               2, const_cast<void*>(grads), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  c->tmap_tall_for = grads;
+  return ADACONS_OK;
+}
+
 // 64 < N <= 512 on the aligned path: clusters of ceil(N / 64) blocks rounded up to 2, 4 or 8.
 // Shares the tensor map (boxes of 64 rows) and the shared-memory carve-up of the N > 64 path.
+// Opt-in (ADACONS_OPT_CLUSTER_PASS1): the blocks of a cluster meet at a barrier once per tile, and a
+// block cannot prefetch past it, so pass 1 runs latency-bound.  Measured, pass 1 alone, bf16 unless
+// noted: N = 128, d = 20 M: 1.47 ms against 1.51 ms for the two-read form (fp32, d = 10 M: 1.13
+// against 1.47); N = 256, d = 8 M: 1.77 against 1.20; N = 512, d = 4 M: 4.22 against 1.22.
+
 int plan_cluster(adacons_ctx* c) {
   c->cl_available = false;
   if (c->N <= kMaxFastN || c->N > 512) return ADACONS_OK;
@@ -683,6 +741,8 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   if (c->big_available && c->big_grid > c->max_partials) c->max_partials = c->big_grid;
   plan_cluster(c);
   if (c->cl_available && c->cl_grid / c->cl_size > c->max_partials) c->max_partials = c->cl_grid / c->cl_size;
+  plan_tall(c);
+  if (c->tall_available && c->tall_grid > c->max_partials) c->max_partials = c->tall_grid;
 
   if (cudaMalloc(&c->flags, sizeof(uint32_t)) != cudaSuccess || cudaMalloc(&c->step, sizeof(long long)) != cudaSuccess ||
       cudaMalloc(&c->d_barrier, 4 * sizeof(unsigned long long)) != cudaSuccess) {
@@ -839,6 +899,21 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     num_partials = c->fast.grid * c->num_chunks;
     c->last_path = 1;
+  } else if (aligned && c->tall_available && c->tall_tiles_opt && !c->cluster_pass1) {
+    int rc = encode_map_tall(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    Pass1Params p;
+    p.N = N; p.num_tiles = c->tall_tiles; p.stages = c->tall_stages; p.stage_bytes = P1H<0>::kStageBytes;
+    p.partials = c->partials; p.flags = c->flags;
+    const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_tall_kernel<0>)
+                                            : reinterpret_cast<const void*>(&pass1_tall_kernel<1>);
+    void* args[2] = {&c->tmap_tall, &p};
+    if (cudaLaunchKernel(k, dim3(c->tall_grid), dim3(kThreads), args, c->tall_smem, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    num_partials = c->tall_grid;
+    c->last_path = 7;
   } else if (aligned && c->cl_available && c->cluster_pass1) {
     int rc = encode_map_big(c, grads);
     if (rc != ADACONS_OK) return rc;
@@ -1023,6 +1098,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
     case ADACONS_OPT_OVERLAP_LAUNCH: c->overlap_launch = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: c->fused_small = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_CLUSTER_PASS1: c->cluster_pass1 = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_TALL_TILES: c->tall_tiles_opt = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_ONE_LAUNCH:
       if (value != 0.0 && value != 1.0 && value != 2.0) return ADACONS_EINVAL;
       c->one_launch = static_cast<int>(value); return ADACONS_OK;
@@ -1036,6 +1112,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       c->pitch = pitch;
       c->tmap_for = nullptr;
       c->tmap_mid2_for = nullptr;
+      c->tmap_tall_for = nullptr;
       int rc = plan_fast(c);
       if (rc != ADACONS_OK) return rc;
       c->tmaps.resize(static_cast<size_t>(c->num_chunks));
@@ -1047,11 +1124,13 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       rc = plan_big(c);
       if (rc != ADACONS_OK) return rc;
       plan_cluster(c);
+      plan_tall(c);
       int need = c->generic_grid;
       if (c->fast.available && c->fast.grid * c->num_chunks > need) need = c->fast.grid * c->num_chunks;
       if (c->fused_available && c->fused_grid > need) need = c->fused_grid;
       if (c->big_available && c->big_grid > need) need = c->big_grid;
       if (c->cl_available && c->cl_grid / c->cl_size > need) need = c->cl_grid / c->cl_size;
+      if (c->tall_available && c->tall_grid > need) need = c->tall_grid;
       if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
         cudaFree(c->partials);
         c->partials = nullptr;
@@ -1095,6 +1174,7 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_OVERLAP_LAUNCH: *value = c->overlap_launch; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: *value = c->fused_small; return ADACONS_OK;
     case ADACONS_OPT_ONE_LAUNCH: *value = c->one_launch; return ADACONS_OK;
+    case ADACONS_OPT_TALL_TILES: *value = c->tall_tiles_opt; return ADACONS_OK;
     case ADACONS_OPT_CLUSTER_PASS1: *value = c->cluster_pass1; return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: *value = static_cast<double>(c->pitch); return ADACONS_OK;
     default: return ADACONS_EINVAL;

@@ -566,6 +566,148 @@ pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams 
   p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst + prm.r0, dst + prm.N + prm.r0, prm.rows);
 }
 
+// ---- pass 1 for 64 < N <= 128 in one read, one block per tile: boxes of 128 rows x 256 bytes ------
+// Twice the rows of pass1_tma_kernel's tallest tile at half the width, so a stage is still 32 KB.
+// A HALF-warp owns a row: lane l of warp w belongs to row group g = 2 w + (l >> 4) and owns the
+// 16-byte column group l & 15 of rows g, g + 16, ..., g + 112 (8 rows, as before; rows past N are
+// zero-filled by TMA).  The 16 groups' partial column sums are exchanged through shared memory in
+// two steps -- every thread first finishes one column of a quarter or half of the groups, in group
+// order, then all read the sums of their own columns -- and the lane reduction at the end stays
+// inside a half-warp.  Same partial-record layout as pass1_tma_kernel.
+template <int DT>
+struct P1H {
+  static constexpr int NR = 8;
+  static constexpr int VEC = Elem<DT>::kVec;
+  static constexpr int NP = VEC / 2;
+  static constexpr int kRows = 128, kGroups = 16;
+  static constexpr int kBoxRowBytesH = 256;
+  static constexpr int TILEC = kBoxRowBytesH / Elem<DT>::kBytes;   // 128 (bf16) / 64 (fp32) columns per tile
+  static constexpr int PARTS = kThreads / TILEC;                   // threads per column in the first exchange step
+  static constexpr int kGroupsPerPart = kGroups / PARTS;
+  static constexpr uint32_t kStageBytes = kRows * kBoxRowBytesH;   // 32 KB
+  static constexpr int kXchFloats = kGroups * TILEC;
+  static constexpr int kSumFloats = PARTS * TILEC;                 // = kThreads
+  static constexpr int kRedFloats = kGroups * NR * 2;
+  static constexpr int kOuterFloats = 2 * NR * kThreads;
+  static constexpr size_t kFixedBytes = (kXchFloats + kSumFloats + kRedFloats + kOuterFloats) * sizeof(float);
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 2)
+pass1_tall_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm) {
+  using C = P1H<DT>;
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  __shared__ int s_abort;
+  const int N = prm.N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = 2 * warp + (lane >> 4), cl = lane & 15;
+  unsigned char* stage_base = smem_raw;
+  float* xch = reinterpret_cast<float*>(smem_raw + static_cast<size_t>(prm.stages) * C::kStageBytes);
+  float* sums = xch + C::kXchFloats;
+  float* red = sums + C::kSumFloats;
+  float* outer = red + C::kRedFloats;
+  uint64_t* full = reinterpret_cast<uint64_t*>(outer + C::kOuterFloats);
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < prm.stages; ++s) mbar_init(&full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async_smem();
+  }
+  __syncthreads();
+  pdl_launch_dependents();
+  const int first = blockIdx.x, stride = gridDim.x;
+  const int my_tiles = first < prm.num_tiles ? (prm.num_tiles - first + stride - 1) / stride : 0;
+  auto issue = [&](int k, int s) {
+    mbar_expect_tx(&full[s], C::kStageBytes);
+    tma_load_2d(stage_base + static_cast<size_t>(s) * C::kStageBytes, &tmap, &full[s], (first + k * stride) * C::TILEC, 0);
+  };
+  int issued = 0;
+  if (tid == 0) {
+    const int pre = my_tiles < prm.stages ? my_tiles : prm.stages;
+    for (int k = 0; k < pre; ++k) issue(k, k);
+    issued = pre;
+  }
+  float2 pacc[C::NR], qacc[C::NR];
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j) pacc[j] = qacc[j] = make_float2(0.f, 0.f);
+  p1_outer_clear<C>(outer);
+  int s = 0;
+  uint32_t parity = 0;
+  for (int k = 0; k < my_tiles; ++k) {
+    uint4 v[C::NR];
+    if (mbar_wait_bounded(&full[s], parity)) {
+      const unsigned char* mine = stage_base + static_cast<size_t>(s) * C::kStageBytes + g * C::kBoxRowBytesH + cl * 16;
+#pragma unroll
+      for (int j = 0; j < C::NR; ++j) v[j] = ld_shared_v4(mine + j * (C::kGroups * C::kBoxRowBytesH));
+    } else {
+#pragma unroll
+      for (int j = 0; j < C::NR; ++j) v[j] = make_uint4(0u, 0u, 0u, 0u);
+      atomicOr(&s_abort, 1);
+    }
+    float2 sp[C::NP];
+    p1_colsum<DT, C>(v, sp);
+#pragma unroll
+    for (int h2 = 0; h2 < C::VEC / 4; ++h2)            // this group's partial sums of the thread's VEC columns
+      *reinterpret_cast<float4*>(xch + g * C::TILEC + cl * C::VEC + 4 * h2) =
+          make_float4(sp[2 * h2].x, sp[2 * h2].y, sp[2 * h2 + 1].x, sp[2 * h2 + 1].y);
+    __syncthreads();                                    // the stage is in registers; the partials are written
+    if (s_abort) break;
+    if (tid == 0 && k + prm.stages < my_tiles) {
+      fence_proxy_async_smem();
+      issue(k + prm.stages, s);
+      issued = k + prm.stages + 1;
+    }
+    {                                                   // step 1: one column, this thread's share of the groups, in group order
+      const int c = tid % C::TILEC, part = tid / C::TILEC;
+      float a = 0.f;
+#pragma unroll
+      for (int r = 0; r < C::kGroupsPerPart; ++r) a += xch[(part * C::kGroupsPerPart + r) * C::TILEC + c];
+      sums[part * C::TILEC + c] = a;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < C::NP; ++h) sp[h] = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int part = 0; part < C::PARTS; ++part)         // step 2: the parts in order
+#pragma unroll
+      for (int h2 = 0; h2 < C::VEC / 4; ++h2) {
+        const float4 w4 = *reinterpret_cast<const float4*>(sums + part * C::TILEC + cl * C::VEC + 4 * h2);
+        sp[2 * h2] = __fadd2_rn(sp[2 * h2], make_float2(w4.x, w4.y));
+        sp[2 * h2 + 1] = __fadd2_rn(sp[2 * h2 + 1], make_float2(w4.z, w4.w));
+      }
+    p1_accumulate<DT, C>(v, sp, pacc, qacc);
+    if ((k & (kFoldTiles - 1)) == kFoldTiles - 1) p1_fold<C>(pacc, qacc, outer);
+    if (++s == prm.stages) { s = 0; parity ^= 1u; }
+  }
+  float* dst = prm.partials + static_cast<size_t>(blockIdx.x) * 2 * N;
+  if (s_abort) {
+    if (tid == 0) p1_drain_after_timeout(full, prm.stages, issued, prm.flags);
+    for (int i = tid; i < 2 * N; i += kThreads) dst[i] = 0.f;
+    return;
+  }
+  // block partial: both accumulation levels, lanes of a half-warp by a fixed xor tree; every row has one owner group
+  p1_fold<C>(pacc, qacc, outer);
+#pragma unroll
+  for (int j = 0; j < C::NR; ++j) {
+    float p = outer[j * kThreads + tid], q = outer[(C::NR + j) * kThreads + tid];
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) {
+      p += __shfl_xor_sync(0xffffffffu, p, o);
+      q += __shfl_xor_sync(0xffffffffu, q, o);
+    }
+    if (cl == 0) {
+      red[(g * C::NR + j) * 2 + 0] = p;
+      red[(g * C::NR + j) * 2 + 1] = q;
+    }
+  }
+  __syncthreads();
+  if (tid < N) {                                        // row tid = group tid % 16, its (tid / 16)-th row
+    const int rg = tid % C::kGroups, rj = tid / C::kGroups;
+    dst[tid] = red[(rg * C::NR + rj) * 2 + 0];
+    dst[N + tid] = red[(rg * C::NR + rj) * 2 + 1];
+  }
+}
+
 // ---- pass 1 for 64 < N <= 512 in ONE read of the matrix: a thread-block cluster per column tile ----
 // A cluster of C = 2, 4 or 8 blocks owns column tiles c, c + clusters, ...; block r of the cluster
 // stages rows [64 r, 64 r + 64) of a tile (one TMA box; rows past N are zero-filled, a block with

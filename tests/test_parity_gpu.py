@@ -647,7 +647,9 @@ def test_config3_full_size(ac):
 @pytest.mark.parametrize("N", [512, 600, 1024])
 def test_many_workers(ac, N):
     w = wl.Workload(f"many{N}", N, 3_000, "f32", 2, "gauss", seed=N)
-    run_case(ac, w, 2, beta=0.9, expect_path=6 if N <= 512 else 4)
+    run_case(ac, w, 2, beta=0.9, expect_path=4)
+    if N <= 512:
+        run_case(ac, w, 2, beta=0.9, options={ac.OPT_CLUSTER_PASS1: 1}, expect_path=6)
     w = wl.Workload(f"manyodd{N}", N, 3_001, "f32", 2, "gauss", seed=N)      # unaligned: generic path
     run_case(ac, w, 2, beta=0.9, expect_path=2)
 
@@ -655,14 +657,24 @@ def test_many_workers(ac, N):
 @pytest.mark.parametrize("N,d,dtype", [(65, 400_008, "bf16"), (100, 300_004, "f32"), (128, 500_000, "bf16"),
                                        (129, 200_000, "bf16"), (200, 150_000, "f32"), (257, 100_008, "bf16"),
                                        (448, 60_000, "bf16"), (512, 50_000, "f32")])
-@pytest.mark.parametrize("cluster", [1, 0], ids=["clusters-one-read", "column-sums-then-dots"])
-def test_more_than_64_workers(ac, N, d, dtype, cluster):
-    """N > 64 on aligned buffers.  Default for N <= 512: a thread-block cluster of 2, 4 or 8 blocks
-    shares each column tile (64 rows per block, the last block's rows ragged or absent) and pass 1
-    reads the matrix once.  Otherwise: column sums to scratch, then one dot-product launch per 64
-    rows."""
+@pytest.mark.parametrize("form", ["default", "clusters", "two-reads"])
+def test_more_than_64_workers(ac, N, d, dtype, form):
+    """N > 64 on aligned buffers.  Default: up to N = 128 pass 1 reads the matrix once from tiles of
+    128 rows x 256 bytes (rows past N zero-filled); beyond, column sums go to scratch and one
+    dot-product launch per 64 rows follows.  Clusters (opt-in): 2, 4 or 8 blocks share each column
+    tile, 64 rows per block, the last block's rows ragged or absent."""
     w = wl.Workload(f"big{N}", N, d, dtype, 3, "gauss", seed=N)
-    run_case(ac, w, 3, beta=0.8, options={ac.OPT_CLUSTER_PASS1: cluster}, expect_path=6 if cluster else 4)
+    opts = {"default": {}, "clusters": {ac.OPT_CLUSTER_PASS1: 1}, "two-reads": {ac.OPT_TALL_TILES: 0, ac.OPT_CLUSTER_PASS1: 0}}[form]
+    path = {"default": 7 if N <= 128 else 4, "clusters": 6, "two-reads": 4}[form]
+    run_case(ac, w, 3, beta=0.8, options=opts, expect_path=path)
+
+
+@pytest.mark.parametrize("N,dtype", [(65, "f32"), (96, "bf16"), (127, "f32"), (128, "bf16"), (128, "f32")])
+def test_tall_tiles_many_tiles_per_block(ac, N, dtype):
+    """The 128-row tiles on a vector long enough that every block walks many of them (the folding of
+    the first-level sums runs several times) with a ragged last tile and heavy-tailed data."""
+    w = wl.Workload(f"tall{N}", N, 3_000_008, dtype, 2, "student_flip", seed=N)
+    run_case(ac, w, 2, beta=0.9, expect_path=7)
 
 
 @pytest.mark.parametrize("N,dtype", [(128, "f32"), (128, "bf16"), (96, "bf16"), (300, "f32")])
@@ -670,13 +682,14 @@ def test_cluster_pass1_many_tiles_per_cluster(ac, N, dtype):
     """Long enough that every cluster walks many tiles (the double-buffered exchange of the partial
     column sums wraps around many times) and the last tile is ragged."""
     w = wl.Workload(f"cl{N}", N, 2_000_008, dtype, 2, "student_flip", seed=N)
-    run_case(ac, w, 2, beta=0.9, expect_path=6)
+    run_case(ac, w, 2, beta=0.9, options={ac.OPT_CLUSTER_PASS1: 1}, expect_path=6)
 
 
-@pytest.mark.parametrize("cluster", [1, 0])
-def test_more_than_64_workers_with_padded_rows(ac, cluster):
-    _padded_case(ac, 96, 123_457, "bf16", 123_464, 2, fused=False, options={ac.OPT_CLUSTER_PASS1: cluster},
-                 expect_path=6 if cluster else 4)
+@pytest.mark.parametrize("form", ["default", "clusters", "two-reads"])
+def test_more_than_64_workers_with_padded_rows(ac, form):
+    opts = {"default": {}, "clusters": {ac.OPT_CLUSTER_PASS1: 1}, "two-reads": {ac.OPT_TALL_TILES: 0, ac.OPT_CLUSTER_PASS1: 0}}[form]
+    _padded_case(ac, 96, 123_457, "bf16", 123_464, 2, fused=False, options=opts,
+                 expect_path={"default": 7, "clusters": 6, "two-reads": 4}[form])
 
 
 # ---- the call neither allocates nor synchronises: it can be recorded once and replayed -----------
