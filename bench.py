@@ -38,8 +38,9 @@ CPU_BASELINE_COLUMNS = 4_000_000       # cpu_baseline leg of the CUDA arm: 3 ste
 # to the columns processed), as a multiple of that kernel's algorithmic bytes.  Keyed by
 # (workload, coefficient mode, kernel); anything else reports no traffic figure.
 NCU_TRAFFIC_RATIO = {
-    ("bert64", "model-wise", "pass1"): (1.0014, "profiles/pass1_pass2_bert64_d20M_full_set.md (d = 20 M, scaled by d)"),
-    ("bert64", "model-wise", "pass2"): (0.9988, "profiles/pass2_wide_mixed16_full_set.md (result larger than L2)"),
+    ("bert64", "model-wise", "pass1"): (1.0016, "profiles/pass1_pass2_bert64_d20M_full_set.md (same kernel, d = 20 M, scaled by d)"),
+    ("bert64", "model-wise", "pass2"): (0.9989, "profiles/pass2_wide_bf16_result_larger_than_L2.md (same kernel, N = 16, d = 80 M; "
+                                                "reads and writes both scale with the bytes processed)"),
 }
 
 
