@@ -893,8 +893,11 @@ def test_replay_of_the_single_pass_kernel_from_a_cuda_graph(ac):
     assert h.state()[1] == 3 and h.status() == 0
 
 
-def test_two_contexts_on_two_streams_are_independent(ac):
-    """Distinct contexts share nothing: interleaved on two streams they give what each gives alone."""
+@pytest.mark.parametrize("one_launch", [0, 2], ids=["three-kernels", "one-launch"])
+def test_two_contexts_on_two_streams_are_independent(ac, one_launch):
+    """Distinct contexts share nothing: interleaved on two streams they give what each gives alone.
+    (Two cooperative one-launch kernels cannot share the GPU; the driver runs them one after the
+    other, and their waits are on their own contexts' words.)"""
     dev = torch.device("cuda:0")
     wa = wl.Workload("ctxa", 16, 900_008, "bf16", 3, "gauss", seed=1)
     wb = wl.Workload("ctxb", 5, 1_300_000, "f32", 3, "gauss_outlier", seed=2)
@@ -904,7 +907,7 @@ def test_two_contexts_on_two_streams_are_independent(ac):
     def alone(w, Gs, dtype):
         h = ac.AdaCons(w.N, w.d, dtype)
         h.set_option(ac.OPT_FUSED_SMALL, 0)
-        h.set_option(ac.OPT_ONE_LAUNCH, 0)
+        h.set_option(ac.OPT_ONE_LAUNCH, one_launch)
         out = torch.empty(w.d, dtype=w.torch_dtype, device=dev)
         outs = []
         for G in Gs:
@@ -918,7 +921,7 @@ def test_two_contexts_on_two_streams_are_independent(ac):
     sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
     ha, hb = ac.AdaCons(wa.N, wa.d, "bf16"), ac.AdaCons(wb.N, wb.d, "f32")
     ha.set_option(ac.OPT_FUSED_SMALL, 0); hb.set_option(ac.OPT_FUSED_SMALL, 0)
-    ha.set_option(ac.OPT_ONE_LAUNCH, 0); hb.set_option(ac.OPT_ONE_LAUNCH, 0)    # two cooperative kernels cannot share the GPU
+    ha.set_option(ac.OPT_ONE_LAUNCH, one_launch); hb.set_option(ac.OPT_ONE_LAUNCH, one_launch)
     oa = [torch.empty(wa.d, dtype=torch.bfloat16, device=dev) for _ in range(3)]
     ob = [torch.empty(wb.d, device=dev) for _ in range(3)]
     torch.cuda.synchronize()
@@ -930,6 +933,7 @@ def test_two_contexts_on_two_streams_are_independent(ac):
         assert torch.equal(oa[t].view(torch.uint8), ref_a[t].view(torch.uint8))
         assert torch.equal(ob[t], ref_b[t])
     assert ha.coeffs(stream=sa).tobytes() == ca.tobytes() and hb.coeffs(stream=sb).tobytes() == cb.tobytes()
+    assert ha.status(stream=sa) == 0 and hb.status(stream=sb) == 0
 
 
 def test_contexts_of_other_shapes_do_not_disturb_an_existing_one(ac):
