@@ -120,6 +120,17 @@ enum adacons_option {
                                   buffers allow it, whatever the size.  0: never.  Same
                                   coefficients, state and output bytes as the three-kernel path
                                   (the block partials are added in the same fixed order).         */
+  ADACONS_OPT_ALIGNED_BODY = 12, /* 1 (default): when the row pitch is a multiple of 16 bytes but the
+                                  matrix starts off a 16-byte boundary (a slice of a larger
+                                  buffer), every row is misaligned by the same amount; with
+                                  N <= 64 pass 1 then runs its TMA-staged kernel on the aligned
+                                  body (from each row's first 16-byte boundary on) and a one-block
+                                  kernel adds the up to 7 columns before it, and if `out` is off
+                                  by the same amount pass 2 does likewise (whole 16-byte groups
+                                  vectorised, head and ragged tail element by element).  0: such
+                                  buffers take the generic path, as a pitch that is not a
+                                  multiple of 16 bytes always does.  Same results either way to
+                                  fp32 accumulation order.                                       */
   ADACONS_OPT_TALL_TILES = 11, /* 1 (default): with 64 < N <= 128 on aligned buffers pass 1 reads the
                                   matrix ONCE, as for N <= 64, from tiles of 128 rows x 256 bytes
                                   (half a warp per row).  0: the two-read form (column sums
@@ -160,13 +171,17 @@ enum adacons_info {
                                         6 = N > 64: clusters, one read in pass 1
                                             (see ADACONS_OPT_CLUSTER_PASS1),
                                         7 = 64 < N <= 128: tiles of 128 rows, one read in pass 1
-                                            (see ADACONS_OPT_TALL_TILES)                         */
+                                            (see ADACONS_OPT_TALL_TILES),
+                                        8 = misaligned base, aligned body: TMA-staged pass 1 plus
+                                            the head columns (see ADACONS_OPT_ALIGNED_BODY)      */
   ADACONS_INFO_TOTAL_LAUNCHES = 6,   /* kernels launched by this context so far                  */
   ADACONS_INFO_LAST_PASS2 = 7        /* pass-2 kernel of the most recent aggregate call: 0 = none
                                         (no call yet, or the single-pass kernel), 1 = generic,
                                         2 = 16-byte vectors, 3 = 32-byte vectors (grads, out and
                                         the row pitch 32-byte aligned), 4 = the second phase of
-                                        the one-launch kernel (TMA-staged chunks of 8 rows)      */
+                                        the one-launch kernel (TMA-staged chunks of 8 rows),
+                                        5 = vector kernel on the aligned body plus element-wise
+                                        edges (grads and out off a 16-byte boundary alike)       */
 };
 
 /*
@@ -196,8 +211,10 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  *   moves 32 bytes per instruction and is about 2 % faster still.  With N <= 64 the matrix is read
  *   twice, and so it is with 64 < N <= 128 (tiles of 128 rows, see ADACONS_OPT_TALL_TILES); with
  *   N > 128 three times (column sums first, then dot products per 64 rows; needs d floats of
- *   scratch, allocated in adacons_create; see ADACONS_OPT_CLUSTER_PASS1).  Misaligned buffers or pitch are served by a
- *   slower generic path with the same results.
+ *   scratch, allocated in adacons_create; see ADACONS_OPT_CLUSTER_PASS1).  A matrix that merely starts off a 16-byte
+ *   boundary keeps the fast pass 1 (ADACONS_OPT_ALIGNED_BODY); a pitch that is not a multiple of
+ *   16 bytes, or N > 64 with a misaligned base, is served by a slower generic path with the same
+ *   results.
  * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
  * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.
  * Errors: EINVAL (NULL pointers, overlap), ECUDA (launch failure), EALIGN (per-segment mode with

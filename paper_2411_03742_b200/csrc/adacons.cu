@@ -154,6 +154,9 @@ struct adacons_ctx {
   std::vector<CUtensorMap> tmaps;       // one per column chunk; tmaps[0] covers everything when d <= 2^30
   const void* tmap_for = nullptr;
 
+  CUtensorMap tmap_body;                // pass 1 on the aligned body of a matrix whose rows start off a 16-byte boundary
+  const void* tmap_body_for = nullptr;
+  int aligned_body = 1;                 // ADACONS_OPT_ALIGNED_BODY
   int last_path = 0;
   int last_pass2 = 0;                   // 0 none, 1 generic, 2 16-byte vectors, 3 32-byte vectors
   long long total_launches = 0;
@@ -520,6 +523,23 @@ int encode_map_mid2(adacons_ctx* c, const void* grads) {
   return ADACONS_OK;
 }
 
+// Tensor map of the aligned body: columns [head, d) of every row, starting on a 16-byte boundary.
+int encode_map_body(adacons_ctx* c, const void* grads, int head) {
+  if (c->tmap_body_for == grads) return ADACONS_OK;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d - head), static_cast<cuuint64_t>(c->N)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(c->N)};
+  const cuuint32_t estr[2] = {1, 1};
+  void* base = const_cast<unsigned char*>(static_cast<const unsigned char*>(grads)) + static_cast<size_t>(head) * c->elem_bytes;
+  const CUresult r = c->encode(&c->tmap_body, c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                               2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  c->tmap_body_for = grads;
+  return ADACONS_OK;
+}
+
 // All chunk maps of a context (its vector was sized when the plan was made).
 int encode_map(adacons_ctx* c, const void* grads) {
   if (c->tmap_for == grads) return ADACONS_OK;
@@ -752,6 +772,7 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
       cudaMemset(c->d_barrier, 0, 4 * sizeof(unsigned long long)) != cudaSuccess) {
     adacons_destroy(c); return ADACONS_ECUDA;
   }
+  c->max_partials += 1;                  // room for the record of the head columns (aligned-body path)
   const size_t b_part = static_cast<size_t>(c->max_partials) * 2 * N * sizeof(float);
   if (cudaMalloc(&c->partials, b_part) != cudaSuccess) { cudaGetLastError(); adacons_destroy(c); return ADACONS_ENOMEM; }
   if (cudaMemset(c->partials, 0, b_part) != cudaSuccess) { adacons_destroy(c); return ADACONS_ECUDA; }
@@ -789,7 +810,11 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   DeviceGuard guard(c->device);
   if (!guard.ok) return ADACONS_ECUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const bool aligned = (g0 % 16 == 0) && (o0 % 16 == 0) && ((c->pitch * c->elem_bytes) % 16 == 0);
+  const bool pitch16 = (c->pitch * c->elem_bytes) % 16 == 0;
+  const bool aligned = (g0 % 16 == 0) && (o0 % 16 == 0) && pitch16;
+  const bool g_aligned = (g0 % 16 == 0) && pitch16;      // pass 1 only reads the matrix
+  // rows that start off a 16-byte boundary, all by the same amount: `head` columns up to the boundary
+  const int head = (pitch16 && g0 % 16 != 0 && g0 % c->elem_bytes == 0) ? static_cast<int>((16 - g0 % 16) / c->elem_bytes) : 0;
   const long long num_vec = (c->d * c->elem_bytes + 15) / 16;              // 16-byte column groups per row
   const int tail_elems = static_cast<int>((c->d * c->elem_bytes % 16) / c->elem_bytes);   // 0: the last group is full
   const long long row_bytes = c->pitch * c->elem_bytes;
@@ -880,7 +905,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     num_partials = 0;
     c->last_path = 1;
-  } else if (aligned && c->fast.available) {
+  } else if (g_aligned && c->fast.available) {
     int rc = encode_map(c, grads);
     if (rc != ADACONS_OK) return rc;
     for (int ch = 0; ch < c->num_chunks; ++ch) {      // one launch per column chunk of 2^30 (normally one)
@@ -899,7 +924,26 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     num_partials = c->fast.grid * c->num_chunks;
     c->last_path = 1;
-  } else if (aligned && c->tall_available && c->tall_tiles_opt && !c->cluster_pass1) {
+  } else if (head > 0 && c->aligned_body && c->fast.available && c->num_chunks == 1 && c->d > head) {
+    // the TMA-staged kernel on the aligned body, the head columns as one more partial record
+    int rc = encode_map_body(c, grads, head);
+    if (rc != ADACONS_OK) return rc;
+    Pass1Params p;
+    p.N = N; p.num_tiles = static_cast<int>((c->d - head + c->fast.tile_cols - 1) / c->fast.tile_cols);
+    p.stages = c->fast.stages; p.stage_bytes = c->fast.stage_bytes; p.partials = c->partials; p.flags = c->flags;
+    void* args[2] = {&c->tmap_body, &p};
+    if (cudaLaunchKernel(c->fast.kernel, dim3(c->fast.grid), dim3(kThreads), args, c->fast.smem_bytes, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    float* rec = c->partials + static_cast<size_t>(c->fast.grid) * 2 * N;
+    if (c->dtype == ADACONS_F32) edge_stats_kernel<0><<<1, kThreads, 0, st>>>(grads, N, c->pitch, head, rec);
+    else edge_stats_kernel<1><<<1, kThreads, 0, st>>>(grads, N, c->pitch, head, rec);
+    if (!launch_ok()) return ADACONS_ECUDA;
+    extra_launches += 1;
+    num_partials = c->fast.grid + 1;
+    c->last_path = 8;
+  } else if (g_aligned && c->tall_available && c->tall_tiles_opt && !c->cluster_pass1) {
     int rc = encode_map_tall(c, grads);
     if (rc != ADACONS_OK) return rc;
     Pass1Params p;
@@ -914,7 +958,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     }
     num_partials = c->tall_grid;
     c->last_path = 7;
-  } else if (aligned && c->cl_available && c->cluster_pass1) {
+  } else if (g_aligned && c->cl_available && c->cluster_pass1) {
     int rc = encode_map_big(c, grads);
     if (rc != ADACONS_OK) return rc;
     Pass1ClusterParams p;
@@ -932,7 +976,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     if (e1 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
     num_partials = c->cl_grid / c->cl_size;
     c->last_path = 6;
-  } else if (aligned && c->big_available) {
+  } else if (g_aligned && c->big_available) {
     int rc = encode_map_big(c, grads);
     if (rc != ADACONS_OK) return rc;
     const unsigned cblocks = static_cast<unsigned>((num_vec + kThreads - 1) / kThreads);
@@ -1011,6 +1055,36 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
 #undef ADACONS_LAUNCH_PASS2
 #undef ADACONS_LAUNCH_PASS2W
     c->last_pass2 = wide ? 3 : 2;
+  } else if (!seg && head > 0 && c->aligned_body && (o0 % 16 == g0 % 16) && c->d > head) {
+    // grads and out start off a 16-byte boundary by the same amount: the vector kernels on the whole
+    // 16-byte groups of the aligned body, the head and the ragged tail element by element
+    const int vec = 16 / c->elem_bytes;
+    const long long body = c->d - head;
+    const long long nv = body / vec;                                    // whole groups only
+    const int tail = static_cast<int>(body - nv * vec);
+    const unsigned char* g8 = static_cast<const unsigned char*>(grads) + static_cast<size_t>(head) * c->elem_bytes;
+    unsigned char* o8 = static_cast<unsigned char*>(out) + static_cast<size_t>(head) * c->elem_bytes;
+    e2 = cudaSuccess;
+    if (nv > 0) {
+      const long long np2 = (nv + 1) / 2;
+      const unsigned blocks = static_cast<unsigned>((np2 + kPass2BlockPairs - 1) / kPass2BlockPairs);
+      const bool wide = (reinterpret_cast<uintptr_t>(g8) % 32 == 0) && (reinterpret_cast<uintptr_t>(o8) % 32 == 0) && (row_bytes % 32 == 0);
+      const int keep = static_cast<long long>(obytes) <= c->l2_bytes ? 1 : 0;
+      const int* nobs = nullptr; const long long* noso = nullptr;
+      if (c->dtype == ADACONS_F32)
+        e2 = wide ? launch_kernel(pass2_wide_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, nv, nobs, noso, 0, keep)
+                  : launch_kernel(pass2_vec_kernel<0, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, nv, nobs, noso, 0);
+      else
+        e2 = wide ? launch_kernel(pass2_wide_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, nv, nobs, noso, 0, keep)
+                  : launch_kernel(pass2_vec_kernel<1, false>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, nv, nobs, noso, 0);
+    }
+    if (e2 == cudaSuccess) {
+      if (c->dtype == ADACONS_F32) edge_combine_kernel<0><<<1, 32, 0, st>>>(grads, out, c->gamma_f32, N, c->d, c->pitch, head, tail);
+      else edge_combine_kernel<1><<<1, 32, 0, st>>>(grads, out, c->gamma_f32, N, c->d, c->pitch, head, tail);
+      e2 = cudaGetLastError();
+      extra_launches += (nv > 0) ? 1 : 0;
+    }
+    c->last_pass2 = 5;
   } else {
     const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);
     if (c->dtype == ADACONS_F32)
@@ -1099,6 +1173,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
     case ADACONS_OPT_FUSED_SMALL: c->fused_small = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_CLUSTER_PASS1: c->cluster_pass1 = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_TALL_TILES: c->tall_tiles_opt = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_ALIGNED_BODY: c->aligned_body = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_ONE_LAUNCH:
       if (value != 0.0 && value != 1.0 && value != 2.0) return ADACONS_EINVAL;
       c->one_launch = static_cast<int>(value); return ADACONS_OK;
@@ -1113,6 +1188,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       c->tmap_for = nullptr;
       c->tmap_mid2_for = nullptr;
       c->tmap_tall_for = nullptr;
+      c->tmap_body_for = nullptr;
       int rc = plan_fast(c);
       if (rc != ADACONS_OK) return rc;
       c->tmaps.resize(static_cast<size_t>(c->num_chunks));
@@ -1131,6 +1207,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       if (c->big_available && c->big_grid > need) need = c->big_grid;
       if (c->cl_available && c->cl_grid / c->cl_size > need) need = c->cl_grid / c->cl_size;
       if (c->tall_available && c->tall_grid > need) need = c->tall_grid;
+      need += 1;                             // the head columns' record (aligned-body path)
       if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
         cudaFree(c->partials);
         c->partials = nullptr;
@@ -1175,6 +1252,7 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_FUSED_SMALL: *value = c->fused_small; return ADACONS_OK;
     case ADACONS_OPT_ONE_LAUNCH: *value = c->one_launch; return ADACONS_OK;
     case ADACONS_OPT_TALL_TILES: *value = c->tall_tiles_opt; return ADACONS_OK;
+    case ADACONS_OPT_ALIGNED_BODY: *value = c->aligned_body; return ADACONS_OK;
     case ADACONS_OPT_CLUSTER_PASS1: *value = c->cluster_pass1; return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: *value = static_cast<double>(c->pitch); return ADACONS_OK;
     default: return ADACONS_EINVAL;

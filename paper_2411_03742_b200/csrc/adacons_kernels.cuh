@@ -1683,6 +1683,59 @@ pass2_generic_kernel(const void* __restrict__ grads, void* __restrict__ out, con
 }
 
 // ----------------------------------------------------------------------------------------------
+// Edges of a matrix whose rows start off a 16-byte boundary (every row by the same amount: the row
+// pitch is a multiple of 16 bytes).  The vectorised kernels then run on the aligned body -- from
+// each row's first 16-byte boundary on -- and these two one-block kernels do the few columns left:
+// edge_stats_kernel adds the first `head` (< 8) columns' share of Eq. 7 as one more partial record,
+// edge_combine_kernel forms Eq. 12 for the head columns and for the last `tail` (< 8) columns that
+// do not fill a 16-byte group (element-wise, so nothing is read or written past the vector).
+// ----------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(kThreads)
+edge_stats_kernel(const void* __restrict__ grads, int N, long long pitch, int head, float* __restrict__ record) {
+  __shared__ float x[kMaxFastN * 8];
+  __shared__ float s[8];
+  const int tid = threadIdx.x;
+  for (int idx = tid; idx < N * head; idx += kThreads) {
+    const int i = idx / head, k = idx - i * head;
+    x[i * 8 + k] = load_elem<DT>(grads, static_cast<long long>(i) * pitch + k);
+  }
+  __syncthreads();
+  if (tid < head) {
+    float a = 0.f;
+    for (int i = 0; i < N; ++i) a += x[i * 8 + tid];
+    s[tid] = a;
+  }
+  __syncthreads();
+  if (tid < N) {
+    float pp = 0.f, qq = 0.f;
+    for (int k = 0; k < head; ++k) {
+      const float v = x[tid * 8 + k];
+      pp = fmaf(v, s[k], pp);
+      qq = fmaf(v, v, qq);
+    }
+    record[tid] = pp;
+    record[N + tid] = qq;
+  }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(32)
+edge_combine_kernel(const void* __restrict__ grads, void* __restrict__ out, const float* __restrict__ gamma, int N,
+                    long long d, long long pitch, int head, int tail) {
+  __shared__ float g_s[kMaxFastN];
+  for (int i = threadIdx.x; i < N; i += 32) g_s[i] = gamma[i];
+  __syncthreads();
+  const int k = threadIdx.x;
+  if (k >= head + tail) return;
+  const long long col = k < head ? k : d - tail + (k - head);
+  float acc = 0.f;
+  for (int i = 0; i < N; ++i) acc = fmaf(load_elem<DT>(grads, static_cast<long long>(i) * pitch + col), g_s[i], acc);
+  if constexpr (DT == 0) reinterpret_cast<float*>(out)[col] = acc;
+  else reinterpret_cast<unsigned short*>(out)[col] = static_cast<unsigned short>(pack_bf16x2_rn(acc, 0.f) & 0xffffu);
+}
+
+// ----------------------------------------------------------------------------------------------
 // Single-pass path for problems that fit in the grid's shared memory (N*d*sizeof(element) up to
 // about 148 x 160 KB): ONE cooperative kernel reads the matrix from HBM once.  Block b keeps all N
 // rows of its column slice in shared memory, computes its partial statistics (Eq. 7), meets the

@@ -144,9 +144,9 @@ def test_one_launch_default_by_size_and_alignment(ac):
     h.aggregate(G, out[4:w.d + 4])                     # out is 16 but not 32 bytes aligned: still one launch
     torch.cuda.synchronize()
     assert h.info(ac.INFO_LAST_PATH) == 5
-    h.aggregate(G, out[1:w.d + 1])                     # out is not 16 bytes aligned: the generic path
+    h.aggregate(G, out[1:w.d + 1])                     # out is not 16 bytes aligned: fast pass 1, generic pass 2
     torch.cuda.synchronize()
-    assert h.info(ac.INFO_LAST_PATH) == 2
+    assert h.info(ac.INFO_LAST_PATH) == 1 and h.info(ac.INFO_LAST_PASS2) == 1
     h.set_option(ac.OPT_ONE_LAUNCH, 0)
     h.aggregate(G, out[:w.d])
     torch.cuda.synchronize()
@@ -278,7 +278,11 @@ def test_single_column_has_tied_coefficients(ac):
     assert_output(out, res, to_f64(G), "f32", "d=1")
 
 
-def test_misaligned_pointers_take_the_generic_path(ac):
+@pytest.mark.parametrize("aligned_body", [1, 0])
+def test_misaligned_base_pointer(ac, aligned_body):
+    """A matrix that starts 4 bytes off a 16-byte boundary with a 16-byte pitch: pass 1 runs on the
+    aligned body plus the head columns (path 8), or on the generic kernels when that is switched off;
+    `out` is aligned here, i.e. off by another amount than the matrix, so pass 2 is the generic one."""
     N, d = 6, 4096
     w = wl.Workload("mis", N, d, "f32", 1, "gauss", seed=3)
     G0 = wl.generate(w, 0, "cuda:0")
@@ -288,12 +292,59 @@ def test_misaligned_pointers_take_the_generic_path(ac):
     assert G.data_ptr() % 16 != 0
     out = torch.empty(d, device="cuda:0")
     h = ac.AdaCons(N, d, "f32")
+    h.set_option(ac.OPT_ALIGNED_BODY, aligned_body)
     h.aggregate(G, out)
     torch.cuda.synchronize()
-    assert h.info(ac.INFO_LAST_PATH) == 2
+    assert h.info(ac.INFO_LAST_PATH) == (8 if aligned_body else 2) and h.info(ac.INFO_LAST_PASS2) == 1
     res = oc.AdaConsOracle(N, d).step(to_f64(G0), storage="f32")
     assert_coeffs(h.coeffs(ac.COEFF_GAMMA), res["gamma"], "gamma")
     assert_output(out, res, to_f64(G0), "f32", "misaligned")
+
+
+ALIGNED_BODY_CASES = [  # dtype, N, d, offset of grads (elements), offset of out (elements)
+    ("f32", 8, 300_000, 1, 1), ("f32", 8, 300_000, 3, 3), ("f32", 5, 300_000, 2, 0), ("f32", 64, 40_000, 1, 5),
+    ("bf16", 16, 400_000, 1, 1), ("bf16", 16, 400_000, 7, 7), ("bf16", 64, 80_000, 5, 13), ("bf16", 3, 400_000, 4, 2),
+    ("f32", 4, 8, 1, 1), ("bf16", 4, 16, 3, 3), ("f32", 4, 4, 3, 3), ("bf16", 2, 8, 7, 7),      # hardly any body
+    ("f32", 32, 2_000_004, 2, 2), ("bf16", 8, 2_000_008, 6, 6),
+]
+
+
+@pytest.mark.parametrize("dtype,N,d,g_off,o_off", ALIGNED_BODY_CASES)
+def test_aligned_body_of_offset_buffers(ac, dtype, N, d, g_off, o_off):
+    """grads and out are slices of larger buffers that start g_off resp. o_off elements after a
+    256-byte boundary; d keeps the row pitch a multiple of 16 bytes.  Pass 1 always takes the aligned
+    body; pass 2 does when both are off by the same number of bytes.  NaN before and after the
+    matrix, sentinels around the result; three steps with momentum against the oracle."""
+    dev = torch.device("cuda:0")
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    eb = 4 if dtype == "f32" else 2
+    assert (d * eb) % 16 == 0 and (g_off * eb) % 16 != 0
+    w = wl.Workload(f"off{N}x{d}", N, d, dtype, 3, "gauss_outlier", seed=g_off * 16 + o_off)
+    gbuf = torch.full((N * d + 64,), float("nan"), dtype=tdt, device=dev)
+    G = gbuf[g_off:g_off + N * d].view(N, d)
+    obuf = torch.full((d + 64,), 7.0, dtype=tdt, device=dev)
+    out = obuf[o_off:o_off + d]
+    h = ac.AdaCons(N, d, dtype)
+    h.set_option(ac.OPT_BETA, 0.8)
+    orc = oc.AdaConsOracle(N, d, beta=0.8)
+    same = (g_off * eb) % 16 == (o_off * eb) % 16
+    for t in range(3):
+        G0 = wl.generate(w, t, dev)
+        G.copy_(G0)
+        h.aggregate(G, out)
+        torch.cuda.synchronize()
+        head = (16 - (g_off * eb) % 16) // eb
+        assert h.info(ac.INFO_LAST_PATH) == (8 if d > head else 2), h.info(ac.INFO_LAST_PATH)
+        assert h.info(ac.INFO_LAST_PASS2) == (5 if same and d > head else 1)
+        G64 = to_f64(G0)
+        res = oracle_step(orc, G64, dtype, h.coeffs(ac.COEFF_A), what=w.name)
+        for k, code in (("p", ac.COEFF_P), ("q", ac.COEFF_Q), ("a", ac.COEFF_A), ("gamma", ac.COEFF_GAMMA)):
+            assert_coeffs(h.coeffs(code)[0], res[k][0], f"{w.name} {k} step {t}")
+        assert_coeffs(h.state()[0][0], res["m"][0], f"{w.name} m step {t}")
+        assert_output(out, res, G64, dtype, f"{w.name} step {t}")
+        assert bool((obuf[:o_off] == 7.0).all()) and bool((obuf[o_off + d:] == 7.0).all()), "wrote outside out"
+        assert h.status() == 0
+    h.close()
 
 
 def test_generic_and_fast_paths_agree(ac):
@@ -309,8 +360,15 @@ def test_generic_and_fast_paths_agree(ac):
     h0.set_option(ac.OPT_ONE_LAUNCH, 0)
     h0.aggregate(G0, o0); h1.aggregate(G1, o1)
     torch.cuda.synchronize()
-    assert (h0.info(ac.INFO_LAST_PATH), h1.info(ac.INFO_LAST_PATH)) == (1, 2)
+    assert (h0.info(ac.INFO_LAST_PATH), h1.info(ac.INFO_LAST_PATH)) == (1, 8)
     np.testing.assert_allclose(h0.coeffs(), h1.coeffs(), rtol=2e-6)
+    h2, o2 = ac.AdaCons(N, d, "bf16"), torch.empty(d, device="cuda:0", dtype=torch.bfloat16)
+    h2.set_option(ac.OPT_ALIGNED_BODY, 0)
+    h2.aggregate(G1, o2)
+    torch.cuda.synchronize()
+    assert h2.info(ac.INFO_LAST_PATH) == 2
+    np.testing.assert_allclose(h0.coeffs(), h2.coeffs(), rtol=2e-6)
+    np.testing.assert_allclose(to_f64(o1), to_f64(o2), rtol=2e-2, atol=1e-6)
 
 
 # ---- per-segment ("layer-wise") coefficients ----------------------------------------------------
