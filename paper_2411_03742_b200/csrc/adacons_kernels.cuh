@@ -1588,6 +1588,51 @@ __device__ __forceinline__ void pass2_wide_pair(const unsigned char* __restrict_
   }
 }
 
+// The same sum for a thread of a block that spans segment boundaries: its first `split` elements
+// take the weights `ga` (one segment), the rest `gb` (the next one); split = 2 VEC when the whole
+// pair lies in one segment.  Every thread of such a block runs this loop, so a warp with a
+// straddling thread does not execute two different loops one after the other.
+template <int DT, int U>
+__device__ __forceinline__ void pass2_wide_pair_two(const unsigned char* __restrict__ col, const float* ga, const float* gb,
+                                                    int split, int N, long long row_bytes,
+                                                    float2 (&acc)[2][Elem<DT>::kVec / 2]) {
+  constexpr int VEC = Elem<DT>::kVec;
+  constexpr int NP = VEC / 2;
+#pragma unroll
+  for (int g = 0; g < 2; ++g)
+#pragma unroll
+    for (int h = 0; h < NP; ++h) acc[g][h] = make_float2(0.f, 0.f);
+  int i0 = 0;
+  for (; i0 + U <= N; i0 += U) {
+    uint4 x[U][2];
+#pragma unroll
+    for (int u = 0; u < U; ++u) ld_stream_v8(col + static_cast<long long>(i0 + u) * row_bytes, x[u][0], x[u][1]);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const float a = ga[i0 + u], b = gb[i0 + u];
+#pragma unroll
+      for (int g = 0; g < 2; ++g)
+#pragma unroll
+        for (int h = 0; h < NP; ++h) {
+          const int e = g * VEC + 2 * h;
+          acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[u][g], h), make_float2(e < split ? a : b, e + 1 < split ? a : b), acc[g][h]);
+        }
+    }
+  }
+  for (; i0 < N; ++i0) {
+    uint4 x[2];
+    ld_stream_v8(col + static_cast<long long>(i0) * row_bytes, x[0], x[1]);
+    const float a = ga[i0], b = gb[i0];
+#pragma unroll
+    for (int g = 0; g < 2; ++g)
+#pragma unroll
+      for (int h = 0; h < NP; ++h) {
+        const int e = g * VEC + 2 * h;
+        acc[g][h] = __ffma2_rn(unpack_pair<DT>(x[g], h), make_float2(e < split ? a : b, e + 1 < split ? a : b), acc[g][h]);
+      }
+  }
+}
+
 // Wide kernel (grads, out and the row pitch 32-byte aligned): thread t of block b owns pair
 // w = num_pairs - (b+1) * 256 + t, i.e. 32 contiguous bytes of every row, fetched with one 256-bit
 // load per row (U rows in flight) and written with one 256-bit store.  The loads are no faster
@@ -1615,7 +1660,10 @@ pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __rest
   const long long w = num_pairs - (static_cast<long long>(blockIdx.x) + 1) * kPass2BlockPairs + threadIdx.x;
   const long long v0 = 2 * w;
   const float* gw = g_s;                             // this thread's row of weights
-  bool straddles = false;                            // its 32 bytes hold a segment boundary
+  const float* gw2 = g_s;                            // ... and that of the next segment, if its 32 bytes hold a boundary
+  int split = 2 * VEC;                               // elements of the pair that belong to the first of the two
+  bool mixed_block = false;
+  bool many = false;                                 // its 32 bytes hold more than one boundary
   int nseg = 1;
   if (!SEG || code >= 0) {
     const float* gsrc = gamma + static_cast<size_t>(SEG ? code : 0) * N;
@@ -1639,21 +1687,33 @@ pass2_wide_kernel(const unsigned char* __restrict__ grads, unsigned char* __rest
       return;
     }
     if (w < 0) return;
+    mixed_block = true;
     nseg = sg1 - sg0 + 1;
     const long long d_cols = (num_vec - 1) * VEC + (tail_elems ? tail_elems : VEC);
     const int sl = seg_find(off_s, nseg, v0 * VEC);
     const long long c_last = (v0 * VEC + 2 * VEC < d_cols ? v0 * VEC + 2 * VEC : d_cols) - 1;
-    straddles = c_last >= off_s[sl + 1];
-    gw = g_s + sl * N;
+    gw = gw2 = g_s + sl * N;
+    if (c_last >= off_s[sl + 1]) {                   // a boundary inside the pair: the next non-empty segment takes over
+      split = static_cast<int>(off_s[sl + 1] - v0 * VEC);
+      int s2 = sl + 1;
+      while (off_s[s2 + 1] <= off_s[sl + 1]) ++s2;   // ends: the block's last segment holds c_last
+      gw2 = g_s + s2 * N;
+      many = c_last >= off_s[s2 + 1];
+    }
   }
-  if (SEG && straddles) {
+  if (SEG && many) {                                 // rare: segments of a few columns
     if (v0 + 1 < num_vec) pass2_mixed_pair_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, w, num_vec, tail_elems, keep);
     else pass2_mixed_vector_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, v0, num_vec, tail_elems, keep);
     return;
   }
+  if (SEG && mixed_block && v0 + 1 >= num_vec && split < 2 * VEC) {   // an odd row's last group with a boundary inside
+    pass2_mixed_vector_smem<DT>(grads, out, g_s, off_s, nseg, N, row_bytes, v0, num_vec, tail_elems, keep);
+    return;
+  }
   if (v0 + 1 < num_vec) {                            // the pair is complete (all but an odd row's last group)
     float2 acc[2][NP];
-    pass2_wide_pair<DT, U>(grads + w * 32, gw, N, row_bytes, acc);
+    if (SEG && mixed_block) pass2_wide_pair_two<DT, U>(grads + w * 32, gw, gw2, split, N, row_bytes, acc);
+    else pass2_wide_pair<DT, U>(grads + w * 32, gw, N, row_bytes, acc);
     if (tail_elems != 0 && v0 + 1 == num_vec - 1) {            // the row's last group is partial
       pass2_store<DT, NP>(out, v0, acc[0], keep);
       pass2_store_tail<DT, NP>(out, v0 + 1, acc[1], tail_elems);
