@@ -309,6 +309,38 @@ ALIGNED_BODY_CASES = [  # dtype, N, d, offset of grads (elements), offset of out
 ]
 
 
+@pytest.mark.parametrize("dtype,N,d,pitch,off", [("f32", 8, 100_003, 100_008, 1), ("bf16", 24, 77_777, 77_784, 3),
+                                                  ("f32", 64, 30_001, 30_004, 2), ("bf16", 5, 9, 16, 5)])
+def test_aligned_body_with_padded_rows(ac, dtype, N, d, pitch, off):
+    """Both at once: rows padded to a 16-byte pitch (d itself is odd) in a buffer that starts off a
+    16-byte boundary, `out` off by the same amount.  NaN in all padding, sentinels around the result."""
+    dev = torch.device("cuda:0")
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    w = wl.Workload(f"offpad{N}x{d}", N, d, dtype, 2, "gauss", seed=off + N)
+    gbuf = torch.full((N * pitch + 64,), float("nan"), dtype=tdt, device=dev)
+    Gp = gbuf[off:off + N * pitch].view(N, pitch)
+    obuf = torch.full((d + 64,), 7.0, dtype=tdt, device=dev)
+    out = obuf[off:off + d]
+    h = ac.AdaCons(N, d, dtype)
+    h.set_option(ac.OPT_ROW_PITCH, pitch)
+    h.set_option(ac.OPT_BETA, 0.8)
+    orc = oc.AdaConsOracle(N, d, beta=0.8)
+    for t in range(2):
+        G0 = wl.generate(w, t, dev)
+        Gp[:, :d] = G0
+        h.aggregate(Gp[:, :d], out)
+        torch.cuda.synchronize()
+        assert h.info(ac.INFO_LAST_PATH) == 8 and h.info(ac.INFO_LAST_PASS2) == 5
+        G64 = to_f64(G0)
+        res = oracle_step(orc, G64, dtype, h.coeffs(ac.COEFF_A), what=w.name)
+        assert_coeffs(h.coeffs(ac.COEFF_GAMMA)[0], res["gamma"][0], f"{w.name} gamma {t}")
+        assert_coeffs(h.state()[0][0], res["m"][0], f"{w.name} m {t}")
+        assert_output(out, res, G64, dtype, f"{w.name} out {t}")
+        assert bool((obuf[:off] == 7.0).all()) and bool((obuf[off + d:] == 7.0).all()), "wrote outside out"
+        assert bool(torch.isnan(Gp[:, d:]).all()) and h.status() == 0
+    h.close()
+
+
 @pytest.mark.parametrize("dtype,N,d,g_off,o_off", ALIGNED_BODY_CASES)
 def test_aligned_body_of_offset_buffers(ac, dtype, N, d, g_off, o_off):
     """grads and out are slices of larger buffers that start g_off resp. o_off elements after a
