@@ -108,3 +108,43 @@ def test_public_header_is_plain_c(tmp_path):
                 ["g++", "-std=c++17", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c++"]):
         res = subprocess.run(cmd + ["-I", inc, str(src)], capture_output=True, text=True)
         assert res.returncode == 0, res.stderr
+
+
+def _header_enum(name):
+    """{member: value} of `enum name { ... }` in include/adacons.h."""
+    text = open(os.path.join(ROOT, "include", "adacons.h")).read()
+    body = re.search(r"enum\s+" + name + r"\s*\{(.*?)\};", text, flags=re.S).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    out = {}
+    for m in re.finditer(r"(ADACONS_[A-Z0-9_]+)\s*=\s*(0x[0-9a-fA-F]+|\d+)u?", body):
+        out[m.group(1)] = int(m.group(2), 0)
+    return out
+
+
+def test_binding_constants_match_the_header():
+    """The ctypes binding repeats the header's enumerations as Python constants: every member must be
+    there with the header's value (a renumbered option would silently set another one)."""
+    from paper_2411_03742_b200 import binding
+    for enum, prefix, strip in (("adacons_option", "OPT_", "ADACONS_OPT_"), ("adacons_info", "INFO_", "ADACONS_INFO_"),
+                                ("adacons_coeff", "COEFF_", "ADACONS_COEFF_"), ("adacons_flag", "FLAG_", "ADACONS_FLAG_"),
+                                ("adacons_error", "", "ADACONS_"), ("adacons_dtype", "", "ADACONS_")):
+        members = _header_enum(enum)
+        assert members, enum
+        for name, value in members.items():
+            py = prefix + name[len(strip):]
+            assert hasattr(binding, py), f"binding lacks {py} ({name})"
+            assert getattr(binding, py) == value, (py, getattr(binding, py), value)
+    values = sorted(_header_enum("adacons_option").values())
+    assert values == list(range(len(values))), "option keys must be dense: the binding numbers them with range()"
+
+
+def test_stats_noalloc_binding_validates_before_it_calls(lib):
+    """Layout mistakes are caught in Python (ValueError), before any pointer reaches the library."""
+    import torch
+    from paper_2411_03742_b200 import binding
+    G, pq = torch.zeros(4, 64), torch.zeros(8, dtype=torch.float64)
+    for bad_G, bad_pq in [(G, pq),                                   # host tensors
+                          (G[:, ::2], pq), (G.t(), pq), (G.double(), pq), (torch.zeros(64), pq),
+                          (G, pq.float()), (G, torch.zeros(7, dtype=torch.float64)), (G, torch.zeros(16, dtype=torch.float64)[::2])]:
+        with pytest.raises(ValueError):
+            binding.stats_noalloc(bad_G, bad_pq)
