@@ -62,7 +62,7 @@ def parse_args(argv=None):
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--shape", default="", help="N,d,dtype of an ad-hoc Gaussian workload instead of a named one, e.g. 128,20000000,bf16")
     ap.add_argument("--cluster-pass1", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_CLUSTER_PASS1 (64 < N <= 512)")
-    ap.add_argument("--tall-tiles", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_TALL_TILES (64 < N <= 128)")
+    ap.add_argument("--tall-tiles", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_TALL_TILES (64 < N <= 256)")
     ap.add_argument("--one-launch", type=int, default=-1, choices=[-1, 0, 1, 2],
                     help="ADACONS_OPT_ONE_LAUNCH (default: the library's own choice by size)")
     return ap.parse_args(argv)
@@ -379,7 +379,7 @@ def run_ours(args):
                    "path": {1: "three kernels (TMA-staged pass 1)", 3: "single-pass kernel (matrix in shared memory)",
                             4: "N > 64: column sums, dot products per 64 rows, pass 2 (three reads)",
                             6: "N > 64: cluster pass 1 (one read), coefficient step, pass 2",
-                            7: "64 < N <= 128: pass 1 on 128-row tiles (one read), coefficient step, pass 2",
+                            7: "64 < N <= 256: pass 1 on 128- or 256-row tiles (one read), coefficient step, pass 2",
                             5: "one launch, two reads (pass 1, coefficient step, pass 2 in one cooperative kernel)"}[path],
                    "l2": (f"inputs ({gbytes / 1e9:.2f} GB) larger than the 126 MB L2; no flush between steps" if nbuf == 1 else
                           f"{nbuf} distinct input matrices of {gbytes / 1e9:.3f} GB used in turn ({nbuf * gbytes / 1e9:.2f} GB "

@@ -131,20 +131,22 @@ enum adacons_option {
                                   buffers take the generic path, as a pitch that is not a
                                   multiple of 16 bytes always does.  Same results either way to
                                   fp32 accumulation order.                                       */
-  ADACONS_OPT_TALL_TILES = 11, /* 1 (default): with 64 < N <= 128 on aligned buffers pass 1 reads the
-                                  matrix ONCE, as for N <= 64, from tiles of 128 rows x 256 bytes
-                                  (half a warp per row).  0: the two-read form (column sums
-                                  first, then dot products per 64 rows), which N > 128 always
-                                  takes unless ADACONS_OPT_CLUSTER_PASS1 says otherwise.  The
-                                  forms agree to fp32 rounding of the column sums.               */
+  ADACONS_OPT_TALL_TILES = 11, /* 1 (default): with 64 < N <= 256 on aligned buffers pass 1 reads the
+                                  matrix ONCE, as for N <= 64, from taller and narrower tiles:
+                                  128 rows x 256 bytes (half a warp per row) up to N = 128,
+                                  256 rows x 128 bytes (a quarter-warp per row) beyond.  0: the
+                                  two-read form (column sums first, then dot products per 64
+                                  rows), which N > 256 always takes unless
+                                  ADACONS_OPT_CLUSTER_PASS1 says otherwise.  The forms agree to
+                                  fp32 rounding of the column sums.                              */
   ADACONS_OPT_CLUSTER_PASS1 = 10 /* 0 (default) / 1: with 64 < N <= 512 on aligned buffers pass 1
                                   reads the matrix ONCE through thread-block clusters of 2, 4 or 8
                                   blocks that share each column tile (64 rows per block) and
                                   exchange partial column sums through distributed shared memory,
                                   one cluster barrier per tile.  Takes precedence over
                                   ADACONS_OPT_TALL_TILES.  Off by default: the barrier per tile
-                                  makes it slower than the alternatives except for N <= 128,
-                                  where the tall tiles are faster still.  The forms agree to
+                                  makes it slower than the alternatives (tall tiles up to
+                                  N = 256, the two-read form beyond).  The forms agree to
                                   fp32 rounding of the column sums.                              */
 };
 
@@ -170,7 +172,7 @@ enum adacons_info {
                                         5 = one launch, two reads (see ADACONS_OPT_ONE_LAUNCH),
                                         6 = N > 64: clusters, one read in pass 1
                                             (see ADACONS_OPT_CLUSTER_PASS1),
-                                        7 = 64 < N <= 128: tiles of 128 rows, one read in pass 1
+                                        7 = 64 < N <= 256: tiles of 128 or 256 rows, one read in pass 1
                                             (see ADACONS_OPT_TALL_TILES),
                                         8 = misaligned base, aligned body: TMA-staged pass 1 plus
                                             the head columns (see ADACONS_OPT_ALIGNED_BODY)      */
@@ -209,8 +211,8 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  *   Fast path: grads and out 16-byte aligned, the row pitch in bytes (d*sizeof(element) unless
  *   ADACONS_OPT_ROW_PITCH says otherwise) a multiple of 16; with all three multiples of 32 pass 2
  *   moves 32 bytes per instruction and is about 2 % faster still.  With N <= 64 the matrix is read
- *   twice, and so it is with 64 < N <= 128 (tiles of 128 rows, see ADACONS_OPT_TALL_TILES); with
- *   N > 128 three times (column sums first, then dot products per 64 rows; needs d floats of
+ *   twice, and so it is with 64 < N <= 256 (taller tiles, see ADACONS_OPT_TALL_TILES); with
+ *   N > 256 three times (column sums first, then dot products per 64 rows; needs d floats of
  *   scratch, allocated in adacons_create; see ADACONS_OPT_CLUSTER_PASS1).  A matrix that merely starts off a 16-byte
  *   boundary keeps the fast pass 1 (ADACONS_OPT_ALIGNED_BODY); a pitch that is not a multiple of
  *   16 bytes, or N > 64 with a misaligned base, is served by a slower generic path with the same

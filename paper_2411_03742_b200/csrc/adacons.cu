@@ -108,7 +108,7 @@ struct adacons_ctx {
   const void* tmap_big_for = nullptr;
   // 64 < N <= 128: one read of the matrix, one block per tile of 128 rows x 256 bytes
   bool tall_available = false;
-  int tall_grid = 0, tall_tiles = 0, tall_stages = 0;
+  int tall_grid = 0, tall_tiles = 0, tall_stages = 0, tall_lpr = 16;   // lanes per row: 16 (128-row tiles) or 8 (256-row tiles)
   size_t tall_smem = 0;
   int tall_tiles_opt = 1;               // ADACONS_OPT_TALL_TILES
   CUtensorMap tmap_tall;
@@ -324,21 +324,28 @@ int plan_big(adacons_ctx* c) {
   return ADACONS_OK;
 }
 
-// 64 < N <= 128 on the aligned path: tiles of 128 rows x 256 bytes, one block per tile (pass1_tall_kernel).
+// 64 < N <= 256 on the aligned path: tiles of 128 rows x 256 bytes (N <= 128) or 256 rows x 128 bytes,
+// one block per tile (pass1_tall_kernel).
+const void* tall_fn(int dtype, int lpr) {
+  if (dtype == ADACONS_F32) return lpr == 16 ? reinterpret_cast<const void*>(&pass1_tall_kernel<0, 16>) : reinterpret_cast<const void*>(&pass1_tall_kernel<0, 8>);
+  return lpr == 16 ? reinterpret_cast<const void*>(&pass1_tall_kernel<1, 16>) : reinterpret_cast<const void*>(&pass1_tall_kernel<1, 8>);
+}
+
 int plan_tall(adacons_ctx* c) {
   c->tall_available = false;
-  if (c->N <= kMaxFastN || c->N > 128) return ADACONS_OK;
+  if (c->N <= kMaxFastN || c->N > 256) return ADACONS_OK;
   if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > kChunkCols) return ADACONS_OK;
-  const int tile_cols = 256 / c->elem_bytes;
+  c->tall_lpr = c->N <= 128 ? 16 : 8;
+  const int tile_cols = c->tall_lpr * 16 / c->elem_bytes;
   c->tall_tiles = static_cast<int>((c->d + tile_cols - 1) / tile_cols);
-  const size_t fixed = c->dtype == ADACONS_F32 ? P1H<0>::kFixedBytes : P1H<1>::kFixedBytes;
-  const size_t stage = P1H<0>::kStageBytes;
+  const size_t fixed = c->dtype == ADACONS_F32 ? (c->tall_lpr == 16 ? P1H<0, 16>::kFixedBytes : P1H<0, 8>::kFixedBytes)
+                                               : (c->tall_lpr == 16 ? P1H<1, 16>::kFixedBytes : P1H<1, 8>::kFixedBytes);
+  const size_t stage = P1H<0, 16>::kStageBytes;
   int stages = static_cast<int>((kPass1SmemBudget - fixed - 64) / stage);
   if (stages > 8) stages = 8;
   if (stages < 2) return ADACONS_OK;
   const size_t smem = stages * stage + fixed + static_cast<size_t>(stages) * 8;
-  const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_tall_kernel<0>)
-                                          : reinterpret_cast<const void*>(&pass1_tall_kernel<1>);
+  const void* k = tall_fn(c->dtype, c->tall_lpr);
   int per_sm = 0;
   if (smem > kPass1SmemCap || !set_smem_cap(k, kPass1SmemCap) ||
       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, smem) != cudaSuccess || per_sm < 1) {
@@ -358,7 +365,7 @@ int encode_map_tall(adacons_ctx* c, const void* grads) {
   if (c->tmap_tall_for == grads) return ADACONS_OK;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(256 / c->elem_bytes), 128u};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(c->tall_lpr * 16 / c->elem_bytes), static_cast<cuuint32_t>(c->tall_lpr == 16 ? 128 : 256)};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = c->encode(&c->tmap_tall,
                                c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
@@ -947,10 +954,9 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     int rc = encode_map_tall(c, grads);
     if (rc != ADACONS_OK) return rc;
     Pass1Params p;
-    p.N = N; p.num_tiles = c->tall_tiles; p.stages = c->tall_stages; p.stage_bytes = P1H<0>::kStageBytes;
+    p.N = N; p.num_tiles = c->tall_tiles; p.stages = c->tall_stages; p.stage_bytes = P1H<0, 16>::kStageBytes;
     p.partials = c->partials; p.flags = c->flags;
-    const void* k = c->dtype == ADACONS_F32 ? reinterpret_cast<const void*>(&pass1_tall_kernel<0>)
-                                            : reinterpret_cast<const void*>(&pass1_tall_kernel<1>);
+    const void* k = tall_fn(c->dtype, c->tall_lpr);
     void* args[2] = {&c->tmap_tall, &p};
     if (cudaLaunchKernel(k, dim3(c->tall_grid), dim3(kThreads), args, c->tall_smem, st) != cudaSuccess) {
       cudaGetLastError();

@@ -445,22 +445,26 @@ pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams 
   p1_block_store<C>(pacc, qacc, sm.outer, sm.red, dst + prm.r0, dst + prm.N + prm.r0, prm.rows);
 }
 
-// ---- pass 1 for 64 < N <= 128 in one read, one block per tile: boxes of 128 rows x 256 bytes ------
-// Twice the rows of pass1_tma_kernel's tallest tile at half the width, so a stage is still 32 KB.
-// A HALF-warp owns a row: lane l of warp w belongs to row group g = 2 w + (l >> 4) and owns the
-// 16-byte column group l & 15 of rows g, g + 16, ..., g + 112 (8 rows, as before; rows past N are
-// zero-filled by TMA).  The 16 groups' partial column sums are exchanged through shared memory in
-// two steps -- every thread first finishes one column of a quarter or half of the groups, in group
-// order, then all read the sums of their own columns -- and the lane reduction at the end stays
-// inside a half-warp.  Same partial-record layout as pass1_tma_kernel.
-template <int DT>
+// ---- pass 1 for 64 < N <= 256 in one read, one block per tile: taller, narrower boxes ------------
+// More rows than pass1_tma_kernel's tallest tile at a fraction of the width, so a stage is still
+// 32 KB: 128 rows x 256 bytes (LPR = 16 lanes per row: a HALF-warp owns a row) or 256 rows x 128
+// bytes (LPR = 8: a quarter-warp; TMA moves 128-byte box rows at 4.6 TB/s at most on this GPU, which
+// is still more than two reads at full speed).  Lane l of warp w belongs to row group
+// g = (32 / LPR) w + l / LPR and owns the 16-byte column group l % LPR of rows g, g + G, ...,
+// g + 7 G (8 rows, as before; G = 8 * 32 / LPR groups; rows past N are zero-filled by TMA).  The
+// groups' partial column sums are exchanged through shared memory in two steps -- every thread
+// first finishes one column of its share of the groups, in group order, then all read the sums of
+// their own columns -- and the lane reduction at the end stays inside the LPR lanes of a row.
+// Same partial-record layout as pass1_tma_kernel.
+template <int DT, int LPR>
 struct P1H {
   static constexpr int NR = 8;
   static constexpr int VEC = Elem<DT>::kVec;
   static constexpr int NP = VEC / 2;
-  static constexpr int kRows = 128, kGroups = 16;
-  static constexpr int kBoxRowBytesH = 256;
-  static constexpr int TILEC = kBoxRowBytesH / Elem<DT>::kBytes;   // 128 (bf16) / 64 (fp32) columns per tile
+  static constexpr int kLanesPerRow = LPR;
+  static constexpr int kGroups = kWarps * (32 / LPR), kRows = kGroups * NR;
+  static constexpr int kBoxRowBytesH = LPR * 16;
+  static constexpr int TILEC = kBoxRowBytesH / Elem<DT>::kBytes;   // columns per tile
   static constexpr int PARTS = kThreads / TILEC;                   // threads per column in the first exchange step
   static constexpr int kGroupsPerPart = kGroups / PARTS;
   static constexpr uint32_t kStageBytes = kRows * kBoxRowBytesH;   // 32 KB
@@ -471,15 +475,15 @@ struct P1H {
   static constexpr size_t kFixedBytes = (kXchFloats + kSumFloats + kRedFloats + kOuterFloats) * sizeof(float);
 };
 
-template <int DT>
+template <int DT, int LPR>
 __global__ void __launch_bounds__(kThreads, 2)
 pass1_tall_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm) {
-  using C = P1H<DT>;
+  using C = P1H<DT, LPR>;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ int s_abort;
   const int N = prm.N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int g = 2 * warp + (lane >> 4), cl = lane & 15;
+  const int g = (32 / LPR) * warp + lane / LPR, cl = lane % LPR;
   unsigned char* stage_base = smem_raw;
   float* xch = reinterpret_cast<float*>(smem_raw + static_cast<size_t>(prm.stages) * C::kStageBytes);
   float* sums = xch + C::kXchFloats;
@@ -564,13 +568,13 @@ pass1_tall_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params pr
     for (int i = tid; i < 2 * N; i += kThreads) dst[i] = 0.f;
     return;
   }
-  // block partial: both accumulation levels, lanes of a half-warp by a fixed xor tree; every row has one owner group
+  // block partial: both accumulation levels, the lanes of a row by a fixed xor tree; every row has one owner group
   p1_fold<C>(pacc, qacc, outer);
 #pragma unroll
   for (int j = 0; j < C::NR; ++j) {
     float p = outer[j * kThreads + tid], q = outer[(C::NR + j) * kThreads + tid];
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) {
+    for (int o = LPR / 2; o > 0; o >>= 1) {
       p += __shfl_xor_sync(0xffffffffu, p, o);
       q += __shfl_xor_sync(0xffffffffu, q, o);
     }
@@ -580,7 +584,7 @@ pass1_tall_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params pr
     }
   }
   __syncthreads();
-  if (tid < N) {                                        // row tid = group tid % 16, its (tid / 16)-th row
+  if (tid < N) {                                        // row tid = group tid % kGroups, its (tid / kGroups)-th row
     const int rg = tid % C::kGroups, rj = tid / C::kGroups;
     dst[tid] = red[(rg * C::NR + rj) * 2 + 0];
     dst[N + tid] = red[(rg * C::NR + rj) * 2 + 1];

@@ -749,21 +749,22 @@ def test_many_workers(ac, N):
                                        (448, 60_000, "bf16"), (512, 50_000, "f32")])
 @pytest.mark.parametrize("form", ["default", "clusters", "two-reads"])
 def test_more_than_64_workers(ac, N, d, dtype, form):
-    """N > 64 on aligned buffers.  Default: up to N = 128 pass 1 reads the matrix once from tiles of
-    128 rows x 256 bytes (rows past N zero-filled); beyond, column sums go to scratch and one
-    dot-product launch per 64 rows follows.  Clusters (opt-in): 2, 4 or 8 blocks share each column
+    """N > 64 on aligned buffers.  Default: up to N = 256 pass 1 reads the matrix once from tiles of
+    128 rows x 256 bytes or 256 rows x 128 bytes (rows past N zero-filled); beyond, column sums go to
+    scratch and one dot-product launch per 64 rows follows.  Clusters (opt-in): 2, 4 or 8 blocks share each column
     tile, 64 rows per block, the last block's rows ragged or absent."""
     w = wl.Workload(f"big{N}", N, d, dtype, 3, "gauss", seed=N)
     opts = {"default": {}, "clusters": {ac.OPT_CLUSTER_PASS1: 1}, "two-reads": {ac.OPT_TALL_TILES: 0, ac.OPT_CLUSTER_PASS1: 0}}[form]
-    path = {"default": 7 if N <= 128 else 4, "clusters": 6, "two-reads": 4}[form]
+    path = {"default": 7 if N <= 256 else 4, "clusters": 6, "two-reads": 4}[form]
     run_case(ac, w, 3, beta=0.8, options=opts, expect_path=path)
 
 
-@pytest.mark.parametrize("N,dtype", [(65, "f32"), (96, "bf16"), (127, "f32"), (128, "bf16"), (128, "f32")])
+@pytest.mark.parametrize("N,dtype", [(65, "f32"), (96, "bf16"), (127, "f32"), (128, "bf16"), (128, "f32"),
+                                     (129, "bf16"), (200, "f32"), (255, "bf16"), (256, "f32"), (256, "bf16")])
 def test_tall_tiles_many_tiles_per_block(ac, N, dtype):
-    """The 128-row tiles on a vector long enough that every block walks many of them (the folding of
+    """The 128- and 256-row tiles on a vector long enough that every block walks many of them (the folding of
     the first-level sums runs several times) with a ragged last tile and heavy-tailed data."""
-    w = wl.Workload(f"tall{N}", N, 3_000_008, dtype, 2, "student_flip", seed=N)
+    w = wl.Workload(f"tall{N}", N, 3_000_008 if N <= 128 else 1_500_008, dtype, 2, "student_flip", seed=N)
     run_case(ac, w, 2, beta=0.9, expect_path=7)
 
 
