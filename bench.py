@@ -63,6 +63,9 @@ def parse_args(argv=None):
     ap.add_argument("--shape", default="", help="N,d,dtype of an ad-hoc Gaussian workload instead of a named one, e.g. 128,20000000,bf16")
     ap.add_argument("--cluster-pass1", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_CLUSTER_PASS1 (64 < N <= 512)")
     ap.add_argument("--tall-tiles", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_TALL_TILES (64 < N <= 256)")
+    ap.add_argument("--column-sharded", action="store_true",
+                    help="each rank holds its own d columns of ONE matrix of world*d columns: pass 1, an all-gather of the "
+                         "statistics records, coefficient step and pass 2 (default for --gpus N > 1: independent replicas)")
     ap.add_argument("--one-launch", type=int, default=-1, choices=[-1, 0, 1, 2],
                     help="ADACONS_OPT_ONE_LAUNCH (default: the library's own choice by size)")
     return ap.parse_args(argv)
@@ -274,9 +277,19 @@ def run_ours(args):
     if args.tall_tiles >= 0:
         h.set_option(ac.OPT_TALL_TILES, args.tall_tiles)
     stream = torch.cuda.current_stream()
+    if args.column_sharded:
+        from paper_2411_03742_b200.sharded import ColumnSharded
+        sh = ColumnSharded(h, rank, world, device=dev)
+        args.no_profile = True        # the two halves are separate calls: only the whole step is timed
+
+        def step_fn(Gt):
+            sh.aggregate(Gt, out)
+    else:
+        def step_fn(Gt):
+            h.aggregate(Gt, out)
 
     for t in range(max(args.warmup, 3)):
-        h.aggregate(Gs[t % nbuf], out)
+        step_fn(Gs[t % nbuf])
     torch.cuda.synchronize()
     # A timed region that saw a thermal or hardware slowdown is measured once more.
     for attempt in range(2):
@@ -290,7 +303,7 @@ def run_ours(args):
         sampler.start()
         ev0.record(stream)
         for t in range(args.steps):
-            h.aggregate(Gs[t % nbuf], out)
+            step_fn(Gs[t % nbuf])
         ev1.record(stream)
         torch.cuda.synchronize()
         clocks = sampler.stop()
@@ -302,12 +315,12 @@ def run_ours(args):
         clocks["remeasured"] = attempt > 0
         if not slowed_anywhere:
             break
-    if args.no_profile:
+    if args.no_profile and not args.column_sharded:
         h.set_option(ac.OPT_PROFILE, 1)
         for t in range(args.steps):
-            h.aggregate(Gs[t % nbuf], out)
+            step_fn(Gs[t % nbuf])
         torch.cuda.synchronize()
-    kernel_ms, kcalls = h.profile()
+    kernel_ms, kcalls = ([0.0, 0.0, 0.0], args.steps) if args.column_sharded else h.profile()
     extra = {}
     if not args.no_extra_loops:
         # (a) the launch sequence a user gets: no events between the kernels, so the coefficient
@@ -317,14 +330,14 @@ def run_ours(args):
         torch.cuda.synchronize()
         e0.record(stream)
         for t in range(args.steps):
-            h.aggregate(Gs[t % nbuf], out)
+            step_fn(Gs[t % nbuf])
         e1.record(stream)
         torch.cuda.synchronize()
         extra["ms_per_step_no_kernel_events"] = e0.elapsed_time(e1) / args.steps
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
         evs[0].record(stream)
         for t in range(args.steps):
-            h.aggregate(Gs[t % nbuf], out)
+            step_fn(Gs[t % nbuf])
             evs[t + 1].record(stream)
         torch.cuda.synchronize()
         per = sorted(evs[t].elapsed_time(evs[t + 1]) for t in range(args.steps))
@@ -344,7 +357,11 @@ def run_ours(args):
 
     # roofline of the dominant kernel, from CUDA events recorded around it inside the timed region
     peak, peak_src = measured_peak_gbs()
-    if path == 3:     # single-pass kernel: the matrix is read from HBM once
+    if args.column_sharded:   # the step as a whole (two calls and, with several ranks, the exchange between them)
+        alg = {"step": step_bytes}
+        kms = {"step": ms_local / args.steps}
+        dom = "step"
+    elif path == 3:     # single-pass kernel: the matrix is read from HBM once
         alg = {"fused": float(w.N) * w.d * b + w.d * b}
         kms = {"fused": kernel_ms[0]}
         dom = "fused"
@@ -374,7 +391,11 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "storage_dtype": w.dtype, "data": "synthetic",
         "config": {"workload": describe(w), "N": w.N, "d": w.d, "storage_dtype": w.dtype,
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "parallelism": (("column-sharded: every GPU holds all N rows of its own d columns; per step one all-gather "
+                                    f"of {h.stats_doubles} doubles per GPU, summed in rank order inside the coefficient kernel")
+                                   if args.column_sharded and world > 1 else
+                                   "single GPU, the step in two halves (adacons_pass1, adacons_finish)" if args.column_sharded else
+                                   "replicas only" if world > 1 else "single GPU"),
                    "coefficients": "per segment" if args.per_segment else "model-wise",
                    "path": {1: "three kernels (TMA-staged pass 1)", 3: "single-pass kernel (matrix in shared memory)",
                             4: "N > 64: column sums, dot products per 64 rows, pass 2 (three reads)",

@@ -177,13 +177,15 @@ enum adacons_info {
                                         8 = misaligned base, aligned body: TMA-staged pass 1 plus
                                             the head columns (see ADACONS_OPT_ALIGNED_BODY)      */
   ADACONS_INFO_TOTAL_LAUNCHES = 6,   /* kernels launched by this context so far                  */
-  ADACONS_INFO_LAST_PASS2 = 7        /* pass-2 kernel of the most recent aggregate call: 0 = none
+  ADACONS_INFO_LAST_PASS2 = 7,       /* pass-2 kernel of the most recent aggregate call: 0 = none
                                         (no call yet, or the single-pass kernel), 1 = generic,
                                         2 = 16-byte vectors, 3 = 32-byte vectors (grads, out and
                                         the row pitch 32-byte aligned), 4 = the second phase of
                                         the one-launch kernel (TMA-staged chunks of 8 rows),
                                         5 = vector kernel on the aligned body plus element-wise
                                         edges (grads and out off a 16-byte boundary alike)       */
+  ADACONS_INFO_STATS_DOUBLES = 8     /* doubles in one shard's statistics (adacons_pass1):
+                                        sets * (2 N + 1)                                         */
 };
 
 /*
@@ -224,6 +226,39 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  * context without its buffers; destroy it).
  */
 int adacons_aggregate(adacons_ctx *ctx, const void *grads, void *out, void *cuda_stream);
+
+/*
+ * The step in two halves, for a matrix whose COLUMNS are spread over several devices (device r
+ * holds columns [c_r, c_{r+1}) of all N rows, one context per device created with the shard's own
+ * d).  The statistics of Eq. 7 are sums over columns, so the shards' sums add up to the whole
+ * matrix's: every device computes its own, the caller exchanges them (an all-gather of a few
+ * KB; nothing else of the step crosses devices), and every device finishes with the same
+ * coefficients, each on its own columns.  The paper spreads the WORKERS over devices instead and
+ * needs two all-reduces of d elements (Algorithm 1, steps 1 and 4); this form is its single-
+ * device arithmetic (Eq. 7, Eq. 11, Eq. 12-13) on another layout, not a step the paper prints.
+ *
+ * adacons_pass1: pass 1 on this shard.
+ *   stats  device pointer, 8-byte aligned, receives ADACONS_INFO_STATS_DOUBLES doubles: per
+ *          coefficient set the N sums sum_k g_ik s_k (N p_i of Eq. 7 before the division by N),
+ *          the N squared norms q_i, and the set's number of columns on this shard.
+ *   Changes neither the momentum state nor the step counter.
+ * adacons_finish: coefficients from all shards' statistics, then pass 2 on this shard.
+ *   stats  device pointer: `shards` records of ADACONS_INFO_STATS_DOUBLES doubles each, in the
+ *          same shard order on every device; they are added in that order in fp64, so all
+ *          devices get the same bits (coefficients, weights, state).
+ *   grads, out  as for adacons_aggregate (the same matrix that adacons_pass1 was given).
+ *   Advances the momentum state by one step.  With one shard, adacons_pass1 followed by
+ *   adacons_finish gives the bits of adacons_aggregate's three-kernel path.
+ * Per-segment mode: give every shard's context ALL the segments, clipped to the shard's column
+ * range (segments that lie elsewhere become empty); the sets then line up across shards.  A set is
+ * "without columns" (no flags, see adacons_flag) only if it is empty on every shard.
+ * Both calls are asynchronous on `cuda_stream`, allocate nothing and never take the one-launch
+ * or single-pass paths.  Errors: as adacons_aggregate; EINVAL also for a NULL or misaligned
+ * `stats` and shards < 1.
+ */
+int adacons_pass1(adacons_ctx *ctx, const void *grads, double *stats, void *cuda_stream);
+int adacons_finish(adacons_ctx *ctx, const void *grads, void *out, const double *stats, int shards,
+                   void *cuda_stream);
 
 /*
  * The same aggregation for callers whose gradients live in HOST memory.

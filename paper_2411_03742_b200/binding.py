@@ -23,7 +23,7 @@ F32, BF16 = 0, 1
 COEFF_A, COEFF_A_TILDE, COEFF_GAMMA, COEFF_P, COEFF_Q = range(5)
 # enum adacons_info
 (INFO_NUM_SEGMENTS, INFO_COEFF_SETS, INFO_PASS1_BLOCKS, INFO_SCRATCH_BYTES, INFO_LAUNCHES_PER_CALL,
- INFO_LAST_PATH, INFO_TOTAL_LAUNCHES, INFO_LAST_PASS2) = range(8)
+ INFO_LAST_PATH, INFO_TOTAL_LAUNCHES, INFO_LAST_PASS2, INFO_STATS_DOUBLES) = range(9)
 # enum adacons_flag
 FLAG_ZERO_ROW, FLAG_DEGENERATE_Z, FLAG_NONFINITE, FLAG_NEG_Z, FLAG_TIMEOUT = 1, 2, 4, 8, 0x100
 # enum adacons_error
@@ -58,6 +58,8 @@ def load_library() -> ctypes.CDLL:
         "adacons_create": [P(vp), i32, i64, i32, P(i64), i32],
         "adacons_aggregate": [vp, vp, vp, vp],
         "adacons_aggregate_host": [vp, vp, vp, vp],
+        "adacons_pass1": [vp, vp, vp, vp],
+        "adacons_finish": [vp, vp, vp, vp, i32, vp],
         "adacons_reset": [vp, vp],
         "adacons_destroy": [vp],
         "adacons_set_option": [vp, i32, dbl],
@@ -207,6 +209,38 @@ class AdaCons:
         gp = host_grads.data_ptr() if hasattr(host_grads, "data_ptr") else host_grads.ctypes.data
         op = host_out.data_ptr() if hasattr(host_out, "data_ptr") else host_out.ctypes.data
         _check(self._lib.adacons_aggregate_host(self._ctx, gp, op, _stream_handle(stream)), "adacons_aggregate_host")
+
+    # -- the step in two halves, for a matrix whose columns are spread over devices ----------------
+    @property
+    def stats_doubles(self) -> int:
+        """Doubles in one shard's statistics record: sets * (2 N + 1)."""
+        return self.info(INFO_STATS_DOUBLES)
+
+    def _check_stats(self, stats, least: int, what: str) -> None:
+        import torch
+        if not (stats.is_cuda and stats.dtype == torch.float64 and stats.is_contiguous() and stats.numel() >= least):
+            raise ValueError(f"{what} must be a contiguous float64 CUDA tensor of at least {least} elements")
+
+    def pass1(self, grads, stats, stream=None) -> None:
+        """Pass 1 on this shard's columns; `stats` (float64 CUDA, stats_doubles elements) receives the
+        shard's statistics.  No state change."""
+        if grads.device != stats.device:
+            raise ValueError("grads and stats must be on the same device")
+        self._check_stats(stats, self.stats_doubles, "stats")
+        check_tensors(self.N, self.d, self.dtype, self._pitch, grads, grads[0], want_cuda=True)
+        _check(self._lib.adacons_pass1(self._ctx, grads.data_ptr(), stats.data_ptr(), _stream_handle(stream)), "adacons_pass1")
+
+    def finish(self, grads, out, stats_all, shards: int, stream=None) -> None:
+        """Coefficients from the statistics of all `shards` shards (stats_all: shards x stats_doubles,
+        the same order on every device), then pass 2 on this shard's columns."""
+        if int(shards) < 1:
+            raise ValueError("shards must be at least 1")
+        if grads.device != stats_all.device:
+            raise ValueError("grads and stats_all must be on the same device")
+        self._check_stats(stats_all, int(shards) * self.stats_doubles, "stats_all")
+        check_tensors(self.N, self.d, self.dtype, self._pitch, grads, out)
+        _check(self._lib.adacons_finish(self._ctx, grads.data_ptr(), out.data_ptr(), stats_all.data_ptr(), int(shards),
+                                        _stream_handle(stream)), "adacons_finish")
 
     def reset(self, stream=None) -> None:
         _check(self._lib.adacons_reset(self._ctx, _stream_handle(stream)), "adacons_reset")

@@ -804,16 +804,28 @@ int adacons_destroy(adacons_ctx* c) {
   return ADACONS_OK;
 }
 
-int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_stream) {
-  if (c == nullptr || grads == nullptr || out == nullptr) return ADACONS_EINVAL;
+}  // extern "C"
+
+namespace {
+
+// Which part of a step a call runs: all of it, or one half of the column-sharded form.
+enum Phase { kWholeStep = 0, kStatisticsOnly = 1, kFromStatistics = 2 };
+
+int run_step(adacons_ctx* c, const void* grads, void* out, void* cuda_stream, Phase phase, double* stats_out,
+             const double* stats_in, int shards) {
+  if (c == nullptr || grads == nullptr) return ADACONS_EINVAL;
+  if (phase != kStatisticsOnly && out == nullptr) return ADACONS_EINVAL;
+  if (phase == kStatisticsOnly && (stats_out == nullptr || reinterpret_cast<uintptr_t>(stats_out) % 8 != 0)) return ADACONS_EINVAL;
+  if (phase == kFromStatistics && (stats_in == nullptr || shards < 1 || reinterpret_cast<uintptr_t>(stats_in) % 8 != 0)) return ADACONS_EINVAL;
   // an option change that ran out of memory half-way leaves the context without its buffers
   if (c->partials == nullptr || c->coef == nullptr || c->gamma_f32 == nullptr || c->m == nullptr || c->z == nullptr)
     return ADACONS_ENOMEM;
   // with padded rows the vector loads may touch the last row's padding too: the matrix is N * pitch elements
   const size_t gbytes = static_cast<size_t>(c->N) * c->pitch * c->elem_bytes;
   const size_t obytes = static_cast<size_t>(c->d) * c->elem_bytes;
-  const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads), o0 = reinterpret_cast<uintptr_t>(out);
-  if (o0 < g0 + gbytes && g0 < o0 + obytes) return ADACONS_EINVAL;   // out overlaps grads
+  // the statistics half writes no result: `out` then only stands for "as aligned as grads"
+  const uintptr_t g0 = reinterpret_cast<uintptr_t>(grads), o0 = phase == kStatisticsOnly ? g0 : reinterpret_cast<uintptr_t>(out);
+  if (phase != kStatisticsOnly && o0 < g0 + gbytes && g0 < o0 + obytes) return ADACONS_EINVAL;   // out overlaps grads
   DeviceGuard guard(c->device);
   if (!guard.ok) return ADACONS_ECUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -826,19 +838,19 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   const int tail_elems = static_cast<int>((c->d * c->elem_bytes % 16) / c->elem_bytes);   // 0: the last group is full
   const long long row_bytes = c->pitch * c->elem_bytes;
   const int N = c->N;
-  int num_partials;
+  int num_partials = 0;
   int extra_launches = 0;
-  cudaEvent_t* ev = (c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
+  cudaEvent_t* ev = (phase == kWholeStep && c->profile && c->prof_ready) ? c->prof_ev[c->prof_calls % adacons_ctx::kProfSlots] : nullptr;
   if (ev) cudaEventRecord(ev[0], st);
 
   // the coefficient kernel may be launched while pass 1 still runs (it waits for it on the device);
   // event records between the kernels would defeat that
-  const bool pdl = (ev == nullptr) && c->overlap_launch;
+  const bool pdl = (ev == nullptr) && c->overlap_launch && phase != kFromStatistics;
   const bool seg = c->per_segment != 0;
   if (seg && !(aligned && c->fast.available && c->seg_kernel != nullptr)) return ADACONS_EALIGN;
 
   // ---- single-pass path: the whole matrix fits in the grid's shared memory ----
-  if (!seg && aligned && c->fused_available && c->fused_small) {
+  if (phase == kWholeStep && !seg && aligned && c->fused_available && c->fused_small) {
     FusedParams f;
     f.N = N; f.num_vec = num_vec; f.tail_elems = tail_elems; f.row_bytes = row_bytes; f.vec_per_block = c->fused_vpb;
     f.grads = static_cast<const unsigned char*>(grads); f.out = static_cast<unsigned char*>(out);
@@ -864,7 +876,7 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   }
 
   // ---- one launch, two reads: mid-size matrices ----
-  if (!seg && aligned && c->mid_available &&
+  if (phase == kWholeStep && !seg && aligned && c->mid_available &&
       (c->one_launch == 2 ||
        (c->one_launch == 1 && static_cast<long long>(c->N) * row_bytes <= kOneLaunchMaxBytes))) {
     int rc = encode_map(c, grads);
@@ -897,7 +909,9 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   }
 
   // ---- pass 1 (Eq. 7) ----
-  if (seg) {
+  if (phase == kFromStatistics) {
+    // the statistics come from the caller
+  } else if (seg) {
     int rc = encode_map(c, grads);
     if (rc != ADACONS_OK) return rc;
     Pass1SegParams p;
@@ -1026,6 +1040,9 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   q.seg_off = seg ? c->d_seg_off : nullptr;
   q.coef = c->coef; q.gamma_f32 = c->gamma_f32; q.m = c->m; q.z = c->z;
   q.flags = c->flags; q.step = c->step;
+  q.cols = c->d;
+  if (phase == kStatisticsOnly) q.stats_out = stats_out;
+  if (phase == kFromStatistics) { q.stats_in = stats_in; q.shards = shards; }
   int cthreads = 1024;
   if (seg) { cthreads = ((2 * N + 31) / 32) * 32; if (cthreads > 1024) cthreads = 1024; }
   if (launch_kernel(coeff_kernel, dim3(c->sets()), dim3(cthreads), 0, st, pdl, q) != cudaSuccess) {
@@ -1033,6 +1050,11 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
     return ADACONS_ECUDA;
   }
   if (ev) cudaEventRecord(ev[2], st);
+  if (phase == kStatisticsOnly) {
+    c->last_launches = 2 + extra_launches;
+    c->total_launches += c->last_launches;
+    return ADACONS_OK;
+  }
 
   // ---- pass 2 (Eq. 12) ----
   cudaError_t e2;
@@ -1101,9 +1123,25 @@ int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_s
   }
   if (e2 != cudaSuccess) { cudaGetLastError(); return ADACONS_ECUDA; }
   if (ev) { cudaEventRecord(ev[3], st); c->prof_calls += 1; }
-  c->last_launches = 3 + extra_launches;
+  c->last_launches = (phase == kFromStatistics ? 2 : 3) + extra_launches;
   c->total_launches += c->last_launches;
   return ADACONS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int adacons_aggregate(adacons_ctx* c, const void* grads, void* out, void* cuda_stream) {
+  return run_step(c, grads, out, cuda_stream, kWholeStep, nullptr, nullptr, 0);
+}
+
+int adacons_pass1(adacons_ctx* c, const void* grads, double* stats, void* cuda_stream) {
+  return run_step(c, grads, nullptr, cuda_stream, kStatisticsOnly, stats, nullptr, 0);
+}
+
+int adacons_finish(adacons_ctx* c, const void* grads, void* out, const double* stats, int shards, void* cuda_stream) {
+  return run_step(c, grads, out, cuda_stream, kFromStatistics, nullptr, stats, shards);
 }
 
 int adacons_aggregate_host(adacons_ctx* c, const void* host_grads, void* host_out, void* cuda_stream) {
@@ -1363,6 +1401,7 @@ int adacons_get_info(adacons_ctx* c, int key, int64_t* value) {
     case ADACONS_INFO_LAST_PATH: *value = c->last_path; return ADACONS_OK;
     case ADACONS_INFO_TOTAL_LAUNCHES: *value = c->total_launches; return ADACONS_OK;
     case ADACONS_INFO_LAST_PASS2: *value = c->last_pass2; return ADACONS_OK;
+    case ADACONS_INFO_STATS_DOUBLES: *value = static_cast<int64_t>(c->sets()) * (2 * c->N + 1); return ADACONS_OK;
     default: return ADACONS_EINVAL;
   }
 }

@@ -26,21 +26,33 @@ struct CoeffParams {
   double* z;             // [sets]      normaliser Z = sum_i u_i of the last call (NaN if not computed)
   uint32_t* flags;       // device status word (OR)
   long long* step;       // aggregation counter
+  // Column-sharded use (coeff_kernel only).  A statistics record of one set is 2N + 1 doubles: the N
+  // sums sum_k g_ik s_k over the set's columns (N p_i of Eq. 7 before the division), the N squared
+  // norms q_i, and the number of columns.  stats_out != nullptr: write this set's record (from the
+  // partial records, in the usual order) and stop -- no coefficient, no state change.  stats_in !=
+  // nullptr: take the statistics from `shards` records per set, [shard][set][2N + 1], added in shard
+  // order, instead of from partial records.
+  double* stats_out = nullptr;
+  const double* stats_in = nullptr;
+  int shards = 0;
+  long long cols = 0;    // global mode: columns of the one set (for the record's last entry)
 };
 
 // Work arrays in shared memory: sh_part holds part_cap doubles (at least 2N), sh_a, sh_u and sh_m N each.
 // The records are split into `groups` interleaved subsequences, which fixes the order of the fp64
 // sum; groups follows from N, part_cap and group_threads alone (not from the block size), so two
 // kernels that pass the same values add the same records in the same order.
+// EXT: the kernel honours stats_out / stats_in (the fused kernels have no use for them).
+template <bool EXT = false>
 __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set, double* sh_part, const int part_cap,
                                            const int group_threads, double* sh_a, double* sh_u, double* sh_m) {
-  __shared__ int sh_bad, sh_zero;
+  __shared__ int sh_bad, sh_zero, sh_nocols;
   __shared__ double sh_Z;
   __shared__ int sh_uniform;
   const int N = prm.N, i = threadIdx.x, T = blockDim.x;
   const int V = 2 * N;
   const size_t per = static_cast<size_t>(prm.sets) * N;   // stride between coefficient kinds
-  if (i == 0) { sh_bad = 0; sh_zero = 0; }
+  if (i == 0) { sh_bad = 0; sh_zero = 0; }   // sh_nocols: written by one thread, and only read, with external statistics
   if (i < N) sh_m[i] = prm.m[static_cast<size_t>(set) * N + i];   // the old state, fetched while the partials are summed
   const int begin = prm.rec_begin ? prm.rec_begin[set] : 0;
   const int count = prm.rec_count ? prm.rec_count[set] : prm.num_partials;
@@ -53,7 +65,18 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
   if (groups > 32) groups = 32;
   if (groups > part_cap / V) groups = part_cap / V;
   if (groups < 1) groups = 1;
-  for (int slot = i; slot < units * groups; slot += T) {
+  const bool external = EXT && prm.stats_in != nullptr;
+  if (external) {                                          // the shards' records of this set, in shard order
+    groups = 1;
+    const size_t rec = static_cast<size_t>(V) + 1;
+    for (int e = i; e <= V; e += T) {
+      double acc = 0.0;
+      for (int r = 0; r < prm.shards; ++r) acc += prm.stats_in[(static_cast<size_t>(r) * prm.sets + set) * rec + e];
+      if (e < V) sh_part[e] = acc;
+      else sh_nocols = acc == 0.0 ? 1 : 0;
+    }
+  }
+  for (int slot = i; !external && slot < units * groups; slot += T) {
     const int g = slot / units, u = slot - g * units;
     double acc[4] = {0.0, 0.0, 0.0, 0.0};
     const float* src = base + static_cast<size_t>(u) * w;
@@ -89,6 +112,12 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
   if (i < N) {
     double P = 0.0, Q = 0.0;
     for (int g = 0; g < groups; ++g) { P += sh_part[g * V + i]; Q += sh_part[g * V + N + i]; }
+    if (EXT && prm.stats_out != nullptr) {
+      double* rec = prm.stats_out + static_cast<size_t>(set) * (V + 1);
+      rec[i] = P;
+      rec[N + i] = Q;
+      if (i == 0) rec[V] = static_cast<double>(prm.seg_off ? prm.seg_off[set + 1] - prm.seg_off[set] : prm.cols);
+    }
     p = P / static_cast<double>(N);   // gbar is the mean of the workers (text before Eq. 7)
     q = Q;
     if (!(isfinite(p) && isfinite(q))) atomicOr(&sh_bad, 1);
@@ -96,10 +125,12 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
     prm.coef[3 * per + set * N + i] = p;
     prm.coef[4 * per + set * N + i] = q;
   }
+  if (EXT && prm.stats_out != nullptr) return;              // uniform: the whole block leaves
   __syncthreads();
   // A segment without columns is no layer: its all-zero statistics take the usual fallbacks
   // (weights 1/N, state unchanged at zero) but are no degeneracy of the data and raise no flag.
-  const bool empty_set = prm.seg_off != nullptr && prm.seg_off[set + 1] == prm.seg_off[set];
+  // (with external statistics: no columns on any shard)
+  const bool empty_set = external ? sh_nocols != 0 : (prm.seg_off != nullptr && prm.seg_off[set + 1] == prm.seg_off[set]);
   uint32_t flags = (sh_zero && !empty_set) ? kFlagZeroRow : 0u;
   const double uniform = 1.0 / static_cast<double>(N);
   if (sh_bad) {   // non-finite statistic: plain mean, momentum state left as it was
@@ -163,19 +194,20 @@ __device__ __forceinline__ void coeff_core(const CoeffParams& prm, const int set
   }
 }
 
+template <bool EXT = false>
 __device__ __forceinline__ void coeff_body(const CoeffParams& prm, const int set) {
   __shared__ double sh_part[2 * kMaxN];
   __shared__ double sh_a[kMaxN];
   __shared__ double sh_u[kMaxN];
   __shared__ double sh_m[kMaxN];
-  coeff_core(prm, set, sh_part, 2 * kMaxN, static_cast<int>(blockDim.x), sh_a, sh_u, sh_m);
+  coeff_core<EXT>(prm, set, sh_part, 2 * kMaxN, static_cast<int>(blockDim.x), sh_a, sh_u, sh_m);
 }
 
 __global__ void __launch_bounds__(kMaxN)
 coeff_kernel(const CoeffParams prm) {
   pdl_launch_dependents();
   pdl_wait();                                              // pass 1 has finished and is visible
-  coeff_body(prm, blockIdx.x);
+  coeff_body<true>(prm, blockIdx.x);
 }
 
 }  // namespace adacons
