@@ -66,6 +66,7 @@ def parse_args(argv=None):
     ap.add_argument("--column-sharded", action="store_true",
                     help="each rank holds its own d columns of ONE matrix of world*d columns: pass 1, an all-gather of the "
                          "statistics records, coefficient step and pass 2 (default for --gpus N > 1: independent replicas)")
+    ap.add_argument("--gram-pass1", type=int, default=-1, help="ADACONS_OPT_GRAM_PASS1 (bf16, N <= 64): tiles per first-level sum; 0 = off")
     ap.add_argument("--one-launch", type=int, default=-1, choices=[-1, 0, 1, 2],
                     help="ADACONS_OPT_ONE_LAUNCH (default: the library's own choice by size)")
     return ap.parse_args(argv)
@@ -276,6 +277,8 @@ def run_ours(args):
         h.set_option(ac.OPT_ONE_LAUNCH, args.one_launch)
     if args.cluster_pass1 >= 0:
         h.set_option(ac.OPT_CLUSTER_PASS1, args.cluster_pass1)
+    if args.gram_pass1 >= 0:
+        h.set_option(ac.OPT_GRAM_PASS1, args.gram_pass1)
     if args.tall_tiles >= 0:
         h.set_option(ac.OPT_TALL_TILES, args.tall_tiles)
     stream = torch.cuda.current_stream()
@@ -348,7 +351,7 @@ def run_ours(args):
     status = h.status()
     assert status == 0, f"library raised status flags {status:#x}"
     path = h.info(ac.INFO_LAST_PATH)
-    assert path in (1, 3, 4, 5, 6, 7), "benchmark must run an aligned path"
+    assert path in (1, 3, 4, 5, 6, 7, 9), "benchmark must run an aligned path"
 
     units_local = float(w.N) * w.d * args.steps
     ms, units = reduce_over_ranks(ms_local, units_local, device=dev)
@@ -403,6 +406,7 @@ def run_ours(args):
                             4: "N > 64: column sums, dot products per 64 rows, pass 2 (three reads)",
                             6: "N > 64: cluster pass 1 (one read), coefficient step, pass 2",
                             7: "64 < N <= 256: pass 1 on 128- or 256-row tiles (one read), coefficient step, pass 2",
+                            9: "pass 1 from the Gram matrix on the tensor cores, coefficient step, pass 2",
                             5: "one launch, two reads (pass 1, coefficient step, pass 2 in one cooperative kernel)"}[path],
                    "l2": (f"inputs ({gbytes / 1e9:.2f} GB) larger than the 126 MB L2; no flush between steps" if nbuf == 1 else
                           f"two distinct input matrices of {gbytes / 1e9:.2f} GB used in turn, each larger than the 126 MB L2; no flush"

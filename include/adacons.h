@@ -131,6 +131,18 @@ enum adacons_option {
                                   buffers take the generic path, as a pitch that is not a
                                   multiple of 16 bytes always does.  Same results either way to
                                   fp32 accumulation order.                                       */
+  ADACONS_OPT_GRAM_PASS1 = 13,  /* bf16, N <= 64, aligned buffers, d <= 2^30.  n >= 1: pass 1 takes
+                                  the statistics from the Gram matrix of every column tile,
+                                  computed on the tensor cores (Eq. 7, third line: N p_i is the
+                                  i-th row sum of G G^T, q_i its diagonal), with n tiles of 256
+                                  columns per first-level accumulation (integer, 1..32).  The
+                                  tensor cores round their running sums toward zero: a sum of
+                                  squares comes out low by about 4e-8 relative per chained
+                                  product (four per tile), hence the bound on n (n = 16: q_i
+                                  low by 2e-6 to 3e-6).  0 (default):
+                                  column sums and dot products on the fp32 pipes, which is both
+                                  more accurate and, as measured, faster; the option exists
+                                  for comparison.                                                */
   ADACONS_OPT_TALL_TILES = 11, /* 1 (default): with 64 < N <= 256 on aligned buffers pass 1 reads the
                                   matrix ONCE, as for N <= 64, from taller and narrower tiles:
                                   128 rows x 256 bytes (half a warp per row) up to N = 128,
@@ -175,7 +187,9 @@ enum adacons_info {
                                         7 = 64 < N <= 256: tiles of 128 or 256 rows, one read in pass 1
                                             (see ADACONS_OPT_TALL_TILES),
                                         8 = misaligned base, aligned body: TMA-staged pass 1 plus
-                                            the head columns (see ADACONS_OPT_ALIGNED_BODY)      */
+                                            the head columns (see ADACONS_OPT_ALIGNED_BODY),
+                                        9 = pass 1 from the Gram matrix on the tensor cores
+                                            (see ADACONS_OPT_GRAM_PASS1)                         */
   ADACONS_INFO_TOTAL_LAUNCHES = 6,   /* kernels launched by this context so far                  */
   ADACONS_INFO_LAST_PASS2 = 7,       /* pass-2 kernel of the most recent aggregate call: 0 = none
                                         (no call yet, or the single-pass kernel), 1 = generic,

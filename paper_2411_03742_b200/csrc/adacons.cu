@@ -118,6 +118,11 @@ struct adacons_ctx {
   int cl_size = 0, cl_grid = 0, cl_tiles = 0;
   size_t cl_smem = 0;
   int cluster_pass1 = 0;                // ADACONS_OPT_CLUSTER_PASS1 (opt-in)
+  // bf16, N <= 64: pass 1 from the Gram matrix on the tensor cores (pass1_gram_kernel)
+  bool gram_available = false;
+  int gram_grid = 0, gram_tiles = 0, gram_stages = 2;
+  size_t gram_smem = 0;
+  int gram_fold = 0;                    // ADACONS_OPT_GRAM_PASS1: 0 = off, n >= 1 = on, n tiles per first-level sum
   int last_launches = 3;
 
   // single-pass path for problems that fit in the grid's shared memory
@@ -411,6 +416,27 @@ int plan_cluster(adacons_ctx* c) {
   c->cl_grid = clusters * c->cl_size;
   c->cl_smem = smem;
   c->cl_available = true;
+  return ADACONS_OK;
+}
+
+// bf16 and N <= 64 on the aligned path: the Gram-matrix pass 1 (pass1_gram_kernel); shares tmap_big (64-row boxes).
+int plan_gram(adacons_ctx* c) {
+  c->gram_available = false;
+  if (c->dtype != ADACONS_BF16 || c->N > kMaxFastN) return ADACONS_OK;
+  if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > kChunkCols) return ADACONS_OK;
+  c->gram_tiles = static_cast<int>((c->d + 255) / 256);
+  c->gram_stages = 2;
+  c->gram_smem = static_cast<size_t>(c->gram_stages) * kGramStageBytes + kGramSecondBytes + static_cast<size_t>(2 * c->gram_stages) * 8;
+  const void* k = reinterpret_cast<const void*>(&pass1_gram_kernel);
+  int per_sm = 0;
+  if (c->gram_smem > kPass1SmemCap || !set_smem_cap(k, kPass1SmemCap) ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, c->gram_smem) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  c->gram_grid = per_sm * c->num_sms;
+  if (c->gram_grid > c->gram_tiles) c->gram_grid = c->gram_tiles;
+  c->gram_available = true;
   return ADACONS_OK;
 }
 
@@ -768,6 +794,8 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   if (c->big_available && c->big_grid > c->max_partials) c->max_partials = c->big_grid;
   plan_cluster(c);
   if (c->cl_available && c->cl_grid / c->cl_size > c->max_partials) c->max_partials = c->cl_grid / c->cl_size;
+  plan_gram(c);
+  if (c->gram_available && c->gram_grid > c->max_partials) c->max_partials = c->gram_grid;
   plan_tall(c);
   if (c->tall_available && c->tall_grid > c->max_partials) c->max_partials = c->tall_grid;
 
@@ -926,6 +954,20 @@ int run_step(adacons_ctx* c, const void* grads, void* out, void* cuda_stream, Ph
     }
     num_partials = 0;
     c->last_path = 1;
+  } else if (g_aligned && c->gram_available && c->gram_fold > 0) {
+    int rc = encode_map_big(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    GramParams p;
+    p.N = N; p.num_tiles = c->gram_tiles; p.stages = c->gram_stages; p.fold_tiles = c->gram_fold;
+    p.partials = c->partials; p.flags = c->flags;
+    void* args[2] = {&c->tmap_big, &p};
+    if (cudaLaunchKernel(reinterpret_cast<const void*>(&pass1_gram_kernel), dim3(c->gram_grid), dim3(kThreads), args,
+                         c->gram_smem, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    num_partials = c->gram_grid;
+    c->last_path = 9;
   } else if (g_aligned && c->fast.available) {
     int rc = encode_map(c, grads);
     if (rc != ADACONS_OK) return rc;
@@ -1216,6 +1258,10 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
     case ADACONS_OPT_OVERLAP_LAUNCH: c->overlap_launch = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_FUSED_SMALL: c->fused_small = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_CLUSTER_PASS1: c->cluster_pass1 = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_GRAM_PASS1:
+      if (value < 0.0 || value > 32.0 || value != static_cast<double>(static_cast<int>(value))) return ADACONS_EINVAL;
+      c->gram_fold = static_cast<int>(value);
+      return ADACONS_OK;
     case ADACONS_OPT_TALL_TILES: c->tall_tiles_opt = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_ALIGNED_BODY: c->aligned_body = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_ONE_LAUNCH:
@@ -1245,12 +1291,14 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       if (rc != ADACONS_OK) return rc;
       plan_cluster(c);
       plan_tall(c);
+      plan_gram(c);
       int need = c->generic_grid;
       if (c->fast.available && c->fast.grid * c->num_chunks > need) need = c->fast.grid * c->num_chunks;
       if (c->fused_available && c->fused_grid > need) need = c->fused_grid;
       if (c->big_available && c->big_grid > need) need = c->big_grid;
       if (c->cl_available && c->cl_grid / c->cl_size > need) need = c->cl_grid / c->cl_size;
       if (c->tall_available && c->tall_grid > need) need = c->tall_grid;
+      if (c->gram_available && c->gram_grid > need) need = c->gram_grid;
       need += 1;                             // the head columns' record (aligned-body path)
       if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
         cudaFree(c->partials);
@@ -1298,6 +1346,7 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_TALL_TILES: *value = c->tall_tiles_opt; return ADACONS_OK;
     case ADACONS_OPT_ALIGNED_BODY: *value = c->aligned_body; return ADACONS_OK;
     case ADACONS_OPT_CLUSTER_PASS1: *value = c->cluster_pass1; return ADACONS_OK;
+    case ADACONS_OPT_GRAM_PASS1: *value = c->gram_fold; return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: *value = static_cast<double>(c->pitch); return ADACONS_OK;
     default: return ADACONS_EINVAL;
   }

@@ -13,6 +13,7 @@
 
 #include "adacons_common.cuh"
 #include "adacons_pass1.cuh"
+#include "adacons_gram.cuh"
 #include "adacons_coeff.cuh"
 #include "adacons_pass2.cuh"
 #include "adacons_fused.cuh"

@@ -1242,3 +1242,37 @@ def test_identical_bf16_gradients_at_scale_are_returned_bit_exactly(ac):
     assert np.all(np.abs(q - q_ref[0]) <= 1e-6 * q_ref[0]) and np.all(np.abs(p - q_ref[0]) <= 1e-6 * q_ref[0])
     np.testing.assert_allclose(h.coeffs()[0], np.full(N, 1.0 / N), rtol=1e-12)
     assert torch.equal(out.view(torch.int16), g.view(torch.int16))
+
+
+# ---- pass 1 from the Gram matrix on the tensor cores (Eq. 7, third line) -----------------------
+@pytest.mark.parametrize("fold", [1, 16, 32])
+@pytest.mark.parametrize("N,d,recipe", [(64, 700_040, "student_flip"), (48, 300_008, "loguniform"), (33, 150_000, "gauss"),
+                                        (16, 400_000, "loguniform"), (5, 90_016, "gauss"), (64, 200, "gauss"), (2, 8, "gauss")])
+def test_gram_pass1(ac, N, d, recipe, fold):
+    """Row sums and diagonal of the tile Gram matrices against the oracle's statistics; rows past N
+    and columns past d come in as zeros; any number of tiles per first-level accumulation."""
+    w = wl.Workload(f"gram{N}x{d}", N, d, "bf16", 3, recipe, seed=17 * N + fold)
+    run_case(ac, w, 3, options={ac.OPT_GRAM_PASS1: fold}, expect_path=9, what=f"gram{N}")
+
+
+def test_gram_pass1_many_tiles_per_block(ac):
+    """A vector long enough that every block walks its ring many times and folds several times (the
+    tensor cores round running sums toward zero: without the second accumulation level q would drift
+    out of tolerance as the vector grows)."""
+    w = wl.Workload("gram-long", 64, 12_000_008, "bf16", 2, "student_flip", seed=77)
+    run_case(ac, w, 2, options={ac.OPT_GRAM_PASS1: 16}, expect_path=9, allow_swaps=False)
+
+
+def test_gram_pass1_option_is_validated_and_ignored_where_it_does_not_apply(ac):
+    h = ac.AdaCons(8, 4096, "f32")
+    for bad in (-1, 0.5, 33):
+        with pytest.raises(ac.AdaConsError):
+            h.set_option(ac.OPT_GRAM_PASS1, bad)
+    h.set_option(ac.OPT_GRAM_PASS1, 16)
+    h.set_option(ac.OPT_FUSED_SMALL, 0); h.set_option(ac.OPT_ONE_LAUNCH, 0)
+    G = torch.randn(8, 4096, device="cuda:0")
+    out = torch.empty(4096, device="cuda:0")
+    h.aggregate(G, out)
+    torch.cuda.synchronize()
+    assert h.info(ac.INFO_LAST_PATH) == 1          # fp32 storage: the ordinary kernel
+    h.close()
