@@ -110,6 +110,12 @@ enum adacons_option {
                                   as data and nothing is written past out[d-1], but the vector
                                   loads may touch it: with a pitch > d the whole N * pitch
                                   elements must be readable (and out must not overlap them).
+                                  The same serves a column range of a wider matrix (base pointer
+                                  at the range's first column, pitch = the matrix's): the
+                                  kernels then read at most 31 bytes past the range in every
+                                  row, other columns of the matrix except after the last row
+                                  of a range that ends the matrix, where those bytes must be
+                                  readable too.
                                   Setting it synchronises the device and may re-allocate scratch. */
   ADACONS_OPT_ONE_LAUNCH = 9,  /* 1 (default): a matrix of up to 1 GiB that does not fit in shared
                                   memory, on 16-byte aligned buffers and pitch with N <= 64, is

@@ -52,8 +52,9 @@ def client(tmp_path_factory):
     return exe
 
 
-def _run(exe, N, d, beta, steps, values, pitch=None):
-    args = [exe, str(N), str(d), repr(beta), str(steps)] + ([str(pitch)] if pitch else [])
+def _run(exe, N, d, beta, steps, values, pitch=None, shards=None):
+    args = [exe, str(N), str(d), repr(beta), str(steps)] + ([str(pitch or d)] if pitch or shards else [])
+    args += [str(shards)] if shards else []
     res = subprocess.run(args, input=" ".join(repr(float(v)) for v in values), capture_output=True, text=True, timeout=120)
     assert res.returncode == 0, res.stderr
     out = []
@@ -91,6 +92,32 @@ def test_collinear_closed_form_through_plain_c(client):
     k = np.array([1.0, 1.0, 1.0, 20.0])
     G = (k[:, None] * x[None, :].astype(np.float64)).astype(np.float32)      # rounded to fp32: collinear to 6e-8
     got = _run(client, 4, d, 0.99, 1, G.ravel())[0]
+    inv = 1.0 / k
+    np.testing.assert_allclose(got["gamma"], inv / inv.sum(), rtol=1e-5)
+    np.testing.assert_allclose(got["out"], (4.0 / inv.sum()) * x.astype(np.float64), rtol=1e-5, atol=1e-5 * np.abs(x).max())
+
+
+def test_hand_worked_example_in_two_halves_through_plain_c(client):
+    """The same rationals from the column-sharded form: one context per column of the d = 2 example
+    (each a 1-column view of the same device matrix, row pitch 2), adacons_pass1 on both, then
+    adacons_finish on both with the two statistics records."""
+    g = _gold()
+    values = np.concatenate([g["step1.G"], g["step2.G"]])
+    got = _run(client, 3, 2, float(g["beta"][0]), 2, values, shards=2)
+    for t, s in enumerate(("step1", "step2")):
+        np.testing.assert_allclose(got[t]["gamma"], g[f"{s}.gamma"], rtol=1e-5, err_msg=f"{s}.gamma")
+        np.testing.assert_allclose(got[t]["m"], g[f"{s}.m"], rtol=1e-5, err_msg=f"{s}.m")
+        np.testing.assert_allclose(got[t]["out"], g[f"{s}.psi"], rtol=1e-5, err_msg=f"{s}.psi")
+        assert got[t]["flags"][0] == 0
+
+
+def test_collinear_closed_form_in_three_ranges_through_plain_c(client):
+    rng = np.random.default_rng(12)
+    d = 4100                                                   # ranges of 1366, 1367, 1367 columns: misaligned views
+    x = rng.standard_normal(d).astype(np.float32)
+    k = np.array([1.0, 2.0, 4.0, 20.0])
+    G = (k[:, None] * x[None, :].astype(np.float64)).astype(np.float32)
+    got = _run(client, 4, d, 0.99, 1, G.ravel(), shards=3)[0]
     inv = 1.0 / k
     np.testing.assert_allclose(got["gamma"], inv / inv.sum(), rtol=1e-5)
     np.testing.assert_allclose(got["out"], (4.0 / inv.sum()) * x.astype(np.float64), rtol=1e-5, atol=1e-5 * np.abs(x).max())
