@@ -179,3 +179,54 @@ def test_bad_arguments_are_refused(ac):
         h.finish(G, out, stats, 0)
     assert h.state()[1] == 0
     h.close()
+
+
+def test_two_halves_replayed_from_a_cuda_graph(ac):
+    """Both halves only enqueue kernels: a whole two-range step can be captured once and replayed."""
+    from parity_util import assert_coeffs
+    dev = torch.device("cuda:0")
+    w = wl.Workload("sharded-graph", 16, 600_000, "bf16", 3, "gauss", seed=31)
+    ranges = column_ranges(w.d, 2, 16)
+    ctxs = [ac.AdaCons(w.N, hi - lo, "bf16") for lo, hi in ranges]
+    n = ctxs[0].stats_doubles
+    stats_all = torch.zeros(2 * n, dtype=torch.float64, device=dev)
+    static = [torch.empty(w.N, hi - lo, dtype=torch.bfloat16, device=dev) for lo, hi in ranges]
+    outs = [torch.empty(hi - lo, dtype=torch.bfloat16, device=dev) for lo, hi in ranges]
+
+    def step():
+        for r in range(2):
+            ctxs[r].pass1(static[r], stats_all[r * n:(r + 1) * n])
+        for r in range(2):
+            ctxs[r].finish(static[r], outs[r], stats_all, 2)
+
+    G = wl.generate(w, 0, dev)
+    for r, (lo, hi) in enumerate(ranges):
+        static[r].copy_(G[:, lo:hi])
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                         # warm-up outside the capture (encodes the tensor maps)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for h in ctxs:
+        h.reset()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    orc = oc.AdaConsOracle(w.N, w.d)
+    for t in range(3):
+        G = wl.generate(w, t, dev)
+        for r, (lo, hi) in enumerate(ranges):
+            static[r].copy_(G[:, lo:hi])
+        graph.replay()
+        torch.cuda.synchronize()
+        G64 = to_f64(G)
+        res = oracle_step(orc, G64, "bf16", ctxs[0].coeffs(ac.COEFF_A), what="sharded graph replay")
+        for h in ctxs:
+            assert_coeffs(h.coeffs(), res["gamma"], f"gamma replay {t}")
+            assert_coeffs(h.state()[0], res["m"], f"m replay {t}")
+        assert_output(torch.cat(outs), res, G64, "bf16", f"sharded replay {t}")
+    assert all(h.state()[1] == 3 and h.status() == 0 for h in ctxs)
+    for h in ctxs:
+        h.close()
