@@ -106,7 +106,7 @@ struct adacons_ctx {
   size_t colsum_bytes = 0;
   CUtensorMap tmap_big;
   const void* tmap_big_for = nullptr;
-  // 64 < N <= 128: one read of the matrix, one block per tile of 128 rows x 256 bytes
+  // 64 < N <= 256: one read of the matrix, one block per tile of 128 rows x 256 bytes or 256 rows x 128 bytes
   bool tall_available = false;
   int tall_grid = 0, tall_tiles = 0, tall_stages = 0, tall_lpr = 16;   // lanes per row: 16 (128-row tiles) or 8 (256-row tiles)
   size_t tall_smem = 0;

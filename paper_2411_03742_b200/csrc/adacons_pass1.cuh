@@ -1,6 +1,6 @@
 // Pass 1 (Eq. 7 of arXiv 2411.03742): column sums, then per worker N p_i = sum_k g_ik s_k and q_i = sum_k g_ik^2,
 // one partial record per block (or per segment a block meets).  All variants: TMA-staged tiles for N <= 64, tall
-// tiles for N <= 128, column sums + dot products for larger N, thread-block clusters (opt-in), per-segment, generic.
+// tiles for N <= 256, column sums + dot products for larger N, thread-block clusters (opt-in), per-segment, generic.
 #pragma once
 
 #include "adacons_common.cuh"
