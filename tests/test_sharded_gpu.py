@@ -230,3 +230,36 @@ def test_two_halves_replayed_from_a_cuda_graph(ac):
     assert all(h.state()[1] == 3 and h.status() == 0 for h in ctxs)
     for h in ctxs:
         h.close()
+
+
+def test_finish_with_non_finite_statistics_falls_back_to_the_mean(ac):
+    """A record that carries NaN (a shard that overflowed) is a non-finite statistic like any other:
+    plain mean on every shard, state left as it was, NONFINITE raised; the next clean step recovers."""
+    dev = torch.device("cuda:0")
+    N, d = 6, 50_000
+    w = wl.Workload("nan-record", N, d, "f32", 2, "gauss", seed=4)
+    h = ac.AdaCons(N, d, "f32")
+    h.set_option(ac.OPT_BETA, 0.5)
+    n = h.stats_doubles
+    stats = torch.empty(2 * n, dtype=torch.float64, device=dev)
+    out = torch.empty(d, device=dev)
+    G = wl.generate(w, 0, dev)
+    h.pass1(G, stats[:n])
+    stats[n:] = 0.0
+    h.finish(G, out, stats, 2)                               # a clean first step (the second record adds nothing)
+    torch.cuda.synchronize()
+    m_before, step_before = h.state()
+    assert step_before == 1 and h.status() == 0
+    G = wl.generate(w, 1, dev)
+    h.pass1(G, stats[:n])
+    stats[n + 2] = float("nan")
+    h.finish(G, out, stats, 2)
+    torch.cuda.synchronize()
+    assert h.status() == ac.FLAG_NONFINITE
+    np.testing.assert_array_equal(h.coeffs(ac.COEFF_GAMMA)[0], np.full(N, 1.0 / N))
+    m_after, step_after = h.state()
+    np.testing.assert_array_equal(m_after, m_before)
+    assert step_after == 2
+    mean = to_f64(G).mean(axis=0)
+    assert np.max(np.abs(to_f64(out) - mean)) <= 1e-5 * float(G.abs().max())
+    h.close()
