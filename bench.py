@@ -62,7 +62,7 @@ def parse_args(argv=None):
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--shape", default="", help="N,d,dtype of an ad-hoc Gaussian workload instead of a named one, e.g. 128,20000000,bf16")
     ap.add_argument("--cluster-pass1", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_CLUSTER_PASS1 (64 < N <= 512)")
-    ap.add_argument("--tall-tiles", type=int, default=-1, choices=[-1, 0, 1], help="ADACONS_OPT_TALL_TILES (64 < N <= 256)")
+    ap.add_argument("--tall-tiles", type=int, default=-1, choices=[-1, 0, 1, 2], help="ADACONS_OPT_TALL_TILES (64 < N <= 256)")
     ap.add_argument("--column-sharded", action="store_true",
                     help="each rank holds its own d columns of ONE matrix of world*d columns: pass 1, an all-gather of the "
                          "statistics records, coefficient step and pass 2 (default for --gpus N > 1: independent replicas)")

@@ -152,11 +152,16 @@ enum adacons_option {
   ADACONS_OPT_TALL_TILES = 11, /* 1 (default): with 64 < N <= 256 on aligned buffers pass 1 reads the
                                   matrix ONCE, as for N <= 64, from taller and narrower tiles:
                                   128 rows x 256 bytes (half a warp per row) up to N = 128,
-                                  256 rows x 128 bytes (a quarter-warp per row) beyond.  0: the
-                                  two-read form (column sums first, then dot products per 64
-                                  rows), which N > 256 always takes unless
+                                  256 rows x 256 bytes on 512 threads beyond.  2: beyond N = 128
+                                  tiles of 256 rows x 128 bytes on 256 threads (a quarter-warp
+                                  per row) instead; slower, because box rows of 128 bytes hold
+                                  the copy engine below the memory's rate, kept for comparison.
+                                  0: the two-read form (column sums first, then dot products per
+                                  64 rows), which N > 256 always takes unless
                                   ADACONS_OPT_CLUSTER_PASS1 says otherwise.  The forms agree to
-                                  fp32 rounding of the column sums.                              */
+                                  fp32 rounding of the column sums.  Errors: EINVAL (other
+                                  values), ENOMEM (the other tile shape needs more partial
+                                  records than the context holds; the setting is left as it was). */
   ADACONS_OPT_CLUSTER_PASS1 = 10 /* 0 (default) / 1: with 64 < N <= 512 on aligned buffers pass 1
                                   reads the matrix ONCE through thread-block clusters of 2, 4 or 8
                                   blocks that share each column tile (64 rows per block) and

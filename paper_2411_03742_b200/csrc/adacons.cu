@@ -108,7 +108,7 @@ struct adacons_ctx {
   const void* tmap_big_for = nullptr;
   // 64 < N <= 256: one read of the matrix, one block per tile of 128 rows x 256 bytes or 256 rows x 128 bytes
   bool tall_available = false;
-  int tall_grid = 0, tall_tiles = 0, tall_stages = 0, tall_lpr = 16;   // lanes per row: 16 (128-row tiles) or 8 (256-row tiles)
+  int tall_grid = 0, tall_tiles = 0, tall_stages = 0;
   size_t tall_smem = 0;
   int tall_tiles_opt = 1;               // ADACONS_OPT_TALL_TILES
   CUtensorMap tmap_tall;
@@ -329,31 +329,44 @@ int plan_big(adacons_ctx* c) {
   return ADACONS_OK;
 }
 
-// 64 < N <= 256 on the aligned path: tiles of 128 rows x 256 bytes (N <= 128) or 256 rows x 128 bytes,
-// one block per tile (pass1_tall_kernel).
-const void* tall_fn(int dtype, int lpr) {
-  if (dtype == ADACONS_F32) return lpr == 16 ? reinterpret_cast<const void*>(&pass1_tall_kernel<0, 16>) : reinterpret_cast<const void*>(&pass1_tall_kernel<0, 8>);
-  return lpr == 16 ? reinterpret_cast<const void*>(&pass1_tall_kernel<1, 16>) : reinterpret_cast<const void*>(&pass1_tall_kernel<1, 8>);
+// 64 < N <= 256 on the aligned path, one block per tile (pass1_tall_kernel): tiles of 128 rows x 256 bytes
+// (N <= 128); beyond, 256 rows x 256 bytes with 512 threads (one block per SM) or, on request
+// (ADACONS_OPT_TALL_TILES = 2), 256 rows x 128 bytes with 256 threads.
+struct TallVariant {
+  const void* kernel;
+  int threads, box_bytes, box_rows;
+  size_t fixed_bytes, stage_bytes;
+};
+template <int DT, int LPR, int TH>
+TallVariant tall_variant_of() {
+  using C = P1H<DT, LPR, TH>;
+  return TallVariant{reinterpret_cast<const void*>(&pass1_tall_kernel<DT, LPR, TH>), TH, C::kBoxRowBytesH, C::kRows,
+                     C::kFixedBytes, C::kStageBytes};
+}
+TallVariant tall_variant(int dtype, int N, int opt) {
+  const bool f32 = dtype == ADACONS_F32;
+  if (N <= 128) return f32 ? tall_variant_of<0, 16, 256>() : tall_variant_of<1, 16, 256>();
+  if (opt == 2) return f32 ? tall_variant_of<0, 8, 256>() : tall_variant_of<1, 8, 256>();
+  return f32 ? tall_variant_of<0, 16, 512>() : tall_variant_of<1, 16, 512>();
 }
 
 int plan_tall(adacons_ctx* c) {
   c->tall_available = false;
   if (c->N <= kMaxFastN || c->N > 256) return ADACONS_OK;
   if ((c->pitch * c->elem_bytes) % 16 != 0 || c->encode == nullptr || c->d > kChunkCols) return ADACONS_OK;
-  c->tall_lpr = c->N <= 128 ? 16 : 8;
-  const int tile_cols = c->tall_lpr * 16 / c->elem_bytes;
+  const TallVariant v = tall_variant(c->dtype, c->N, c->tall_tiles_opt);
+  const int tile_cols = v.box_bytes / c->elem_bytes;
   c->tall_tiles = static_cast<int>((c->d + tile_cols - 1) / tile_cols);
-  const size_t fixed = c->dtype == ADACONS_F32 ? (c->tall_lpr == 16 ? P1H<0, 16>::kFixedBytes : P1H<0, 8>::kFixedBytes)
-                                               : (c->tall_lpr == 16 ? P1H<1, 16>::kFixedBytes : P1H<1, 8>::kFixedBytes);
-  const size_t stage = P1H<0, 16>::kStageBytes;
-  int stages = static_cast<int>((kPass1SmemBudget - fixed - 64) / stage);
+  // 256 threads: two blocks per SM share its shared memory; 512 threads: one block has it all
+  const size_t budget = v.threads == kThreads ? kPass1SmemBudget : 2 * kPass1SmemBudget;
+  int stages = static_cast<int>((budget - v.fixed_bytes - 64) / v.stage_bytes);
   if (stages > 8) stages = 8;
   if (stages < 2) return ADACONS_OK;
-  const size_t smem = stages * stage + fixed + static_cast<size_t>(stages) * 8;
-  const void* k = tall_fn(c->dtype, c->tall_lpr);
+  const size_t smem = stages * v.stage_bytes + v.fixed_bytes + static_cast<size_t>(stages) * 8;
+  const size_t cap = v.threads == kThreads ? kPass1SmemCap : 2 * kPass1SmemCap;
   int per_sm = 0;
-  if (smem > kPass1SmemCap || !set_smem_cap(k, kPass1SmemCap) ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kThreads, smem) != cudaSuccess || per_sm < 1) {
+  if (smem > cap || !set_smem_cap(v.kernel, cap) ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, v.kernel, v.threads, smem) != cudaSuccess || per_sm < 1) {
     cudaGetLastError();
     return ADACONS_OK;
   }
@@ -370,7 +383,8 @@ int encode_map_tall(adacons_ctx* c, const void* grads) {
   if (c->tmap_tall_for == grads) return ADACONS_OK;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->d), static_cast<cuuint64_t>(c->N)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c->pitch) * c->elem_bytes};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(c->tall_lpr * 16 / c->elem_bytes), static_cast<cuuint32_t>(c->tall_lpr == 16 ? 128 : 256)};
+  const TallVariant v = tall_variant(c->dtype, c->N, c->tall_tiles_opt);
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(v.box_bytes / c->elem_bytes), static_cast<cuuint32_t>(v.box_rows)};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = c->encode(&c->tmap_tall,
                                c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
@@ -1010,11 +1024,11 @@ int run_step(adacons_ctx* c, const void* grads, void* out, void* cuda_stream, Ph
     int rc = encode_map_tall(c, grads);
     if (rc != ADACONS_OK) return rc;
     Pass1Params p;
-    p.N = N; p.num_tiles = c->tall_tiles; p.stages = c->tall_stages; p.stage_bytes = P1H<0, 16>::kStageBytes;
+    const TallVariant v = tall_variant(c->dtype, N, c->tall_tiles_opt);
+    p.N = N; p.num_tiles = c->tall_tiles; p.stages = c->tall_stages; p.stage_bytes = static_cast<uint32_t>(v.stage_bytes);
     p.partials = c->partials; p.flags = c->flags;
-    const void* k = tall_fn(c->dtype, c->tall_lpr);
     void* args[2] = {&c->tmap_tall, &p};
-    if (cudaLaunchKernel(k, dim3(c->tall_grid), dim3(kThreads), args, c->tall_smem, st) != cudaSuccess) {
+    if (cudaLaunchKernel(v.kernel, dim3(c->tall_grid), dim3(v.threads), args, c->tall_smem, st) != cudaSuccess) {
       cudaGetLastError();
       return ADACONS_ECUDA;
     }
@@ -1262,7 +1276,18 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       if (value < 0.0 || value > 32.0 || value != static_cast<double>(static_cast<int>(value))) return ADACONS_EINVAL;
       c->gram_fold = static_cast<int>(value);
       return ADACONS_OK;
-    case ADACONS_OPT_TALL_TILES: c->tall_tiles_opt = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_TALL_TILES: {
+      if (value != 0.0 && value != 1.0 && value != 2.0) return ADACONS_EINVAL;
+      const int before = c->tall_tiles_opt;
+      c->tall_tiles_opt = static_cast<int>(value);
+      if (c->tall_tiles_opt != 0 && before != 0 && c->tall_tiles_opt != before && c->N > 128) {   // another tile shape
+        DeviceGuard guard(c->device);
+        if (!guard.ok) return ADACONS_ECUDA;
+        plan_tall(c);
+        if (c->tall_available && c->tall_grid > c->max_partials) { c->tall_tiles_opt = before; plan_tall(c); return ADACONS_ENOMEM; }
+      }
+      return ADACONS_OK;
+    }
     case ADACONS_OPT_ALIGNED_BODY: c->aligned_body = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_ONE_LAUNCH:
       if (value != 0.0 && value != 1.0 && value != 2.0) return ADACONS_EINVAL;

@@ -35,6 +35,7 @@ struct P1 {
   static constexpr int kXchFloats = (WR > 1) ? 2 * kXchOne : 0;
   static constexpr int kRedFloats = kWarps * NR * 2;
   static constexpr int kOuterFloats = 2 * NR * kThreads;        // second-level accumulators, [2][NR][thread]
+  static constexpr int kBlockThreads = kThreads;
 };
 
 struct P1Smem {            // carve-up of the dynamic shared memory of both pass-1 kernels
@@ -170,14 +171,14 @@ constexpr int kFoldTiles = 32;
 template <class C>
 __device__ __forceinline__ void p1_outer_clear(float* outer) {
 #pragma unroll
-  for (int j = 0; j < 2 * C::NR; ++j) outer[j * kThreads + threadIdx.x] = 0.f;
+  for (int j = 0; j < 2 * C::NR; ++j) outer[j * C::kBlockThreads + threadIdx.x] = 0.f;
 }
 template <class C>
 __device__ __forceinline__ void p1_fold(float2 (&pacc)[C::NR], float2 (&qacc)[C::NR], float* outer) {
 #pragma unroll
   for (int j = 0; j < C::NR; ++j) {
-    outer[j * kThreads + threadIdx.x] += pacc[j].x + pacc[j].y;
-    outer[(C::NR + j) * kThreads + threadIdx.x] += qacc[j].x + qacc[j].y;
+    outer[j * C::kBlockThreads + threadIdx.x] += pacc[j].x + pacc[j].y;
+    outer[(C::NR + j) * C::kBlockThreads + threadIdx.x] += qacc[j].x + qacc[j].y;
     pacc[j] = qacc[j] = make_float2(0.f, 0.f);
   }
 }
@@ -449,36 +450,38 @@ pass1_dot_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1DotParams 
 // More rows than pass1_tma_kernel's tallest tile at a fraction of the width, so a stage is still
 // 32 KB: 128 rows x 256 bytes (LPR = 16 lanes per row: a HALF-warp owns a row) or 256 rows x 128
 // bytes (LPR = 8: a quarter-warp; TMA moves 128-byte box rows at 4.6 TB/s at most on this GPU, which
-// is still more than two reads at full speed).  Lane l of warp w belongs to row group
+// is still more than two reads at full speed).  With TH = 512 threads and LPR = 16 a block takes
+// 256 rows x 256 bytes (64 KB per stage, one block per SM).  Lane l of warp w belongs to row group
 // g = (32 / LPR) w + l / LPR and owns the 16-byte column group l % LPR of rows g, g + G, ...,
 // g + 7 G (8 rows, as before; G = 8 * 32 / LPR groups; rows past N are zero-filled by TMA).  The
 // groups' partial column sums are exchanged through shared memory in two steps -- every thread
 // first finishes one column of its share of the groups, in group order, then all read the sums of
 // their own columns -- and the lane reduction at the end stays inside the LPR lanes of a row.
 // Same partial-record layout as pass1_tma_kernel.
-template <int DT, int LPR>
+template <int DT, int LPR, int TH = kThreads>
 struct P1H {
   static constexpr int NR = 8;
+  static constexpr int kBlockThreads = TH;
   static constexpr int VEC = Elem<DT>::kVec;
   static constexpr int NP = VEC / 2;
   static constexpr int kLanesPerRow = LPR;
-  static constexpr int kGroups = kWarps * (32 / LPR), kRows = kGroups * NR;
+  static constexpr int kGroups = (TH / 32) * (32 / LPR), kRows = kGroups * NR;
   static constexpr int kBoxRowBytesH = LPR * 16;
   static constexpr int TILEC = kBoxRowBytesH / Elem<DT>::kBytes;   // columns per tile
-  static constexpr int PARTS = kThreads / TILEC;                   // threads per column in the first exchange step
+  static constexpr int PARTS = TH / TILEC;                         // threads per column in the first exchange step
   static constexpr int kGroupsPerPart = kGroups / PARTS;
-  static constexpr uint32_t kStageBytes = kRows * kBoxRowBytesH;   // 32 KB
+  static constexpr uint32_t kStageBytes = kRows * kBoxRowBytesH;   // 32 KB (64 KB with 512 threads)
   static constexpr int kXchFloats = kGroups * TILEC;
-  static constexpr int kSumFloats = PARTS * TILEC;                 // = kThreads
+  static constexpr int kSumFloats = PARTS * TILEC;                 // = TH
   static constexpr int kRedFloats = kGroups * NR * 2;
-  static constexpr int kOuterFloats = 2 * NR * kThreads;
+  static constexpr int kOuterFloats = 2 * NR * TH;
   static constexpr size_t kFixedBytes = (kXchFloats + kSumFloats + kRedFloats + kOuterFloats) * sizeof(float);
 };
 
-template <int DT, int LPR>
-__global__ void __launch_bounds__(kThreads, 2)
+template <int DT, int LPR, int TH>
+__global__ void __launch_bounds__(TH, TH == kThreads ? 2 : 1)
 pass1_tall_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params prm) {
-  using C = P1H<DT, LPR>;
+  using C = P1H<DT, LPR, TH>;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   __shared__ int s_abort;
   const int N = prm.N;
@@ -565,14 +568,14 @@ pass1_tall_kernel(const __grid_constant__ CUtensorMap tmap, const Pass1Params pr
   float* dst = prm.partials + static_cast<size_t>(blockIdx.x) * 2 * N;
   if (s_abort) {
     if (tid == 0) p1_drain_after_timeout(full, prm.stages, issued, prm.flags);
-    for (int i = tid; i < 2 * N; i += kThreads) dst[i] = 0.f;
+    for (int i = tid; i < 2 * N; i += TH) dst[i] = 0.f;
     return;
   }
   // block partial: both accumulation levels, the lanes of a row by a fixed xor tree; every row has one owner group
   p1_fold<C>(pacc, qacc, outer);
 #pragma unroll
   for (int j = 0; j < C::NR; ++j) {
-    float p = outer[j * kThreads + tid], q = outer[(C::NR + j) * kThreads + tid];
+    float p = outer[j * TH + tid], q = outer[(C::NR + j) * TH + tid];
 #pragma unroll
     for (int o = LPR / 2; o > 0; o >>= 1) {
       p += __shfl_xor_sync(0xffffffffu, p, o);

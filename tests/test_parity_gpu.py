@@ -768,6 +768,14 @@ def test_tall_tiles_many_tiles_per_block(ac, N, dtype):
     run_case(ac, w, 2, beta=0.9, expect_path=7)
 
 
+@pytest.mark.parametrize("N,dtype", [(129, "f32"), (200, "bf16"), (256, "f32"), (256, "bf16")])
+def test_tall_tiles_quarter_warp_variant(ac, N, dtype):
+    """ADACONS_OPT_TALL_TILES = 2: above 128 workers, tiles of 256 rows x 128 bytes on 256 threads (a
+    quarter-warp per row) instead of 256 rows x 256 bytes on 512 threads."""
+    w = wl.Workload(f"tallq{N}", N, 1_500_008, dtype, 2, "student_flip", seed=N + 1)
+    run_case(ac, w, 2, beta=0.9, options={ac.OPT_TALL_TILES: 2}, expect_path=7)
+
+
 @pytest.mark.parametrize("N,dtype", [(128, "f32"), (128, "bf16"), (96, "bf16"), (300, "f32")])
 def test_cluster_pass1_many_tiles_per_cluster(ac, N, dtype):
     """Long enough that every cluster walks many tiles (the double-buffered exchange of the partial
