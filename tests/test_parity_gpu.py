@@ -764,7 +764,7 @@ def test_more_than_64_workers(ac, N, d, dtype, form):
 def test_tall_tiles_many_tiles_per_block(ac, N, dtype):
     """The 128- and 256-row tiles on a vector long enough that every block walks many of them (the folding of
     the first-level sums runs several times) with a ragged last tile and heavy-tailed data."""
-    w = wl.Workload(f"tall{N}", N, 3_000_008 if N <= 128 else 1_500_008, dtype, 2, "student_flip", seed=N)
+    w = wl.Workload(f"tall{N}", N, 1_600_008 if N <= 128 else 800_008, dtype, 2, "student_flip", seed=N)
     run_case(ac, w, 2, beta=0.9, expect_path=7)
 
 
@@ -772,7 +772,7 @@ def test_tall_tiles_many_tiles_per_block(ac, N, dtype):
 def test_tall_tiles_quarter_warp_variant(ac, N, dtype):
     """ADACONS_OPT_TALL_TILES = 2: above 128 workers, tiles of 256 rows x 128 bytes on 256 threads (a
     quarter-warp per row) instead of 256 rows x 256 bytes on 512 threads."""
-    w = wl.Workload(f"tallq{N}", N, 1_500_008, dtype, 2, "student_flip", seed=N + 1)
+    w = wl.Workload(f"tallq{N}", N, 800_008, dtype, 2, "student_flip", seed=N + 1)
     run_case(ac, w, 2, beta=0.9, options={ac.OPT_TALL_TILES: 2}, expect_path=7)
 
 
@@ -780,7 +780,7 @@ def test_tall_tiles_quarter_warp_variant(ac, N, dtype):
 def test_cluster_pass1_many_tiles_per_cluster(ac, N, dtype):
     """Long enough that every cluster walks many tiles (the double-buffered exchange of the partial
     column sums wraps around many times) and the last tile is ragged."""
-    w = wl.Workload(f"cl{N}", N, 2_000_008, dtype, 2, "student_flip", seed=N)
+    w = wl.Workload(f"cl{N}", N, 2_000_008 if N <= 128 else 800_008, dtype, 2, "student_flip", seed=N)
     run_case(ac, w, 2, beta=0.9, options={ac.OPT_CLUSTER_PASS1: 1}, expect_path=6)
 
 
@@ -1267,7 +1267,7 @@ def test_gram_pass1_many_tiles_per_block(ac):
     """A vector long enough that every block walks its ring many times and folds several times (the
     tensor cores round running sums toward zero: without the second accumulation level q would drift
     out of tolerance as the vector grows)."""
-    w = wl.Workload("gram-long", 64, 12_000_008, "bf16", 2, "student_flip", seed=77)
+    w = wl.Workload("gram-long", 64, 6_000_008, "bf16", 2, "student_flip", seed=77)
     run_case(ac, w, 2, options={ac.OPT_GRAM_PASS1: 16}, expect_path=9, allow_swaps=False)
 
 
