@@ -137,6 +137,14 @@ enum adacons_option {
                                   buffers take the generic path, as a pitch that is not a
                                   multiple of 16 bytes always does.  Same results either way to
                                   fp32 accumulation order.                                       */
+  ADACONS_OPT_SHIFTED_LOADS = 14, /* 1 (default): a matrix whose rows start at arbitrary element
+                                  offsets (a row pitch that is not a multiple of 16 bytes, e.g.
+                                  contiguous rows of an odd length) or a result buffer off the
+                                  rows' alignment is still read with 16-byte loads, each row's
+                                  bytes shifted into place in registers; the first and last
+                                  16 to 31 bytes of the vector are done element by element.
+                                  0: such buffers take the scalar kernels.  Same results to
+                                  fp32 accumulation order (pass 2: the same bytes).             */
   ADACONS_OPT_GRAM_PASS1 = 13,  /* bf16, N <= 64, aligned buffers, d <= 2^30.  n >= 1: pass 1 takes
                                   the statistics from the Gram matrix of every column tile,
                                   computed on the tensor cores (Eq. 7, third line: N p_i is the
@@ -208,7 +216,9 @@ enum adacons_info {
                                         the row pitch 32-byte aligned), 4 = the second phase of
                                         the one-launch kernel (TMA-staged chunks of 8 rows),
                                         5 = vector kernel on the aligned body plus element-wise
-                                        edges (grads and out off a 16-byte boundary alike)       */
+                                        edges (grads and out off a 16-byte boundary alike),
+                                        6 = 16-byte loads shifted into place per row
+                                        (see ADACONS_OPT_SHIFTED_LOADS)                          */
   ADACONS_INFO_STATS_DOUBLES = 8     /* doubles in one shard's statistics (adacons_pass1):
                                         sets * (2 N + 1)                                         */
 };

@@ -19,7 +19,7 @@ F32, BF16 = 0, 1
 # enum adacons_option
 (OPT_BETA, OPT_MOMENTUM, OPT_SORTED, OPT_NORMALIZE, OPT_PER_SEGMENT, OPT_PROFILE, OPT_OVERLAP_LAUNCH,
  OPT_FUSED_SMALL, OPT_ROW_PITCH, OPT_ONE_LAUNCH, OPT_CLUSTER_PASS1, OPT_TALL_TILES, OPT_ALIGNED_BODY,
- OPT_GRAM_PASS1) = range(14)
+ OPT_GRAM_PASS1, OPT_SHIFTED_LOADS) = range(15)
 # enum adacons_coeff
 COEFF_A, COEFF_A_TILDE, COEFF_GAMMA, COEFF_P, COEFF_Q = range(5)
 # enum adacons_info

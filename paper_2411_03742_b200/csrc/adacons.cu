@@ -118,6 +118,7 @@ struct adacons_ctx {
   int cl_size = 0, cl_grid = 0, cl_tiles = 0;
   size_t cl_smem = 0;
   int cluster_pass1 = 0;                // ADACONS_OPT_CLUSTER_PASS1 (opt-in)
+  int shifted_loads = 1;                // ADACONS_OPT_SHIFTED_LOADS
   // bf16, N <= 64: pass 1 from the Gram matrix on the tensor cores (pass1_gram_kernel)
   bool gram_available = false;
   int gram_grid = 0, gram_tiles = 0, gram_stages = 2;
@@ -1169,6 +1170,27 @@ int run_step(adacons_ctx* c, const void* grads, void* out, void* cuda_stream, Ph
       extra_launches += (nv > 0) ? 1 : 0;
     }
     c->last_pass2 = 5;
+  } else if (!seg && c->shifted_loads && g0 % c->elem_bytes == 0 && o0 % c->elem_bytes == 0 && c->d >= 4 * (16 / c->elem_bytes)) {
+    // rows (or out) at any element offset: 16-byte groups of out, each row's bytes realigned in registers
+    const int vec = 16 / c->elem_bytes;
+    const int head = static_cast<int>(((16 - o0 % 16) % 16) / c->elem_bytes) + vec;        // vec .. 2 vec - 1 columns
+    const long long groups = (c->d - 2 * vec - head) / vec + 1;                             // >= 1; the last one ends 2 vec columns before d at the latest
+    const int tail = static_cast<int>(c->d - head - groups * vec);                          // vec .. 2 vec - 1 columns
+    const unsigned char* g8 = static_cast<const unsigned char*>(grads);
+    unsigned char* o8 = static_cast<unsigned char*>(out) + static_cast<size_t>(head) * c->elem_bytes;
+    const long long body_off = static_cast<long long>(head) * c->elem_bytes;
+    const unsigned blocks = static_cast<unsigned>((groups + kThreads - 1) / kThreads);
+    if (c->dtype == ADACONS_F32)
+      e2 = launch_kernel(pass2_shift_kernel<0>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, body_off, groups);
+    else
+      e2 = launch_kernel(pass2_shift_kernel<1>, dim3(blocks), dim3(kThreads), 0, st, false, g8, o8, c->gamma_f32, N, row_bytes, body_off, groups);
+    if (e2 == cudaSuccess) {
+      if (c->dtype == ADACONS_F32) edge_combine_kernel<0><<<1, 32, 0, st>>>(grads, out, c->gamma_f32, N, c->d, c->pitch, head, tail);
+      else edge_combine_kernel<1><<<1, 32, 0, st>>>(grads, out, c->gamma_f32, N, c->d, c->pitch, head, tail);
+      e2 = cudaGetLastError();
+      extra_launches += 1;
+    }
+    c->last_pass2 = 6;
   } else {
     const unsigned blocks = static_cast<unsigned>((c->d + kThreads - 1) / kThreads);
     if (c->dtype == ADACONS_F32)
@@ -1289,6 +1311,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       return ADACONS_OK;
     }
     case ADACONS_OPT_ALIGNED_BODY: c->aligned_body = value != 0.0; return ADACONS_OK;
+    case ADACONS_OPT_SHIFTED_LOADS: c->shifted_loads = value != 0.0; return ADACONS_OK;
     case ADACONS_OPT_ONE_LAUNCH:
       if (value != 0.0 && value != 1.0 && value != 2.0) return ADACONS_EINVAL;
       c->one_launch = static_cast<int>(value); return ADACONS_OK;
@@ -1370,6 +1393,7 @@ int adacons_get_option(adacons_ctx* c, int key, double* value) {
     case ADACONS_OPT_ONE_LAUNCH: *value = c->one_launch; return ADACONS_OK;
     case ADACONS_OPT_TALL_TILES: *value = c->tall_tiles_opt; return ADACONS_OK;
     case ADACONS_OPT_ALIGNED_BODY: *value = c->aligned_body; return ADACONS_OK;
+    case ADACONS_OPT_SHIFTED_LOADS: *value = c->shifted_loads; return ADACONS_OK;
     case ADACONS_OPT_CLUSTER_PASS1: *value = c->cluster_pass1; return ADACONS_OK;
     case ADACONS_OPT_GRAM_PASS1: *value = c->gram_fold; return ADACONS_OK;
     case ADACONS_OPT_ROW_PITCH: *value = static_cast<double>(c->pitch); return ADACONS_OK;

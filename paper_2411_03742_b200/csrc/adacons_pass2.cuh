@@ -542,12 +542,86 @@ pass2_generic_kernel(const void* __restrict__ grads, void* __restrict__ out, con
 }
 
 // ----------------------------------------------------------------------------------------------
+// Pass 2 for rows that start anywhere (a row pitch that is not a multiple of 16 bytes, or `out` off
+// a 16-byte boundary by another amount than the rows): vector loads all the same.  The body of the
+// vector is cut into 16-byte groups of OUT (so the stores are aligned); the 16 bytes of row i that
+// belong to a group start `shift_i` bytes into an aligned 16-byte group of the matrix, the same
+// shift for every group of the row.  A thread loads that aligned group and the next one and
+// extracts its bytes with funnel shifts; which words it takes depends on the row alone, so the
+// choice is a branch the whole grid takes alike.  The second load is the first load of the
+// neighbouring thread (an L1 hit).  Rows are added in index order with the rounding of the other
+// pass-2 kernels, so the bytes agree with theirs.  The body leaves out the first 16 to 31 bytes and
+// the last 16 to 31 bytes of the vector (edge_combine_kernel), so no load leaves a row.
+// ----------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {   // read-only path, L1 allocation allowed
+  uint4 v;
+  asm("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+// bytes [shift, shift + 16) of the 32 bytes lo:hi; shift is a multiple of 2
+__device__ __forceinline__ uint4 realign_16(const uint4& lo, const uint4& hi, const int shift) {
+  const uint32_t r = static_cast<uint32_t>(shift & 3) * 8u;
+  switch (shift >> 2) {
+    case 0: return make_uint4(__funnelshift_r(lo.x, lo.y, r), __funnelshift_r(lo.y, lo.z, r), __funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r));
+    case 1: return make_uint4(__funnelshift_r(lo.y, lo.z, r), __funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r));
+    case 2: return make_uint4(__funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r), __funnelshift_r(hi.y, hi.z, r));
+    default: return make_uint4(__funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r), __funnelshift_r(hi.y, hi.z, r), __funnelshift_r(hi.z, hi.w, r));
+  }
+}
+
+constexpr int kPass2ShiftRows = 4;   // rows per batch: 2 * kPass2ShiftRows 16-byte loads in flight per thread
+
+// grads: byte address of element (0, 0); body_off: byte offset of the body's first column within a row;
+// out_body: the (16-byte aligned) address of that column in the result; num_groups 16-byte groups follow.
+template <int DT>
+__global__ void __launch_bounds__(kThreads)
+pass2_shift_kernel(const unsigned char* __restrict__ grads, unsigned char* __restrict__ out_body, const float* __restrict__ gamma,
+                   int N, long long row_bytes, long long body_off, long long num_groups) {
+  constexpr int NP = Elem<DT>::kVec / 2;
+  constexpr int U = kPass2ShiftRows;
+  __shared__ float g_s[kMaxN];
+  __shared__ unsigned char shift_s[kMaxN];
+  pdl_wait();
+  for (int i = threadIdx.x; i < N; i += kThreads) {
+    g_s[i] = gamma[i];
+    shift_s[i] = static_cast<unsigned char>((reinterpret_cast<unsigned long long>(grads) + static_cast<unsigned long long>(i) * row_bytes + body_off) & 15ull);
+  }
+  __syncthreads();
+  const long long j = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+  if (j >= num_groups) return;
+  const unsigned char* col = grads + body_off + j * 16;
+  float2 acc[NP];
+#pragma unroll
+  for (int h = 0; h < NP; ++h) acc[h] = make_float2(0.f, 0.f);
+  for (int i0 = 0; i0 < N; i0 += U) {
+    uint4 lo[U], hi[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u < N ? i0 + u : N - 1;     // rows past the end repeat the last one and get weight 0
+      const unsigned char* a = col + static_cast<long long>(i) * row_bytes - shift_s[i];
+      lo[u] = ld_nc_v4(a);
+      hi[u] = ld_nc_v4(a + 16);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u < N ? i0 + u : N - 1;
+      const float g = i0 + u < N ? g_s[i] : 0.f;
+      const uint4 x = realign_16(lo[u], hi[u], shift_s[i]);
+      const float2 g2 = make_float2(g, g);
+#pragma unroll
+      for (int h = 0; h < NP; ++h) acc[h] = __ffma2_rn(unpack_pair<DT>(x, h), g2, acc[h]);
+    }
+  }
+  pass2_store<DT, NP>(out_body, j, acc);
+}
+
+// ----------------------------------------------------------------------------------------------
 // Edges of a matrix whose rows start off a 16-byte boundary (every row by the same amount: the row
 // pitch is a multiple of 16 bytes).  The vectorised kernels then run on the aligned body -- from
 // each row's first 16-byte boundary on -- and these two one-block kernels do the few columns left:
 // edge_stats_kernel adds the first `head` (< 8) columns' share of Eq. 7 as one more partial record,
-// edge_combine_kernel forms Eq. 12 for the head columns and for the last `tail` (< 8) columns that
-// do not fill a 16-byte group (element-wise, so nothing is read or written past the vector).
+// edge_combine_kernel forms Eq. 12 for the first `head` and the last `tail` columns (32 in all at
+// most; element-wise, so nothing is read or written past the vector).
 // ----------------------------------------------------------------------------------------------
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
@@ -582,10 +656,10 @@ template <int DT>
 __global__ void __launch_bounds__(32)
 edge_combine_kernel(const void* __restrict__ grads, void* __restrict__ out, const float* __restrict__ gamma, int N,
                     long long d, long long pitch, int head, int tail) {
-  __shared__ float g_s[kMaxFastN];
+  __shared__ float g_s[kMaxN];
   for (int i = threadIdx.x; i < N; i += 32) g_s[i] = gamma[i];
   __syncthreads();
-  const int k = threadIdx.x;
+  const int k = threadIdx.x;                       // head + tail <= 32
   if (k >= head + tail) return;
   const long long col = k < head ? k : d - tail + (k - head);
   float acc = 0.f;

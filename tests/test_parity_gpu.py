@@ -144,9 +144,9 @@ def test_one_launch_default_by_size_and_alignment(ac):
     h.aggregate(G, out[4:w.d + 4])                     # out is 16 but not 32 bytes aligned: still one launch
     torch.cuda.synchronize()
     assert h.info(ac.INFO_LAST_PATH) == 5
-    h.aggregate(G, out[1:w.d + 1])                     # out is not 16 bytes aligned: fast pass 1, generic pass 2
+    h.aggregate(G, out[1:w.d + 1])                     # out is not 16 bytes aligned: fast pass 1, pass 2 with shifted loads
     torch.cuda.synchronize()
-    assert h.info(ac.INFO_LAST_PATH) == 1 and h.info(ac.INFO_LAST_PASS2) == 1
+    assert h.info(ac.INFO_LAST_PATH) == 1 and h.info(ac.INFO_LAST_PASS2) == 6
     h.set_option(ac.OPT_ONE_LAUNCH, 0)
     h.aggregate(G, out[:w.d])
     torch.cuda.synchronize()
@@ -282,7 +282,7 @@ def test_single_column_has_tied_coefficients(ac):
 def test_misaligned_base_pointer(ac, aligned_body):
     """A matrix that starts 4 bytes off a 16-byte boundary with a 16-byte pitch: pass 1 runs on the
     aligned body plus the head columns (path 8), or on the generic kernels when that is switched off;
-    `out` is aligned here, i.e. off by another amount than the matrix, so pass 2 is the generic one."""
+    `out` is aligned here, i.e. off by another amount than the matrix, so pass 2 shifts its loads into place."""
     N, d = 6, 4096
     w = wl.Workload("mis", N, d, "f32", 1, "gauss", seed=3)
     G0 = wl.generate(w, 0, "cuda:0")
@@ -295,7 +295,7 @@ def test_misaligned_base_pointer(ac, aligned_body):
     h.set_option(ac.OPT_ALIGNED_BODY, aligned_body)
     h.aggregate(G, out)
     torch.cuda.synchronize()
-    assert h.info(ac.INFO_LAST_PATH) == (8 if aligned_body else 2) and h.info(ac.INFO_LAST_PASS2) == 1
+    assert h.info(ac.INFO_LAST_PATH) == (8 if aligned_body else 2) and h.info(ac.INFO_LAST_PASS2) == 6
     res = oc.AdaConsOracle(N, d).step(to_f64(G0), storage="f32")
     assert_coeffs(h.coeffs(ac.COEFF_GAMMA), res["gamma"], "gamma")
     assert_output(out, res, to_f64(G0), "f32", "misaligned")
@@ -367,7 +367,7 @@ def test_aligned_body_of_offset_buffers(ac, dtype, N, d, g_off, o_off):
         torch.cuda.synchronize()
         head = (16 - (g_off * eb) % 16) // eb
         assert h.info(ac.INFO_LAST_PATH) == (8 if d > head else 2), h.info(ac.INFO_LAST_PATH)
-        assert h.info(ac.INFO_LAST_PASS2) == (5 if same and d > head else 1)
+        assert h.info(ac.INFO_LAST_PASS2) == (5 if same and d > head else 6 if d >= 4 * (16 // eb) else 1)
         G64 = to_f64(G0)
         res = oracle_step(orc, G64, dtype, h.coeffs(ac.COEFF_A), what=w.name)
         for k, code in (("p", ac.COEFF_P), ("q", ac.COEFF_Q), ("a", ac.COEFF_A), ("gamma", ac.COEFF_GAMMA)):
@@ -1284,3 +1284,50 @@ def test_gram_pass1_option_is_validated_and_ignored_where_it_does_not_apply(ac):
     torch.cuda.synchronize()
     assert h.info(ac.INFO_LAST_PATH) == 1          # fp32 storage: the ordinary kernel
     h.close()
+
+
+# ---- rows at arbitrary element offsets: 16-byte loads shifted into place ---------------------------
+SHIFTED_CASES = [("f32", 8, 100_003, 0, 0), ("f32", 5, 70_001, 1, 2), ("f32", 16, 50_002, 3, 0), ("bf16", 16, 90_001, 0, 0),
+                 ("bf16", 7, 65_539, 1, 5), ("bf16", 64, 40_007, 3, 3), ("bf16", 3, 33, 1, 0), ("f32", 3, 16, 0, 1),
+                 ("bf16", 100, 30_011, 2, 7), ("f32", 130, 20_001, 1, 1)]
+
+
+@pytest.mark.parametrize("dtype,N,d,g_off,o_off", SHIFTED_CASES)
+def test_rows_at_arbitrary_offsets(ac, dtype, N, d, g_off, o_off):
+    """Contiguous rows whose length is not a multiple of 16 bytes: every row starts at another offset
+    from a 16-byte boundary, and so may the result.  The vector kernels shift each row's bytes into
+    place; the scalar kernels (option off) must give the same output bytes.  NaN all around the
+    matrix and sentinels around the result: nothing outside is used or touched."""
+    dev = torch.device("cuda:0")
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    eb = 4 if dtype == "f32" else 2
+    w = wl.Workload(f"shift{N}x{d}", N, d, dtype, 3, "gauss_outlier", seed=7 * g_off + o_off + N)
+    gbuf = torch.full((N * d + 64,), float("nan"), dtype=tdt, device=dev)
+    G = gbuf[g_off:g_off + N * d].view(N, d)
+    obufs = [torch.full((d + 64,), 7.0, dtype=tdt, device=dev) for _ in range(2)]
+    outs = [b[o_off:o_off + d] for b in obufs]
+    hs = [ac.AdaCons(N, d, dtype) for _ in range(2)]
+    hs[1].set_option(ac.OPT_SHIFTED_LOADS, 0)
+    for h in hs:
+        h.set_option(ac.OPT_BETA, 0.8)
+    orc = oc.AdaConsOracle(N, d, beta=0.8)
+    for t in range(3):
+        G0 = wl.generate(w, t, dev)
+        G.copy_(G0)
+        for h, o in zip(hs, outs):
+            h.aggregate(G, o)
+        torch.cuda.synchronize()
+        assert hs[0].info(ac.INFO_LAST_PASS2) == (6 if d >= 4 * (16 // eb) else 1) and hs[1].info(ac.INFO_LAST_PASS2) == 1
+        G64 = to_f64(G0)
+        res = oracle_step(orc, G64, dtype, hs[0].coeffs(ac.COEFF_A), what=w.name)
+        for k, code in (("p", ac.COEFF_P), ("q", ac.COEFF_Q), ("a", ac.COEFF_A), ("gamma", ac.COEFF_GAMMA)):
+            assert_coeffs(hs[0].coeffs(code)[0], res[k][0], f"{w.name} {k} step {t}")
+        assert_coeffs(hs[0].state()[0][0], res["m"][0], f"{w.name} m step {t}")
+        assert_output(outs[0], res, G64, dtype, f"{w.name} step {t}")
+        assert torch.equal(outs[0].view(torch.uint8), outs[1].view(torch.uint8))
+        for b in obufs:
+            assert bool((b[:o_off] == 7.0).all()) and bool((b[o_off + d:] == 7.0).all())
+        assert bool(torch.isnan(gbuf[:g_off]).all()) and bool(torch.isnan(gbuf[g_off + N * d:]).all())
+        assert hs[0].status() == 0
+    for h in hs:
+        h.close()
