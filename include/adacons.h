@@ -140,11 +140,14 @@ enum adacons_option {
   ADACONS_OPT_SHIFTED_LOADS = 14, /* 1 (default): a matrix whose rows start at arbitrary element
                                   offsets (a row pitch that is not a multiple of 16 bytes, e.g.
                                   contiguous rows of an odd length) or a result buffer off the
-                                  rows' alignment is still read with 16-byte loads, each row's
-                                  bytes shifted into place in registers; the first and last
-                                  16 to 31 bytes of the vector are done element by element.
-                                  0: such buffers take the scalar kernels.  Same results to
-                                  fp32 accumulation order (pass 2: the same bytes).             */
+                                  rows' alignment is still moved 16 bytes at a time (pass 1,
+                                  N <= 64: the staged kernel with one tensor map per class of
+                                  rows that share an offset, taken for bf16 always and for fp32
+                                  when a class has 4 rows or more; pass 2: 16-byte loads), each
+                                  row's bytes shifted into place in registers; the first and
+                                  last 16 to 31 bytes of the vector are done element by element.  0: such buffers take the scalar
+                                  kernels.  Same results to fp32 accumulation order (pass 2
+                                  given the same weights: the same bytes).                      */
   ADACONS_OPT_GRAM_PASS1 = 13,  /* bf16, N <= 64, aligned buffers, d <= 2^30.  n >= 1: pass 1 takes
                                   the statistics from the Gram matrix of every column tile,
                                   computed on the tensor cores (Eq. 7, third line: N p_i is the
@@ -208,7 +211,10 @@ enum adacons_info {
                                         8 = misaligned base, aligned body: TMA-staged pass 1 plus
                                             the head columns (see ADACONS_OPT_ALIGNED_BODY),
                                         9 = pass 1 from the Gram matrix on the tensor cores
-                                            (see ADACONS_OPT_GRAM_PASS1)                         */
+                                            (see ADACONS_OPT_GRAM_PASS1),
+                                        10 = rows at arbitrary element offsets: staged pass 1 with
+                                            a tensor map per class of equally offset rows
+                                            (see ADACONS_OPT_SHIFTED_LOADS)                       */
   ADACONS_INFO_TOTAL_LAUNCHES = 6,   /* kernels launched by this context so far                  */
   ADACONS_INFO_LAST_PASS2 = 7,       /* pass-2 kernel of the most recent aggregate call: 0 = none
                                         (no call yet, or the single-pass kernel), 1 = generic,

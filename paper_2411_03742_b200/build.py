@@ -17,7 +17,7 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libadacons_b200.so")
 SOURCES = ["adacons.cu"]
 DEPS = ["adacons.cu", "adacons_kernels.cuh", "adacons_common.cuh", "adacons_pass1.cuh", "adacons_coeff.cuh",
-        "adacons_pass2.cuh", "adacons_fused.cuh", "adacons_gram.cuh"]
+        "adacons_pass2.cuh", "adacons_fused.cuh", "adacons_gram.cuh", "adacons_shift.cuh"]
 
 
 def _nvcc() -> str:

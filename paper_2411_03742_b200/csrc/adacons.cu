@@ -119,6 +119,12 @@ struct adacons_ctx {
   size_t cl_smem = 0;
   int cluster_pass1 = 0;                // ADACONS_OPT_CLUSTER_PASS1 (opt-in)
   int shifted_loads = 1;                // ADACONS_OPT_SHIFTED_LOADS
+  Pass1Plan shift;                      // pass1_shift_kernel: rows at arbitrary element offsets (N <= 64)
+  long long shift_body_cols = 0;
+  int shift_head = 0, shift_tail = 0;
+  ShiftMaps shift_maps;                 // one tensor map per row class, for the matrix at shift_maps_for
+  const void* shift_maps_for = nullptr;
+  int shift_classes = 1, shift_class_base[kShiftMaxClasses] = {0}, shift_class_shift[kShiftMaxClasses] = {0};
   // bf16, N <= 64: pass 1 from the Gram matrix on the tensor cores (pass1_gram_kernel)
   bool gram_available = false;
   int gram_grid = 0, gram_tiles = 0, gram_stages = 2;
@@ -193,6 +199,25 @@ const void* select_pass1(int dtype, int NR, int WR) {
   if (WR == 2) return pass1_fn<DT, 8, 2>();                  \
   if (WR == 4) return pass1_fn<DT, 8, 4>();                  \
   return pass1_fn<DT, 8, 8>();
+  if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
+  ADACONS_PICK(1)
+#undef ADACONS_PICK
+}
+
+template <int DT, int NR, int WR>
+const void* pass1_shift_fn() { return reinterpret_cast<const void*>(&pass1_shift_kernel<DT, NR, WR>); }
+
+const void* select_pass1_shift(int dtype, int NR, int WR) {
+#define ADACONS_PICK(DT)                                     \
+  if (WR == 1) {                                             \
+    if (NR == 1) return pass1_shift_fn<DT, 1, 1>();          \
+    if (NR == 2) return pass1_shift_fn<DT, 2, 1>();          \
+    if (NR == 4) return pass1_shift_fn<DT, 4, 1>();          \
+    return pass1_shift_fn<DT, 8, 1>();                       \
+  }                                                          \
+  if (WR == 2) return pass1_shift_fn<DT, 8, 2>();            \
+  if (WR == 4) return pass1_shift_fn<DT, 8, 4>();            \
+  return pass1_shift_fn<DT, 8, 8>();
   if (dtype == ADACONS_F32) { ADACONS_PICK(0) }
   ADACONS_PICK(1)
 #undef ADACONS_PICK
@@ -291,6 +316,91 @@ int plan_fast(adacons_ctx* c) {
   f.grid = per_sm * c->num_sms;
   if (f.grid > f.num_tiles) f.grid = f.num_tiles;
   f.available = true;
+  return ADACONS_OK;
+}
+
+// N <= 64, rows at arbitrary element offsets (any pitch): one tensor map per class of rows that share an
+// offset from a 16-byte boundary (pass1_shift_kernel).  The body is the whole 16-byte column groups
+// between one vector width of head columns and one to two vector widths of tail columns.
+int plan_shift(adacons_ctx* c) {
+  Pass1Plan& f = c->shift;
+  f.available = false;
+  c->shift_maps_for = nullptr;
+  const int N = c->N;
+  const int vec = 16 / c->elem_bytes;
+  if (N > kMaxFastN || c->d < 4 * vec || c->d > kChunkCols || c->encode == nullptr) return ADACONS_OK;
+  // A tensor copy costs the copy engine a fixed 30 ns or so besides its bytes, so the k classes must not be too
+  // thin: with 4 KB per copy (8 rows) the kernel reads at 4.4-5.0 TB/s, with 1 KB at 2.3-2.6 TB/s.  The scalar
+  // kernel does 2.6-3.4 TB/s on fp32 and 1.2-1.5 TB/s on bf16, hence: bf16 always, fp32 from 4 rows per class on.
+  {
+    const unsigned rem = static_cast<unsigned>((static_cast<unsigned long long>(c->pitch) * c->elem_bytes) % 16);
+    const int k = rem == 0 ? 1 : static_cast<int>(16u / (rem & (~rem + 1u)));
+    if (c->dtype == ADACONS_F32 && N < 4 * k) return ADACONS_OK;
+  }
+  c->shift_head = vec;
+  c->shift_body_cols = (c->d - 2 * vec) / vec * vec;
+  c->shift_tail = static_cast<int>(c->d - vec - c->shift_body_cols);
+  int WR, NR;
+  if (N <= 8) { WR = 1; NR = N <= 1 ? 1 : N <= 2 ? 2 : N <= 4 ? 4 : 8; }
+  else if (N <= 16) { WR = 2; NR = 8; }
+  else if (N <= 32) { WR = 4; NR = 8; }
+  else { WR = 8; NR = 8; }
+  const int WC = kWarps / WR;
+  f.NR = NR; f.WR = WR;
+  f.tile_cols = WC * kShiftGroups * vec;
+  f.num_tiles = static_cast<int>((c->shift_body_cols + f.tile_cols - 1) / f.tile_cols);
+  f.stage_bytes = static_cast<uint32_t>(WC) * N * kBoxRowBytes;
+  const size_t xch = WR > 1 ? static_cast<size_t>(2) * WR * WC * 32 * vec * sizeof(float) : 0;
+  const size_t fixed = xch + static_cast<size_t>(kWarps) * NR * 2 * sizeof(float) + static_cast<size_t>(2) * NR * kThreads * sizeof(float);
+  int stages = static_cast<int>((kPass1SmemBudget - fixed - 64) / f.stage_bytes);
+  if (stages > 8) stages = 8;
+  if (stages < 2) stages = 2;
+  f.stages = stages;
+  f.smem_bytes = static_cast<size_t>(stages) * f.stage_bytes + fixed + static_cast<size_t>(stages) * 8;
+  f.kernel = select_pass1_shift(c->dtype, NR, WR);
+  int per_sm = 0;
+  if (f.smem_bytes > kPass1SmemCap || !set_smem_cap(f.kernel, kPass1SmemCap) ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, f.kernel, kThreads, f.smem_bytes) != cudaSuccess || per_sm < 1) {
+    cudaGetLastError();
+    return ADACONS_OK;
+  }
+  f.grid = per_sm * c->num_sms;
+  if (f.grid > f.num_tiles) f.grid = f.num_tiles;
+  f.available = true;
+  return ADACONS_OK;
+}
+
+// The tensor maps of pass1_shift_kernel for a matrix at `grads`: rows c, c + k, c + 2k, ... (k = 16 / gcd(pitch in
+// bytes, 16)) start at the same offset from a 16-byte boundary and are k * pitch apart, a legal stride.
+int encode_shift_maps(adacons_ctx* c, const void* grads) {
+  if (c->shift_maps_for == grads) return ADACONS_OK;
+  const unsigned long long g0 = reinterpret_cast<unsigned long long>(grads);
+  const unsigned long long row_bytes = static_cast<unsigned long long>(c->pitch) * c->elem_bytes;
+  const unsigned rem = static_cast<unsigned>(row_bytes % 16);
+  int k = 1;
+  if (rem != 0) k = static_cast<int>(16u / (rem & (~rem + 1u)));      // gcd(rem, 16) is rem's lowest set bit
+  c->shift_classes = k;
+  int base_slot = 0;
+  for (int cl = 0; cl < k; ++cl) {
+    const int rows = cl < c->N ? (c->N - cl + k - 1) / k : 0;
+    c->shift_class_base[cl] = base_slot;
+    base_slot += rows;
+    c->shift_class_shift[cl] = 0;
+    if (rows == 0) continue;
+    const unsigned long long a = g0 + static_cast<unsigned long long>(cl) * row_bytes + static_cast<unsigned long long>(c->shift_head) * c->elem_bytes;
+    const unsigned shift = static_cast<unsigned>(a % 16);
+    c->shift_class_shift[cl] = static_cast<int>(shift);
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c->shift_body_cols) + shift / c->elem_bytes, static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(k) * row_bytes};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBoxRowBytes / c->elem_bytes), static_cast<cuuint32_t>(rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = c->encode(&c->shift_maps.m[cl],
+                                 c->dtype == ADACONS_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                 2, reinterpret_cast<void*>(a - shift), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return ADACONS_ECUDA;
+  }
+  c->shift_maps_for = grads;
   return ADACONS_OK;
 }
 
@@ -811,6 +921,8 @@ int adacons_create(adacons_ctx** out, int N, int64_t d, int dtype, const int64_t
   if (c->cl_available && c->cl_grid / c->cl_size > c->max_partials) c->max_partials = c->cl_grid / c->cl_size;
   plan_gram(c);
   if (c->gram_available && c->gram_grid > c->max_partials) c->max_partials = c->gram_grid;
+  plan_shift(c);
+  if (c->shift.available && c->shift.grid > c->max_partials) c->max_partials = c->shift.grid;
   plan_tall(c);
   if (c->tall_available && c->tall_grid > c->max_partials) c->max_partials = c->tall_grid;
 
@@ -1015,8 +1127,8 @@ int run_step(adacons_ctx* c, const void* grads, void* out, void* cuda_stream, Ph
       return ADACONS_ECUDA;
     }
     float* rec = c->partials + static_cast<size_t>(c->fast.grid) * 2 * N;
-    if (c->dtype == ADACONS_F32) edge_stats_kernel<0><<<1, kThreads, 0, st>>>(grads, N, c->pitch, head, rec);
-    else edge_stats_kernel<1><<<1, kThreads, 0, st>>>(grads, N, c->pitch, head, rec);
+    if (c->dtype == ADACONS_F32) edge_stats_kernel<0><<<1, kThreads, 0, st>>>(grads, N, c->d, c->pitch, head, 0, rec);
+    else edge_stats_kernel<1><<<1, kThreads, 0, st>>>(grads, N, c->d, c->pitch, head, 0, rec);
     if (!launch_ok()) return ADACONS_ECUDA;
     extra_launches += 1;
     num_partials = c->fast.grid + 1;
@@ -1076,6 +1188,28 @@ int run_step(adacons_ctx* c, const void* grads, void* out, void* cuda_stream, Ph
     }
     num_partials = c->big_grid;
     c->last_path = 4;
+  } else if (c->shifted_loads && c->shift.available && g0 % c->elem_bytes == 0) {
+    // rows at arbitrary element offsets: a tensor map per class of equally offset rows, shifted into place in
+    // registers; head and tail columns as one more record
+    int rc = encode_shift_maps(c, grads);
+    if (rc != ADACONS_OK) return rc;
+    Pass1ShiftParams p;
+    p.N = N; p.num_tiles = c->shift.num_tiles; p.stages = c->shift.stages; p.stage_bytes = c->shift.stage_bytes;
+    p.classes = c->shift_classes;
+    for (int cl = 0; cl < kShiftMaxClasses; ++cl) { p.class_base[cl] = c->shift_class_base[cl]; p.class_shift[cl] = c->shift_class_shift[cl]; }
+    p.partials = c->partials; p.flags = c->flags;
+    void* args[2] = {&c->shift_maps, &p};
+    if (cudaLaunchKernel(c->shift.kernel, dim3(c->shift.grid), dim3(kThreads), args, c->shift.smem_bytes, st) != cudaSuccess) {
+      cudaGetLastError();
+      return ADACONS_ECUDA;
+    }
+    float* rec = c->partials + static_cast<size_t>(c->shift.grid) * 2 * N;
+    if (c->dtype == ADACONS_F32) edge_stats_kernel<0><<<1, kThreads, 0, st>>>(grads, N, c->d, c->pitch, c->shift_head, c->shift_tail, rec);
+    else edge_stats_kernel<1><<<1, kThreads, 0, st>>>(grads, N, c->d, c->pitch, c->shift_head, c->shift_tail, rec);
+    if (!launch_ok()) return ADACONS_ECUDA;
+    extra_launches += 1;
+    num_partials = c->shift.grid + 1;
+    c->last_path = 10;
   } else {
     if (c->dtype == ADACONS_F32)
       pass1_generic_kernel<0><<<c->generic_grid, kThreads, c->generic_smem, st>>>(grads, N, c->d, c->pitch, c->generic_tiles, c->partials);
@@ -1340,6 +1474,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       plan_cluster(c);
       plan_tall(c);
       plan_gram(c);
+      plan_shift(c);
       int need = c->generic_grid;
       if (c->fast.available && c->fast.grid * c->num_chunks > need) need = c->fast.grid * c->num_chunks;
       if (c->fused_available && c->fused_grid > need) need = c->fused_grid;
@@ -1347,6 +1482,7 @@ int adacons_set_option(adacons_ctx* c, int key, double value) {
       if (c->cl_available && c->cl_grid / c->cl_size > need) need = c->cl_grid / c->cl_size;
       if (c->tall_available && c->tall_grid > need) need = c->tall_grid;
       if (c->gram_available && c->gram_grid > need) need = c->gram_grid;
+      if (c->shift.available && c->shift.grid > need) need = c->shift.grid;
       need += 1;                             // the head columns' record (aligned-body path)
       if (need > c->max_partials) {          // the other paths may use more blocks than the old plan
         cudaFree(c->partials);

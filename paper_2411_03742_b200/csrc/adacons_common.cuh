@@ -102,6 +102,22 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint4& a, const uint
                  ::"l"(p), "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w) : "memory");
 }
 
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {   // read-only path, L1 allocation allowed
+  uint4 v;
+  asm("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+// bytes [shift, shift + 16) of the 32 bytes lo:hi; shift is a multiple of 2
+__device__ __forceinline__ uint4 realign_16(const uint4& lo, const uint4& hi, const int shift) {
+  const uint32_t r = static_cast<uint32_t>(shift & 3) * 8u;
+  switch (shift >> 2) {
+    case 0: return make_uint4(__funnelshift_r(lo.x, lo.y, r), __funnelshift_r(lo.y, lo.z, r), __funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r));
+    case 1: return make_uint4(__funnelshift_r(lo.y, lo.z, r), __funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r));
+    case 2: return make_uint4(__funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r), __funnelshift_r(hi.y, hi.z, r));
+    default: return make_uint4(__funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r), __funnelshift_r(hi.y, hi.z, r), __funnelshift_r(hi.z, hi.w, r));
+  }
+}
+
 // A 16-byte vector as VEC/2 pairs of fp32 values (bf16 -> fp32 is exact: a 16-bit shift).
 template <int DT> __device__ __forceinline__ float2 unpack_pair(const uint4& v, int k);
 template <> __device__ __forceinline__ float2 unpack_pair<0>(const uint4& v, int k) {

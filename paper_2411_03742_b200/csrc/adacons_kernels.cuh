@@ -14,6 +14,7 @@
 #include "adacons_common.cuh"
 #include "adacons_pass1.cuh"
 #include "adacons_gram.cuh"
+#include "adacons_shift.cuh"
 #include "adacons_coeff.cuh"
 #include "adacons_pass2.cuh"
 #include "adacons_fused.cuh"

@@ -553,22 +553,6 @@ pass2_generic_kernel(const void* __restrict__ grads, void* __restrict__ out, con
 // pass-2 kernels, so the bytes agree with theirs.  The body leaves out the first 16 to 31 bytes and
 // the last 16 to 31 bytes of the vector (edge_combine_kernel), so no load leaves a row.
 // ----------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {   // read-only path, L1 allocation allowed
-  uint4 v;
-  asm("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-  return v;
-}
-// bytes [shift, shift + 16) of the 32 bytes lo:hi; shift is a multiple of 2
-__device__ __forceinline__ uint4 realign_16(const uint4& lo, const uint4& hi, const int shift) {
-  const uint32_t r = static_cast<uint32_t>(shift & 3) * 8u;
-  switch (shift >> 2) {
-    case 0: return make_uint4(__funnelshift_r(lo.x, lo.y, r), __funnelshift_r(lo.y, lo.z, r), __funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r));
-    case 1: return make_uint4(__funnelshift_r(lo.y, lo.z, r), __funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r));
-    case 2: return make_uint4(__funnelshift_r(lo.z, lo.w, r), __funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r), __funnelshift_r(hi.y, hi.z, r));
-    default: return make_uint4(__funnelshift_r(lo.w, hi.x, r), __funnelshift_r(hi.x, hi.y, r), __funnelshift_r(hi.y, hi.z, r), __funnelshift_r(hi.z, hi.w, r));
-  }
-}
-
 constexpr int kPass2ShiftRows = 4;   // rows per batch: 2 * kPass2ShiftRows 16-byte loads in flight per thread
 
 // grads: byte address of element (0, 0); body_off: byte offset of the body's first column within a row;
@@ -619,31 +603,35 @@ pass2_shift_kernel(const unsigned char* __restrict__ grads, unsigned char* __res
 // Edges of a matrix whose rows start off a 16-byte boundary (every row by the same amount: the row
 // pitch is a multiple of 16 bytes).  The vectorised kernels then run on the aligned body -- from
 // each row's first 16-byte boundary on -- and these two one-block kernels do the few columns left:
-// edge_stats_kernel adds the first `head` (< 8) columns' share of Eq. 7 as one more partial record,
+// edge_stats_kernel adds the share of the first `head` and the last `tail` columns (24 in all at
+// most) in Eq. 7 as one more partial record,
 // edge_combine_kernel forms Eq. 12 for the first `head` and the last `tail` columns (32 in all at
 // most; element-wise, so nothing is read or written past the vector).
 // ----------------------------------------------------------------------------------------------
+constexpr int kEdgeCols = 24;   // most columns the statistics edge kernel takes (head + tail)
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
-edge_stats_kernel(const void* __restrict__ grads, int N, long long pitch, int head, float* __restrict__ record) {
-  __shared__ float x[kMaxFastN * 8];
-  __shared__ float s[8];
+edge_stats_kernel(const void* __restrict__ grads, int N, long long d, long long pitch, int head, int tail, float* __restrict__ record) {
+  __shared__ float x[kMaxFastN * kEdgeCols];
+  __shared__ float s[kEdgeCols];
   const int tid = threadIdx.x;
-  for (int idx = tid; idx < N * head; idx += kThreads) {
-    const int i = idx / head, k = idx - i * head;
-    x[i * 8 + k] = load_elem<DT>(grads, static_cast<long long>(i) * pitch + k);
+  const int cols = head + tail;                    // columns [0, head) and [d - tail, d)
+  for (int idx = tid; idx < N * cols; idx += kThreads) {
+    const int i = idx / cols, k = idx - i * cols;
+    const long long col = k < head ? k : d - tail + (k - head);
+    x[i * kEdgeCols + k] = load_elem<DT>(grads, static_cast<long long>(i) * pitch + col);
   }
   __syncthreads();
-  if (tid < head) {
+  if (tid < cols) {
     float a = 0.f;
-    for (int i = 0; i < N; ++i) a += x[i * 8 + tid];
+    for (int i = 0; i < N; ++i) a += x[i * kEdgeCols + tid];
     s[tid] = a;
   }
   __syncthreads();
   if (tid < N) {
     float pp = 0.f, qq = 0.f;
-    for (int k = 0; k < head; ++k) {
-      const float v = x[tid * 8 + k];
+    for (int k = 0; k < cols; ++k) {
+      const float v = x[tid * kEdgeCols + k];
       pp = fmaf(v, s[k], pp);
       qq = fmaf(v, v, qq);
     }

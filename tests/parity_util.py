@@ -154,3 +154,13 @@ def streamed_statistics(G, slab=2_000_000, threads=8):
     with ThreadPoolExecutor(max_workers=threads) as ex:
         parts = list(ex.map(one, starts))
     return sum(p for p, _ in parts), sum(q for _, q in parts)
+
+
+def shifted_pass1_applies(N, d, dtype, pitch=None):
+    """Whether pass 1 takes the per-class tensor maps (ADACONS_INFO_LAST_PATH 10) for rows `pitch` elements apart
+    that the staged kernels cannot take: up to 64 workers, a body of at least one 16-byte group, and classes of
+    rows thick enough (bf16 always; fp32 from 4 rows per class on, k = 16 / gcd(pitch in bytes, 16) classes)."""
+    eb = 4 if dtype == "f32" else 2
+    rem = ((pitch or d) * eb) % 16
+    k = 1 if rem == 0 else 16 // (rem & -rem)
+    return N <= 64 and d >= 4 * (16 // eb) and (dtype == "bf16" or N >= 4 * k)

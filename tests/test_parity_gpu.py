@@ -10,7 +10,7 @@ import torch
 from oracle import adacons_oracle as oc
 from paper_2411_03742_b200 import workloads as wl
 from parity_util import (COEFF_RTOL, OUT_TOL, ULP, assert_coeffs, assert_coeffs_by_set, assert_output, oracle_step,
-                         ranks_of, streamed_statistics, tally, to_f64, with_kernel_slot_order)
+                         ranks_of, shifted_pass1_applies, streamed_statistics, tally, to_f64, with_kernel_slot_order)
 
 pytestmark = pytest.mark.gpu
 
@@ -281,7 +281,7 @@ def test_single_column_has_tied_coefficients(ac):
 @pytest.mark.parametrize("aligned_body", [1, 0])
 def test_misaligned_base_pointer(ac, aligned_body):
     """A matrix that starts 4 bytes off a 16-byte boundary with a 16-byte pitch: pass 1 runs on the
-    aligned body plus the head columns (path 8), or on the generic kernels when that is switched off;
+    aligned body plus the head columns (path 8), or on tensor copies per row class, shifted into place in registers (path 10), when that is switched off;
     `out` is aligned here, i.e. off by another amount than the matrix, so pass 2 shifts its loads into place."""
     N, d = 6, 4096
     w = wl.Workload("mis", N, d, "f32", 1, "gauss", seed=3)
@@ -295,7 +295,7 @@ def test_misaligned_base_pointer(ac, aligned_body):
     h.set_option(ac.OPT_ALIGNED_BODY, aligned_body)
     h.aggregate(G, out)
     torch.cuda.synchronize()
-    assert h.info(ac.INFO_LAST_PATH) == (8 if aligned_body else 2) and h.info(ac.INFO_LAST_PASS2) == 6
+    assert h.info(ac.INFO_LAST_PATH) == (8 if aligned_body else 10) and h.info(ac.INFO_LAST_PASS2) == 6
     res = oc.AdaConsOracle(N, d).step(to_f64(G0), storage="f32")
     assert_coeffs(h.coeffs(ac.COEFF_GAMMA), res["gamma"], "gamma")
     assert_output(out, res, to_f64(G0), "f32", "misaligned")
@@ -398,9 +398,17 @@ def test_generic_and_fast_paths_agree(ac):
     h2.set_option(ac.OPT_ALIGNED_BODY, 0)
     h2.aggregate(G1, o2)
     torch.cuda.synchronize()
-    assert h2.info(ac.INFO_LAST_PATH) == 2
+    assert h2.info(ac.INFO_LAST_PATH) == 10
     np.testing.assert_allclose(h0.coeffs(), h2.coeffs(), rtol=2e-6)
     np.testing.assert_allclose(to_f64(o1), to_f64(o2), rtol=2e-2, atol=1e-6)
+    h3, o3 = ac.AdaCons(N, d, "bf16"), torch.empty(d, device="cuda:0", dtype=torch.bfloat16)
+    h3.set_option(ac.OPT_ALIGNED_BODY, 0)
+    h3.set_option(ac.OPT_SHIFTED_LOADS, 0)
+    h3.aggregate(G1, o3)
+    torch.cuda.synchronize()
+    assert h3.info(ac.INFO_LAST_PATH) == 2 and h3.info(ac.INFO_LAST_PASS2) == 1
+    np.testing.assert_allclose(h0.coeffs(), h3.coeffs(), rtol=2e-6)
+    np.testing.assert_allclose(to_f64(o1), to_f64(o3), rtol=2e-2, atol=1e-6)
 
 
 # ---- per-segment ("layer-wise") coefficients ----------------------------------------------------
@@ -944,7 +952,12 @@ def test_row_pitch_validation_and_unaligned_pitch(ac):
     h = ac.AdaCons(4, 1001, "f32")
     with pytest.raises(ac.AdaConsError):
         h.set_option(ac.OPT_ROW_PITCH, 1000)            # shorter than a row
-    _padded_case(ac, 4, 1001, "f32", 1003, 1, fused=True, expect_path=2)   # pitch not 16-byte: generic path
+    # a pitch that is not a multiple of 16 bytes: a tensor map per class of equally offset rows where the classes
+    # are thick enough, else the scalar pass 1; pass 2 with shifted loads either way
+    _padded_case(ac, 4, 1001, "f32", 1003, 1, fused=True, expect_path=2, expect_pass2=6)
+    _padded_case(ac, 16, 1001, "f32", 1003, 1, fused=True, expect_path=10, expect_pass2=6)
+    _padded_case(ac, 4, 1001, "bf16", 1003, 1, fused=True, expect_path=10, expect_pass2=6)
+    _padded_case(ac, 4, 1001, "bf16", 1003, 1, fused=True, options={ac.OPT_SHIFTED_LOADS: 0}, expect_path=2, expect_pass2=1)
 
 
 def test_host_entry_point_with_padded_rows(ac):
@@ -1287,7 +1300,7 @@ def test_gram_pass1_option_is_validated_and_ignored_where_it_does_not_apply(ac):
 
 
 # ---- rows at arbitrary element offsets: 16-byte loads shifted into place ---------------------------
-SHIFTED_CASES = [("f32", 8, 100_003, 0, 0), ("f32", 5, 70_001, 1, 2), ("f32", 16, 50_002, 3, 0), ("bf16", 16, 90_001, 0, 0),
+SHIFTED_CASES = [("f32", 8, 100_003, 0, 0), ("f32", 32, 60_001, 0, 0), ("f32", 64, 30_002, 1, 0), ("f32", 17, 44_445, 2, 3), ("f32", 5, 70_001, 1, 2), ("f32", 16, 50_002, 3, 0), ("bf16", 16, 90_001, 0, 0),
                  ("bf16", 7, 65_539, 1, 5), ("bf16", 64, 40_007, 3, 3), ("bf16", 3, 33, 1, 0), ("f32", 3, 16, 0, 1),
                  ("bf16", 100, 30_011, 2, 7), ("f32", 130, 20_001, 1, 1)]
 
@@ -1296,7 +1309,7 @@ SHIFTED_CASES = [("f32", 8, 100_003, 0, 0), ("f32", 5, 70_001, 1, 2), ("f32", 16
 def test_rows_at_arbitrary_offsets(ac, dtype, N, d, g_off, o_off):
     """Contiguous rows whose length is not a multiple of 16 bytes: every row starts at another offset
     from a 16-byte boundary, and so may the result.  The vector kernels shift each row's bytes into
-    place; the scalar kernels (option off) must give the same output bytes.  NaN all around the
+    place (pass 1 for N <= 64, pass 2 always); the scalar kernels (option off) must agree.  NaN all around the
     matrix and sentinels around the result: nothing outside is used or touched."""
     dev = torch.device("cuda:0")
     tdt = torch.float32 if dtype == "f32" else torch.bfloat16
@@ -1317,14 +1330,23 @@ def test_rows_at_arbitrary_offsets(ac, dtype, N, d, g_off, o_off):
         for h, o in zip(hs, outs):
             h.aggregate(G, o)
         torch.cuda.synchronize()
-        assert hs[0].info(ac.INFO_LAST_PASS2) == (6 if d >= 4 * (16 // eb) else 1) and hs[1].info(ac.INFO_LAST_PASS2) == 1
+        shifted = d >= 4 * (16 // eb)
+        assert hs[0].info(ac.INFO_LAST_PASS2) == (6 if shifted else 1) and hs[1].info(ac.INFO_LAST_PASS2) == 1
+        if (d * eb) % 16 == 0:                          # rows 16 bytes apart: the staged kernels apply (here only out is off)
+            want = 1 if (g_off * eb) % 16 == 0 else 8
+            assert hs[0].info(ac.INFO_LAST_PATH) == want and hs[1].info(ac.INFO_LAST_PATH) == want
+        else:
+            assert hs[0].info(ac.INFO_LAST_PATH) == (10 if shifted_pass1_applies(N, d, dtype) else 2) and hs[1].info(ac.INFO_LAST_PATH) == 2
         G64 = to_f64(G0)
         res = oracle_step(orc, G64, dtype, hs[0].coeffs(ac.COEFF_A), what=w.name)
         for k, code in (("p", ac.COEFF_P), ("q", ac.COEFF_Q), ("a", ac.COEFF_A), ("gamma", ac.COEFF_GAMMA)):
             assert_coeffs(hs[0].coeffs(code)[0], res[k][0], f"{w.name} {k} step {t}")
         assert_coeffs(hs[0].state()[0][0], res["m"][0], f"{w.name} m step {t}")
         assert_output(outs[0], res, G64, dtype, f"{w.name} step {t}")
-        assert torch.equal(outs[0].view(torch.uint8), outs[1].view(torch.uint8))
+        if hs[0].info(ac.INFO_LAST_PATH) == hs[1].info(ac.INFO_LAST_PATH):   # the same pass 1, hence the same weights: pass 2 must give the same bytes
+            assert torch.equal(outs[0].view(torch.uint8), outs[1].view(torch.uint8))
+        else:
+            np.testing.assert_allclose(hs[0].coeffs(), hs[1].coeffs(), rtol=4e-6, atol=1e-9)
         for b in obufs:
             assert bool((b[:o_off] == 7.0).all()) and bool((b[o_off + d:] == 7.0).all())
         assert bool(torch.isnan(gbuf[:g_off]).all()) and bool(torch.isnan(gbuf[g_off + N * d:]).all())
