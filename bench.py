@@ -351,7 +351,7 @@ def run_ours(args):
     status = h.status()
     assert status == 0, f"library raised status flags {status:#x}"
     path = h.info(ac.INFO_LAST_PATH)
-    assert path in (1, 3, 4, 5, 6, 7, 9), "benchmark must run an aligned path"
+    assert path in (1, 3, 4, 5, 6, 7, 9, 10), "benchmark must run a vectorised path"
 
     units_local = float(w.N) * w.d * args.steps
     ms, units = reduce_over_ranks(ms_local, units_local, device=dev)
@@ -407,6 +407,7 @@ def run_ours(args):
                             6: "N > 64: cluster pass 1 (one read), coefficient step, pass 2",
                             7: "64 < N <= 256: pass 1 on 128- or 256-row tiles (one read), coefficient step, pass 2",
                             9: "pass 1 from the Gram matrix on the tensor cores, coefficient step, pass 2",
+                            10: "rows at arbitrary offsets: pass 1 with a tensor map per row class, coefficient step, pass 2 with shifted loads",
                             5: "one launch, two reads (pass 1, coefficient step, pass 2 in one cooperative kernel)"}[path],
                    "l2": (f"inputs ({gbytes / 1e9:.2f} GB) larger than the 126 MB L2; no flush between steps" if nbuf == 1 else
                           f"two distinct input matrices of {gbytes / 1e9:.2f} GB used in turn, each larger than the 126 MB L2; no flush"
