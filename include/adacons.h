@@ -258,8 +258,9 @@ int adacons_create(adacons_ctx **out, int N, int64_t d, int dtype,
  *   N > 256 three times (column sums first, then dot products per 64 rows; needs d floats of
  *   scratch, allocated in adacons_create; see ADACONS_OPT_CLUSTER_PASS1).  A matrix that merely starts off a 16-byte
  *   boundary keeps the fast pass 1 (ADACONS_OPT_ALIGNED_BODY); a pitch that is not a multiple of
- *   16 bytes, or N > 64 with a misaligned base, is served by a slower generic path with the same
- *   results.
+ *   16 bytes (contiguous rows of an odd length) is still moved 16 bytes at a time, at about
+ *   two thirds of the aligned speed (ADACONS_OPT_SHIFTED_LOADS); scalar kernels serve what is
+ *   left (such a pitch with N > 64, vectors of a few elements) with the same results.
  * Enqueues its kernels on `cuda_stream` and returns; performs no host synchronisation and no
  * allocation.  Advances the momentum state by one step.  Owner of every buffer: the caller.
  * Errors: EINVAL (NULL pointers, overlap), ECUDA (launch failure), EALIGN (per-segment mode with
