@@ -402,6 +402,8 @@ def run_ours(args):
                                    "single GPU, the step in two halves (adacons_pass1, adacons_finish)" if args.column_sharded else
                                    "replicas only" if world > 1 else "single GPU"),
                    "coefficients": "per segment" if args.per_segment else "model-wise",
+                   "library_options": {k: v for k, v in (("one_launch", args.one_launch), ("cluster_pass1", args.cluster_pass1),
+                                                         ("tall_tiles", args.tall_tiles), ("gram_pass1", args.gram_pass1)) if v >= 0},
                    "path": {1: "three kernels (TMA-staged pass 1)", 3: "single-pass kernel (matrix in shared memory)",
                             4: "N > 64: column sums, dot products per 64 rows, pass 2 (three reads)",
                             6: "N > 64: cluster pass 1 (one read), coefficient step, pass 2",
