@@ -1353,3 +1353,33 @@ def test_rows_at_arbitrary_offsets(ac, dtype, N, d, g_off, o_off):
         assert hs[0].status() == 0
     for h in hs:
         h.close()
+
+
+def test_gram_pass1_sums_round_toward_zero(ac):
+    """Why the tensor-core pass 1 folds its accumulators: the tensor cores round their running sums
+    toward zero, so a sum of squares comes out LOW by an amount that grows with the number of chained
+    products (four per tile).  With one tile per fold the error is that of the fp32-pipe kernel; with 32
+    it is several 1e-6, still inside the 1e-5 tolerance.  Printed with -s for the record."""
+    dev = torch.device("cuda:0")
+    N, d = 64, 6_000_008
+    w = wl.Workload("gram-rounding", N, d, "bf16", 1, "student_flip", seed=5)
+    G = wl.generate(w, 0, dev)
+    p_or, q_or = streamed_statistics(G)
+    out = torch.empty(d, dtype=torch.bfloat16, device=dev)
+    bias = {}
+    for fold in (0, 1, 4, 16, 32):
+        h = ac.AdaCons(N, d, "bf16")
+        h.set_option(ac.OPT_ONE_LAUNCH, 0)
+        h.set_option(ac.OPT_GRAM_PASS1, fold)
+        h.aggregate(G, out)
+        torch.cuda.synchronize()
+        assert h.info(ac.INFO_LAST_PATH) == (9 if fold else 1)
+        q = h.coeffs(ac.COEFF_Q)[0]
+        p = h.coeffs(ac.COEFF_P)[0]
+        bias[fold] = float(np.mean((q - q_or) / q_or))
+        print(f"tiles per fold {fold:2d}: mean signed rel. error of q {bias[fold]:+.2e}, max |rel. error| of p "
+              f"{float(np.max(np.abs(p - p_or) / np.abs(p_or))):.2e}")
+        assert np.max(np.abs(q - q_or) / q_or) <= COEFF_RTOL
+        h.close()
+    assert abs(bias[1]) < 5e-7 and abs(bias[0]) < 5e-7
+    assert bias[32] < bias[16] < bias[4] < 0.0 and -1e-5 < bias[32] < -1e-6
