@@ -67,6 +67,8 @@ def parse_args(argv=None):
                     help="each rank holds its own d columns of ONE matrix of world*d columns: pass 1, an all-gather of the "
                          "statistics records, coefficient step and pass 2 (default for --gpus N > 1: independent replicas)")
     ap.add_argument("--gram-pass1", type=int, default=-1, help="ADACONS_OPT_GRAM_PASS1 (bf16, N <= 64): tiles per first-level sum; 0 = off")
+    ap.add_argument("--shifted-loads", type=int, default=-1, choices=[-1, 0, 1],
+                    help="ADACONS_OPT_SHIFTED_LOADS (rows at arbitrary element offsets, e.g. --shape with an odd d)")
     ap.add_argument("--one-launch", type=int, default=-1, choices=[-1, 0, 1, 2],
                     help="ADACONS_OPT_ONE_LAUNCH (default: the library's own choice by size)")
     return ap.parse_args(argv)
@@ -279,6 +281,8 @@ def run_ours(args):
         h.set_option(ac.OPT_CLUSTER_PASS1, args.cluster_pass1)
     if args.gram_pass1 >= 0:
         h.set_option(ac.OPT_GRAM_PASS1, args.gram_pass1)
+    if args.shifted_loads >= 0:
+        h.set_option(ac.OPT_SHIFTED_LOADS, args.shifted_loads)
     if args.tall_tiles >= 0:
         h.set_option(ac.OPT_TALL_TILES, args.tall_tiles)
     stream = torch.cuda.current_stream()
@@ -351,7 +355,7 @@ def run_ours(args):
     status = h.status()
     assert status == 0, f"library raised status flags {status:#x}"
     path = h.info(ac.INFO_LAST_PATH)
-    assert path in (1, 3, 4, 5, 6, 7, 9, 10), "benchmark must run a vectorised path"
+    assert path in (1, 3, 4, 5, 6, 7, 9, 10) or (path == 2 and args.shape), "a named workload must run a vectorised path"
 
     units_local = float(w.N) * w.d * args.steps
     ms, units = reduce_over_ranks(ms_local, units_local, device=dev)
@@ -403,12 +407,14 @@ def run_ours(args):
                                    "replicas only" if world > 1 else "single GPU"),
                    "coefficients": "per segment" if args.per_segment else "model-wise",
                    "library_options": {k: v for k, v in (("one_launch", args.one_launch), ("cluster_pass1", args.cluster_pass1),
-                                                         ("tall_tiles", args.tall_tiles), ("gram_pass1", args.gram_pass1)) if v >= 0},
+                                                         ("tall_tiles", args.tall_tiles), ("gram_pass1", args.gram_pass1),
+                                                         ("shifted_loads", args.shifted_loads)) if v >= 0},
                    "path": {1: "three kernels (TMA-staged pass 1)", 3: "single-pass kernel (matrix in shared memory)",
                             4: "N > 64: column sums, dot products per 64 rows, pass 2 (three reads)",
                             6: "N > 64: cluster pass 1 (one read), coefficient step, pass 2",
                             7: "64 < N <= 256: pass 1 on 128- or 256-row tiles (one read), coefficient step, pass 2",
                             9: "pass 1 from the Gram matrix on the tensor cores, coefficient step, pass 2",
+                            2: "scalar kernels (rows at arbitrary offsets, shifted loads switched off or not applicable)",
                             10: "rows at arbitrary offsets: pass 1 with a tensor map per row class, coefficient step, pass 2 with shifted loads",
                             5: "one launch, two reads (pass 1, coefficient step, pass 2 in one cooperative kernel)"}[path],
                    "l2": (f"inputs ({gbytes / 1e9:.2f} GB) larger than the 126 MB L2; no flush between steps" if nbuf == 1 else
